@@ -1,0 +1,350 @@
+"""Pins for the fp64 oracle: each check fixes a piece of oracle/admmq_oracle.py
+against something other than itself -- hand-worked values (tests/golden), closed
+forms, brute force on tiny inputs, library routines, and invariants the paper
+proves.  All CPU, no GPU, a few seconds each.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import scipy.linalg
+
+from oracle import admmq_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_kv(name):
+    out = {}
+    for line in open(os.path.join(GOLD, name)):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        k, *v = line.split()
+        out[k] = np.array([float(x) for x in v])
+    return out
+
+
+def _problem(n, p, N, seed, outliers=2, scale=20.0):
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((N, n))
+    X[:, rng.permutation(n)[:outliers]] *= scale
+    W = 0.02 * rng.standard_normal((p, n))
+    H = O.hessian_finalize(O.hessian_accumulate(None, X), N)
+    return X, W, H
+
+
+# ------------------------------------------------------------------ golden, hand-worked
+def test_w_update_hand_worked_2x2():
+    g = _read_kv("w_update_2x2.txt")
+    H = g["H"].reshape(2, 2)
+    lam, U = O.eig_factor(H)
+    Wh = g["W_hat"][None, :]
+    W = O.w_update(lam, U, Wh @ H, g["D"][None, :], g["V"][None, :], float(g["rho"][0]))
+    assert np.allclose(W[0], g["W"], rtol=0, atol=1e-14)
+    W2 = O.w_update_cholesky(H, Wh @ H, g["D"][None, :], g["V"][None, :], float(g["rho"][0]))
+    assert np.allclose(W2[0], g["W"], rtol=0, atol=1e-14)
+
+
+def test_projection_hand_worked():
+    rows = [l.split() for l in open(os.path.join(GOLD, "projection_cases.txt"))
+            if l.strip() and not l.startswith("#")]
+    wt = np.array([[float(r[0]) for r in rows]])
+    k, D = O.project(wt, np.full(len(rows), 2.0), np.array([[0.5]]), np.array([[-1.0]]), 2)
+    assert k[0].tolist() == [int(r[1]) for r in rows]
+    assert np.allclose(D[0], [float(r[2]) for r in rows], atol=1e-15)
+
+
+def test_move_cost_hand_worked():
+    g = _read_kv("move_cost_2x2.txt")
+    H = g["H"].reshape(2, 2)
+    # grid: Delta = 0.5, z0 = -1, 3 bits; W_q = [0.5, 0.0] (codes 3, 2); W_hat = W_q - eps
+    delta, z0 = np.array([[0.5]]), np.array([[-1.0]])
+    codes = np.array([[3, 2]], dtype=np.uint8)
+    Wq = O.dequantize(codes, delta, z0)
+    W_hat = Wq - g["eps"][None, :]
+    assert abs(O.objective(H, W_hat, Wq) - g["loss"][0]) < 1e-15
+    ls = O.local_search(H, W_hat, codes, delta, z0, bits=3, max_moves=1)
+    # the best single move is the hand-worked one (entry 0, -Delta): costs of the 4 candidates are
+    # (0,+): 2*.5*.75+.5 = 1.25 ; (0,-): -0.25 ; (1,+-): 0 +- 0 + .5 = 0.5
+    assert ls.codes.tolist() == [[2, 2]]
+    assert np.allclose(ls.g[0], g["g_new"], atol=1e-15)
+    assert abs(O.objective(H, W_hat, ls.Wq) - (g["loss"][0] + g["change"][0])) < 1e-15
+
+
+# ------------------------------------------------------------------ Hessian, damping, scaling
+def test_hessian_chunked_equals_one_shot_and_entry_definition():
+    rng = np.random.default_rng(1)
+    X = rng.standard_normal((300, 12))
+    Hc = None
+    for a in range(0, 300, 64):
+        Hc = O.hessian_accumulate(Hc, X[a:a + 64])
+    H1 = O.hessian_accumulate(None, X)
+    assert np.allclose(Hc, H1, rtol=1e-13, atol=1e-12)
+    # entry-by-entry definition H_ab = sum_t X_ta X_tb
+    for a, b in [(0, 0), (3, 7), (11, 2)]:
+        assert abs(H1[a, b] - sum(X[t, a] * X[t, b] for t in range(300))) < 1e-10
+
+
+def test_damping_is_one_percent_of_mean_diagonal():
+    rng = np.random.default_rng(2)
+    X = rng.standard_normal((50, 6))
+    Hr = O.hessian_accumulate(None, X)
+    H = O.hessian_finalize(Hr, 50, 0.01)
+    lam = 0.01 * np.mean(np.diag(Hr / 50))
+    assert np.allclose(H - Hr / 50, lam * np.eye(6), atol=1e-15)
+    Hl = O.hessian_finalize(Hr, 50, 0.01, literal_trace=True)
+    assert np.allclose(Hl - Hr / 50, 6 * lam * np.eye(6), atol=1e-14)
+    assert np.all(np.linalg.eigvalsh(H) > 0)
+
+
+def test_preconditioning_unit_diagonal_and_objective_identity():
+    _, W, H = _problem(16, 5, 200, 3)
+    s, Ht, Ws = O.precondition(H, W)
+    assert np.allclose(np.diag(Ht), 1.0, atol=1e-14)
+    assert np.all(np.linalg.eigvalsh(Ht) > 0)
+    # Eq. 3: the scaled objective equals the unscaled one for any candidate
+    rng = np.random.default_rng(4)
+    Wc = W + 0.01 * rng.standard_normal(W.shape)
+    unscaled = O.objective(H, W, Wc)
+    scaled = O.objective(Ht, Ws, Wc * s[None, :])
+    assert abs(unscaled - scaled) <= 1e-12 * abs(unscaled)
+
+
+# ------------------------------------------------------------------ grid and projection
+@pytest.mark.parametrize("bits,gs,sym", [(2, 0, True), (3, 4, False), (4, 8, False), (3, 8, True)])
+def test_grid_fit_brute_force(bits, gs, sym):
+    rng = np.random.default_rng(5)
+    W = rng.standard_normal((6, 16)) * 0.02
+    W[2, 4:8] = 0.0125  # a constant group
+    delta, z0 = O.grid_fit(W, bits, gs, sym)
+    g = 16 if gs == 0 else gs
+    L = (1 << bits) - 1
+    for j in range(6):
+        for q in range(16 // g):
+            blk = W[j, q * g:(q + 1) * g]
+            lo, hi = (-(np.abs(blk).max()), np.abs(blk).max()) if sym else (blk.min(), blk.max())
+            if hi == lo:
+                assert delta[j, q] == 1.0 and z0[j, q] == lo
+                continue
+            assert abs(delta[j, q] - (hi - lo) / L) < 1e-18 and z0[j, q] == lo
+            # every weight inside the grid's range, RTN error at most Delta/2
+            k, D = O.project(blk[None, :], np.ones(g), delta[j:j + 1, q:q + 1], z0[j:j + 1, q:q + 1], bits)
+            assert np.all(np.abs(D[0] - blk) <= delta[j, q] / 2 * (1 + 1e-12))
+
+
+def test_projection_is_nearest_grid_point_brute_force():
+    rng = np.random.default_rng(6)
+    p, n, bits, gs = 7, 24, 3, 8
+    W = rng.standard_normal((p, n)) * 0.02
+    delta, z0 = O.grid_fit(W, bits, gs, False)
+    s = np.exp(rng.standard_normal(n))
+    Wt = (W + 0.05 * rng.standard_normal((p, n))) * s[None, :]   # also exercises the clamp
+    k, D = O.project(Wt, s, delta, z0, bits)
+    for j in range(p):
+        for i in range(n):
+            levels = s[i] * (z0[j, i // gs] + delta[j, i // gs] * np.arange(1 << bits))
+            kb = int(np.argmin(np.abs(levels - Wt[j, i])))
+            assert kb == k[j, i] and abs(levels[kb] - D[j, i]) < 1e-15
+    assert k.max() == (1 << bits) - 1 and k.min() == 0
+
+
+# ------------------------------------------------------------------ W-update
+def test_w_update_solves_linear_system_and_matches_cholesky():
+    _, W, H = _problem(48, 9, 400, 7)
+    s, Ht, Ws = O.precondition(H, W)
+    lam, U = O.eig_factor(Ht)
+    rng = np.random.default_rng(8)
+    D = Ws + 0.01 * rng.standard_normal(Ws.shape)
+    V = 0.01 * rng.standard_normal(Ws.shape)
+    HW = Ws @ Ht
+    for rho in (1e-2, 0.1, 3.0, 1e4):
+        Wn = O.w_update(lam, U, HW, D, V, rho)
+        rhs = HW + rho * D - V
+        res = Wn @ (Ht + rho * np.eye(48)) - rhs          # transposed system
+        assert np.linalg.norm(res) <= 1e-10 * np.linalg.norm(rhs)
+        Wc = O.w_update_cholesky(Ht, HW, D, V, rho)
+        assert np.linalg.norm(Wn - Wc) <= 1e-10 * np.linalg.norm(Wc)
+        # and against an independent library solve of the untransposed system
+        Wl = np.linalg.solve(Ht + rho * np.eye(48), rhs.T).T
+        assert np.linalg.norm(Wn - Wl) <= 1e-10 * np.linalg.norm(Wl)
+
+
+# ------------------------------------------------------------------ ADMM as a whole
+def _rtn_codes(W, bits, gs, sym):
+    delta, z0 = O.grid_fit(W, bits, gs, sym)
+    n = W.shape[1]
+    k, _ = O.project(W, np.ones(n), delta, z0, bits)
+    return k
+
+
+@pytest.mark.parametrize("precond", [True, False])
+def test_first_iteration_is_rtn_for_any_hessian(precond):
+    _, W, H = _problem(32, 11, 300, 9)
+    a = O.admm(H, W, 3, 8, False, np.array([0.37]), precond=precond)
+    assert np.array_equal(a.codes, _rtn_codes(W, 3, 8, False))
+
+
+def test_key_inequality_feasibility_and_residual_trend():
+    _, W, H = _problem(40, 13, 500, 10, outliers=3)
+    bits, gs = 3, 8
+    rho = O.rho_schedule(120, 0.1, 1.1)
+    snaps = []
+    a = O.admm(H, W, bits, gs, False, rho, probe=lambda t, st: snaps.append(
+        (st["D"].copy(), st["V"].copy(), st["rho"], st["W"].copy())))
+    delta, z0 = O.grid_fit(W, bits, gs, False)
+    s = np.sqrt(np.diag(H))
+    for t in range(1, len(snaps)):
+        D_t, V_t, rt, W_t1 = snaps[t]
+        tgt = W_t1 + V_t / rt
+        _, D_t1 = O.project(tgt, s, delta, z0, bits)
+        # Eq. 15: the new projection is at least as close to the target as the old D
+        assert np.linalg.norm(D_t1 - tgt) <= np.linalg.norm(D_t - tgt) * (1 + 1e-12)
+        # feasibility: D^(t), t >= 1, is on the grid with codes in range
+        y = D_t / s[None, :]
+        kk = (y - O._expand(z0, 40)) / O._expand(delta, 40)
+        assert np.allclose(kk, np.rint(kk), atol=1e-8) and kk.min() > -1e-8 and kk.max() < 7 + 1e-8
+    # Theorem 1: rho_t * residual stays bounded; codes freeze once rho is large
+    tail = rho[60:] * np.maximum(a.r[60:], a.sres[60:])
+    assert tail.max() <= 50 * max(tail[0], 1e-12) + 1e-9
+    assert a.changed[-20:].sum() == 0
+    assert a.r[-1] < 1e-3 * a.r[1]
+
+
+def test_cholesky_route_gives_the_same_run():
+    _, W, H = _problem(24, 6, 300, 11)
+    rho = O.rho_schedule(30, 0.1, 1.3)
+    a = O.admm(H, W, 3, 0, False, rho)
+    b = O.admm(H, W, 3, 0, False, rho, use_cholesky=True)
+    assert np.array_equal(a.codes, b.codes)
+    assert np.allclose(a.r, b.r, rtol=1e-8, atol=1e-14)
+
+
+def test_diagonal_hessian_gives_rtn():
+    rng = np.random.default_rng(12)
+    n, p, bits = 24, 9, 3
+    W = 0.02 * rng.standard_normal((p, n))
+    H = np.diag(np.exp(rng.standard_normal(n)))
+    rtn = _rtn_codes(W, bits, 0, False)
+    # (a) ADMM alone with rho_t >= 1 for every t
+    a = O.admm(H, W, bits, 0, False, O.rho_schedule(40, 1.0, 1.2))
+    assert np.array_equal(a.codes, rtn)
+    # (b) any schedule followed by local search run to convergence
+    res = O.quantize_layer(H, W, bits, 0, False, O.rho_schedule(60, 0.01, 1.2))
+    assert np.array_equal(res.ls.codes, rtn)
+    # (c) a single iteration
+    assert np.array_equal(O.admm(H, W, bits, 0, False, np.array([0.05])).codes, rtn)
+
+
+def test_fine_grid_limit_stays_next_to_dense_weights():
+    # b = 8 on a per-channel grid: the constraint is nearly inactive, so ADMM on the strongly
+    # convex quadratic must end within two grid steps of W_hat (the unconstrained minimiser)
+    # in every entry -- a dropped term or wrong sign in the W- or V-update drifts far away.
+    _, W, H = _problem(20, 5, 200, 13)
+    a = O.admm(H, W, 8, 0, False, O.rho_schedule(150, 0.1, 1.1))
+    assert np.all(np.abs(a.Wq - W) <= 2.0 * a.delta)
+    # and with the grid made of W_hat's own values (caller grid, Delta -> levels hit W_hat exactly)
+    # the fixed point is W_hat itself: codes of RTN, zero error
+    delta, z0 = O.grid_fit(W, 8, 0, False)
+    Wg = O.dequantize(_rtn_codes(W, 8, 0, False), delta, z0)           # weights already on the grid
+    b = O.admm(H, Wg, 8, 0, False, O.rho_schedule(60, 0.1, 1.2), grid=(delta, z0))
+    assert np.allclose(b.Wq, Wg, atol=1e-15) and b.r[-1] < 1e-9
+
+
+def test_admm_beats_rtn_on_outlier_problem():
+    _, W, H = _problem(64, 32, 2000, 14, outliers=3)
+    res = O.quantize_layer(H, W, 3, 0, False, O.rho_schedule(150, 0.1, 1.1))
+    rtn = O.dequantize(_rtn_codes(W, 3, 0, False), *O.grid_fit(W, 3, 0, False))
+    e_rtn = O.objective(H, W, rtn)
+    assert res.err_admm < e_rtn
+    assert res.err_final <= res.err_admm
+
+
+# ------------------------------------------------------------------ local search
+def test_local_search_invariants():
+    _, W, H = _problem(32, 10, 300, 15)
+    delta, z0 = O.grid_fit(W, 3, 8, False)
+    codes = _rtn_codes(W, 3, 8, False)
+    e0 = O.objective(H, W, O.dequantize(codes, delta, z0))
+    prev = e0
+    cur = codes
+    total = 0
+    for _ in range(400):                      # one move at a time: strictly decreasing objective
+        ls = O.local_search(H, W, cur, delta, z0, 3, max_moves=1)
+        if ls.moves.sum() == 0:
+            break
+        e = O.objective(H, W, ls.Wq)
+        assert e < prev
+        # each column's decrease equals the closed-form cost of its move (checked in aggregate)
+        prev, cur = e, ls.codes
+        total += int(ls.moves.sum())
+    full = O.local_search(H, W, codes, delta, z0, 3)
+    assert np.array_equal(full.codes, cur) and int(full.moves.sum()) == total
+    # maintained gradient equals the recomputed one
+    assert np.allclose(full.g, (full.Wq - W) @ H, rtol=1e-10, atol=1e-12)
+    # identity E = sum_j eps_j . g_j
+    assert abs(np.sum((full.Wq - W) * full.g) - O.objective(H, W, full.Wq)) < 1e-12 * e0
+    assert np.array_equal(full.Wq, O.dequantize(full.codes, delta, z0)) or \
+        np.allclose(full.Wq, O.dequantize(full.codes, delta, z0), atol=1e-15)
+
+
+def test_local_search_closed_form_cost_vs_recomputed_loss():
+    _, W, H = _problem(12, 4, 100, 16)
+    delta, z0 = O.grid_fit(W, 2, 0, False)
+    codes = _rtn_codes(W, 2, 0, False)
+    Wq = O.dequantize(codes, delta, z0)
+    g = (Wq - W) @ H
+    for j in range(4):
+        e0 = (Wq[j] - W[j]) @ H @ (Wq[j] - W[j])
+        for i in range(12):
+            for sg in (+1, -1):
+                d = sg * delta[j, 0]
+                w2 = Wq[j].copy()
+                w2[i] += d
+                e1 = (w2 - W[j]) @ H @ (w2 - W[j])
+                assert abs((e1 - e0) - (2 * d * g[j, i] + d * d * H[i, i])) < 1e-12 * max(e0, 1e-30) + 1e-18
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_local_search_brute_force_tiny(seed):
+    """d_in = 8, 2 bits: enumerate all 4^8 assignments per column."""
+    n, p, bits = 8, 3, 2
+    _, W, H = _problem(n, p, 64, 100 + seed, outliers=1, scale=5.0)
+    res = O.quantize_layer(H, W, bits, 0, False, O.rho_schedule(40, 0.05, 1.3))
+    delta, z0 = res.admm.delta, res.admm.z0
+    all_codes = np.array(list(itertools.product(range(4), repeat=n)))       # [65536, 8]
+    tau = 1e-6
+    for j in range(p):
+        cand = z0[j, 0] + delta[j, 0] * all_codes                            # [65536, 8]
+        E = cand - W[j][None, :]
+        loss = np.einsum("ci,ik,ck->c", E, H, E)
+        mine = res.ls.codes[j].astype(int)
+        idx = int(np.dot(mine, 4 ** np.arange(n - 1, -1, -1)))
+        assert np.array_equal(all_codes[idx], mine)
+        my_loss = loss[idx]
+        assert my_loss >= loss.min() - 1e-15
+        # 1-move local optimum: no neighbour (one code +-1) improves by more than the threshold
+        for i in range(n):
+            for sg in (+1, -1):
+                nb = mine.copy()
+                nb[i] += sg
+                if nb[i] < 0 or nb[i] > 3:
+                    continue
+                nidx = int(np.dot(nb, 4 ** np.arange(n - 1, -1, -1)))
+                assert loss[nidx] >= my_loss - tau * H[i, i] * delta[j, 0] ** 2 - 1e-15
+        # local search never made the column worse than the ADMM point
+        aidx = int(np.dot(res.admm.codes[j].astype(int), 4 ** np.arange(n - 1, -1, -1)))
+        assert my_loss <= loss[aidx] + 1e-15
+
+
+def test_local_search_respects_move_cap_and_bounds():
+    _, W, H = _problem(16, 6, 100, 17)
+    delta, z0 = O.grid_fit(W, 2, 0, False)
+    rng = np.random.default_rng(18)
+    codes = rng.integers(0, 4, size=(6, 16)).astype(np.uint8)      # a poor start: many moves
+    ls = O.local_search(H, W, codes, delta, z0, 2, max_moves=3)
+    assert ls.moves.max() <= 3 and ls.capped.any()
+    full = O.local_search(H, W, codes, delta, z0, 2)
+    assert full.codes.max() <= 3 and not full.capped.any()
+    assert O.objective(H, W, full.Wq) < O.objective(H, W, O.dequantize(codes, delta, z0))
