@@ -1,0 +1,189 @@
+/*
+ * admmq.h -- C ABI of the B200 (sm_100a) ADMM-Q layer-wise quantization solver.
+ *
+ * The library solves, for one linear layer,
+ *     min_W  Tr((W - W_hat)^T H (W - W_hat))   s.t.  W on a low-bit uniform grid,
+ *     H = X^T X / N + lambda I                                        (Eq. 1, Eq. 2)
+ * by the operator-splitting iteration of Algorithm 1 followed by a greedy
+ * local search (Sec. 3.5).  Paper notation: n = d_in (input channels, size of H),
+ * p = d_out (output channels), N = calibration rows.
+ *
+ * Conventions shared by every call
+ *  - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller owns
+ *    every buffer, including the workspace; the library never allocates or frees
+ *    device memory (admmq_create allocates only a small host struct).
+ *  - Every n-by-p matrix of the paper (W_hat, codes, W_q) is passed TRANSPOSED as a
+ *    row-major [d_out][d_in] array (the layout of a linear layer's weight): row j is
+ *    output channel j, input channels are contiguous.
+ *  - Work is enqueued on the CUDA stream given to admmq_create and is asynchronous
+ *    unless a call says that it synchronises.  No call throws, aborts or traps.
+ *  - Argument, shape and call-order errors are returned at once, with nothing
+ *    enqueued.  Numerical failures found on the device (non-finite input, a
+ *    non-positive Hessian diagonal or pivot, a wait that ran out) are recorded in a
+ *    device status word: admmq_last_device_status synchronises and returns it, and a
+ *    call given a non-NULL host report returns it too.  Outputs are unspecified
+ *    after an error.
+ *  - Device pointers must be 16-byte aligned; d_in must be a multiple of 8 and at
+ *    most ADMMQ_MAX_D_IN; d_in must be a multiple of the group size.
+ *  - Call order: create -> hessian_reset -> hessian_accumulate* -> factor ->
+ *    (quantize_layer -> local_search)* -> destroy.  Several weight matrices that
+ *    share one H may reuse one factor.  A call out of order returns ADMMQ_ERR_STATE.
+ */
+#ifndef ADMMQ_H_
+#define ADMMQ_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ADMMQ_MAX_D_IN 14336
+#define ADMMQ_MAX_BITS 8
+
+typedef struct admmq_ctx admmq_ctx; /* opaque */
+
+typedef enum {
+  ADMMQ_OK = 0,
+  ADMMQ_ERR_INVALID_ARG = 1,  /* NULL pointer, bad enum, bad struct_size, misaligned pointer */
+  ADMMQ_ERR_SHAPE = 2,        /* sizes outside the supported range or not divisible as required */
+  ADMMQ_ERR_STATE = 3,        /* call out of order */
+  ADMMQ_ERR_WORKSPACE = 4,    /* workspace too small */
+  ADMMQ_ERR_NOT_SPD = 5,      /* non-positive Hessian diagonal or pivot (device status) */
+  ADMMQ_ERR_NONFINITE = 6,    /* NaN/Inf met in H or W_hat (device status) */
+  ADMMQ_ERR_TIMEOUT = 7,      /* a bounded device-side wait ran out (device status) */
+  ADMMQ_ERR_CUDA = 8,         /* a CUDA runtime/driver call failed */
+  ADMMQ_ERR_UNSUPPORTED = 9,  /* valid request that this build does not implement */
+  ADMMQ_WARN_MOVE_CAP = 10    /* local search stopped at max_moves_per_col in some column */
+} admmq_status;
+
+typedef enum { ADMMQ_F32 = 0, ADMMQ_BF16 = 1 } admmq_dtype;
+
+/* How the product (H~ + rho I)^{-1} of the W-update (Eq. 7) is applied.
+ * TRIDIAG: one orthogonal reduction H~ = Q T Q^T (T tridiagonal), reused for every rho, with an O(n)
+ *          LDL^T of T + rho I per penalty value -- the role the single eigendecomposition plays in
+ *          Algorithm 1 line 3.  The only kind implemented. */
+typedef enum { ADMMQ_FACTOR_TRIDIAG = 0, ADMMQ_FACTOR_CHOLESKY = 1, ADMMQ_FACTOR_EIG = 2 } admmq_factor_kind;
+
+/* Which matrix-product kernels run.  TENSOR: tcgen05 tensor-core kernels on split-bf16 operands with
+ * fp32 accumulation (the product path).  SIMT: plain fp32 FMA kernels on the same operands, kept as an
+ * on-device cross-check. */
+typedef enum { ADMMQ_GEMM_TENSOR = 0, ADMMQ_GEMM_SIMT = 1 } admmq_gemm_kind;
+
+const char* admmq_status_string(admmq_status s);
+
+/* Bytes of device workspace a context needs for layers with d_in input channels, at most d_out_max
+ * output channels and at most T_max ADMM iterations.  Returns 0 for unsupported sizes. */
+size_t admmq_workspace_bytes(int d_in, int d_out_max, int T_max);
+
+/* Creates a context for one value of d_in.  d_workspace: device memory of at least
+ * admmq_workspace_bytes(...) bytes, 256-byte aligned, owned by the caller and kept alive until
+ * admmq_destroy.  cuda_stream: a cudaStream_t (NULL = the default stream).  Synchronous. */
+admmq_status admmq_create(admmq_ctx** ctx, int d_in, int d_out_max, int T_max, void* d_workspace,
+                          size_t workspace_bytes, void* cuda_stream);
+admmq_status admmq_destroy(admmq_ctx* ctx); /* frees the host struct only */
+admmq_status admmq_set_gemm_kind(admmq_ctx* ctx, admmq_gemm_kind kind);
+
+/* Synchronises the stream and returns the device status word (ADMMQ_OK if none was raised). */
+admmq_status admmq_last_device_status(admmq_ctx* ctx);
+
+/* ---- Step 1: Hessian accumulation, H_raw += X^T X, N += n_tokens  (Sec. 3.1: H = X^T X). ----------
+ * d_X: [n_tokens][ldx] row-major, dtype fp32 or bf16; the first d_in columns of each row are used;
+ * ldx >= d_in, and ldx * sizeof(element) a multiple of 16.  Only read.  May be called any number of
+ * times after admmq_hessian_reset; accumulation is in fp32. */
+admmq_status admmq_hessian_reset(admmq_ctx* ctx);
+admmq_status admmq_hessian_accumulate(admmq_ctx* ctx, const void* d_X, admmq_dtype dtype,
+                                      long long n_tokens, long long ldx);
+/* Alternative to accumulation: the caller supplies the UNDAMPED Hessian X^T X / N directly
+ * (Algorithm 1 takes H as its input).  d_H: [d_in][d_in] fp32, symmetric.  Counts as N = 1. */
+admmq_status admmq_hessian_set(admmq_ctx* ctx, const float* d_H);
+
+/* ---- Step 2: damping, diagonal scaling, factorisation. ---------------------------------------------
+ * H = H_raw / N + damp_frac * mean(diag(H_raw / N)) I                         (App. D, damping)
+ * s_i = sqrt(H_ii),  H~ = diag(1/s) H diag(1/s)                   (Sec. 3.2; Algorithm 1 lines 1-2)
+ * then the one-time factorisation of H~ (Algorithm 1 line 3) and the per-penalty factors for
+ * rho[0..T).  rho: HOST array of T penalties, or NULL for rho0 * gamma^t (Sec. 3.6). */
+typedef struct {
+  size_t struct_size;     /* sizeof(admmq_factor_cfg) */
+  double damp_frac;       /* 0.01 in the paper */
+  int precondition;       /* 1: diagonal scaling on (paper default); 0: s_i = 1 */
+  int kind;               /* admmq_factor_kind */
+  int T;                  /* number of ADMM iterations, 1..T_max */
+  const double* h_rho;    /* host array [T] or NULL */
+  double rho0, gamma;     /* used when h_rho == NULL */
+} admmq_factor_cfg;
+admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg);
+
+/* ---- Step 3: the ADMM loop (Algorithm 1 lines 4-11; Eq. 7-10). -------------------------------------
+ * d_W0: pre-trained weights [d_out][d_in] fp32 (unscaled), only read.
+ * Outputs, caller-allocated:
+ *   d_codes [d_out][d_in] uint8     codes k of D^(T), 0 <= k <= 2^bits - 1
+ *   d_scale, d_zero [d_out][d_in/group] fp32   grid Delta and z0 (inputs when use_caller_grid)
+ *   d_Wq [d_out][d_in] fp32 or NULL  W_q = z0 + Delta * k  (Algorithm 1 line 11)
+ *   d_resid [T][2] fp32 or NULL      (||W^(t+1) - D^(t+1)||_F, ||D^(t+1) - D^(t)||_F), Theorem 1
+ * The grid is the min-max grid of the unscaled weights (Sec. 3.4): asymmetric lo = min, hi = max;
+ * symmetric hi = max|w|, lo = -hi; Delta = (hi - lo)/(2^bits - 1), z0 = lo; Delta = 1 for a constant
+ * group.  Rounding is to nearest, ties to even, then clamped to the grid's range.
+ * h_report NULL: nothing is synchronised.  Non-NULL: the call synchronises, fills the report and
+ * returns the device status. */
+typedef struct {
+  size_t struct_size;   /* sizeof(admmq_quant_cfg) */
+  int bits;             /* 2..8 */
+  int group_size;       /* along d_in; 0 or d_in: one group per output channel */
+  int symmetric;        /* 0 asymmetric, 1 symmetric */
+  int use_caller_grid;  /* 1: d_scale / d_zero are inputs */
+} admmq_quant_cfg;
+typedef struct {
+  double err_before;    /* Tr(E^T H E), E = W_q - W_hat, at entry (local search) / of the ADMM result */
+  double err_after;     /* same, at exit (local search only; = err_before for quantize_layer) */
+  long long moves;      /* local-search moves applied, all columns */
+  int iters_run;        /* ADMM iterations run */
+  int capped_columns;   /* columns that hit max_moves_per_col */
+  float ms;             /* device time of the call, CUDA events */
+} admmq_report;
+admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out,
+                                  const admmq_quant_cfg* cfg, unsigned char* d_codes, float* d_scale,
+                                  float* d_zero, float* d_Wq, float* d_resid, admmq_report* h_report);
+
+/* One W-update (Eq. 7) from a caller-supplied state, for step-by-step checking:
+ * d_codes [d_out][d_in] uint8 defines D = s * (z0 + Delta k); d_V [d_out][d_in] fp32 is the dual in
+ * scaled coordinates; d_W_out [d_out][d_in] fp32 receives W^(t+1) (scaled coordinates).  Needs a prior
+ * admmq_factor; the penalty may be any rho > 0 (its per-penalty factor is computed on the fly). */
+admmq_status admmq_w_update(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
+                            const unsigned char* d_codes, const float* d_scale, const float* d_zero,
+                            const float* d_V, double rho, float* d_W_out);
+
+/* ---- Step 4: local search (Sec. 3.5, Eq. 11 restricted to one perturbed entry). --------------------
+ * Every output channel independently: with g = H (W_q - W_hat) (unscaled damped H held by the
+ * context), moving entry i by d = +-Delta changes the loss by c = 2 d g_i + d^2 H_ii.  The move of
+ * smallest c that keeps the code in range (ties: smallest i, then +Delta first) is applied while
+ * c < -accept_tol * H_ii * Delta^2, then g += d H[:, i].  Codes (and d_Wq if non-NULL) are updated in
+ * place.  Returns ADMMQ_WARN_MOVE_CAP (a success) through the report path if a column hit the cap. */
+typedef struct {
+  size_t struct_size;           /* sizeof(admmq_ls_cfg) */
+  int bits;
+  int group_size;
+  long long max_moves_per_col;  /* 0: 8 * d_in */
+  double accept_tol;            /* relative threshold tau; the paper gives none, 1e-6 by default */
+} admmq_ls_cfg;
+admmq_status admmq_local_search(admmq_ctx* ctx, const float* d_W0, int d_out, const admmq_ls_cfg* cfg,
+                                unsigned char* d_codes, const float* d_scale, const float* d_zero,
+                                float* d_Wq, admmq_report* h_report);
+
+/* Tr(E^T H E) with E = (z0 + Delta k) - W_hat and the unscaled damped H (Eq. 2 without the 1/2, as in
+ * Sec. 3.5).  Synchronises; the value is written to *h_err (host). */
+admmq_status admmq_objective(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
+                             const unsigned char* d_codes, const float* d_scale, const float* d_zero,
+                             double* h_err);
+
+/* Copies of internal state for checking (synchronise).  d_H_out [d_in][d_in] fp32: the damped unscaled
+ * H; d_s_out [d_in] fp32: s_i = sqrt(H_ii) (1 when preconditioning is off).  Either may be NULL. */
+admmq_status admmq_get_hessian(admmq_ctx* ctx, float* d_H_out, float* d_s_out);
+
+/* Number of kernels this context has launched so far (host counter). */
+long long admmq_launch_count(const admmq_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADMMQ_H_ */

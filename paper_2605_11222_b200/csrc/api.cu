@@ -1,0 +1,469 @@
+// extern "C" entry points of libadmmq: argument checks, workspace carve-up and the host-side
+// sequencing of the kernels.  All numerical work runs in the CUDA kernels of this library.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "../../include/admmq.h"
+#include "internal.h"
+
+using namespace admmq;
+
+struct admmq_ctx {
+  Ctx c;
+  double* rho_dev = nullptr;
+  long long* d_moves = nullptr;
+  int* d_capped = nullptr;
+  int slots_cap = 0;
+  double rho_adhoc = 0.0;
+};
+
+namespace {
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Carver {
+  char* base;
+  size_t off = 0;
+  template <typename T>
+  T* take(size_t count) {
+    off = align_up(off, 256);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+int slots_cap_for(int n, int p) {
+  const int simt = ((p + 63) / 64) * ((n + 63) / 64);
+  return simt > 256 ? simt : 256;
+}
+
+// Lays the workspace out; with base == nullptr only measures it.
+size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
+  Carver cv{base};
+  Ctx dummy;
+  Ctx& c = a ? a->c : dummy;
+  const size_t nn = (size_t)n * n, pn = (size_t)p * n;
+  c.status = cv.take<int>(64);
+  c.scal = cv.take<double>(32);
+  long long* moves = cv.take<long long>(8);
+  int* capped = cv.take<int>(16);
+  double* rho_dev = cv.take<double>((size_t)T + 1);
+  c.H_raw = cv.take<float>(nn);
+  c.H = cv.take<float>(nn);
+  c.s = cv.take<float>(n);
+  c.hdiag = cv.take<float>(n);
+  c.A64 = cv.take<double>(nn);
+  c.P64 = cv.take<double>(nn);
+  c.td = cv.take<double>(n);
+  c.te = cv.take<double>(n);
+  c.beta = cv.take<double>(n);
+  c.pvec = cv.take<double>(n);
+  c.stage_l = cv.take<double>((size_t)(T + 1) * n);
+  c.stage_invd = cv.take<double>((size_t)(T + 1) * n);
+  c.Q_hi = cv.take<bf16>(nn);
+  c.Q_lo = cv.take<bf16>(nn);
+  c.QT_hi = cv.take<bf16>(nn);
+  c.QT_lo = cv.take<bf16>(nn);
+  c.H_hi = cv.take<bf16>(nn);
+  c.H_lo = cv.take<bf16>(nn);
+  c.Whs = cv.take<float>(pn);
+  c.V = cv.take<float>(pn);
+  c.Y = cv.take<float>(pn);
+  c.R_hi = cv.take<bf16>(pn);
+  c.R_lo = cv.take<bf16>(pn);
+  c.Y_hi = cv.take<bf16>(pn);
+  c.Y_lo = cv.take<bf16>(pn);
+  const int slots = slots_cap_for(n, p);
+  c.partials = cv.take<float>((size_t)T * slots * 2);
+  c.partial_slots = slots;
+  c.XT_hi = cv.take<bf16>((size_t)n * XT_ROWS);
+  c.XT_lo = cv.take<bf16>((size_t)n * XT_ROWS);
+  if (a) {
+    a->rho_dev = rho_dev;
+    a->d_moves = moves;
+    a->d_capped = capped;
+    a->slots_cap = slots;
+  }
+  return align_up(cv.off, 256);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool sizes_ok(int d_in, int d_out, int T) {
+  return d_in >= 8 && d_in <= ADMMQ_MAX_D_IN && (d_in % 8) == 0 && d_out >= 1 && d_out <= (1 << 20) &&
+         T >= 1 && T <= 4096;
+}
+
+cudaError_t product(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiParams& e) {
+  return c->gemm_kind == ADMMQ_GEMM_SIMT ? gemm_simt(c, A, B, M, N, K, e) : gemm_tc(c, A, B, M, N, K, e);
+}
+
+admmq_status read_status(admmq_ctx* a) {
+  int st = 0;
+  if (cudaStreamSynchronize(a->c.stream) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  if (cudaMemcpy(&st, a->c.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  if (cudaGetLastError() != cudaSuccess) return ADMMQ_ERR_CUDA;
+  return (admmq_status)st;
+}
+
+int group_of(int d_in, int gs) { return (gs == 0 || gs == d_in) ? d_in : gs; }
+
+// g = E H with E = W_q - W_hat, into c->Y; E planes go through the R buffers.
+cudaError_t gradient(admmq_ctx* a, const float* W0, int p, int gs, const unsigned char* codes,
+                     const float* delta, const float* zero) {
+  Ctx* c = &a->c;
+  launch_error_planes(c, W0, p, gs, codes, delta, zero, c->R_hi, c->R_lo);
+  EpiParams e{};
+  e.kind = EPI_STORE;
+  e.C = c->Y;
+  e.ldc = c->n;
+  return product(c, Planes{c->R_hi, c->R_lo, c->n}, Planes{c->H_hi, c->H_lo, c->n}, p, c->n, c->n, e);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* admmq_status_string(admmq_status s) {
+  switch (s) {
+    case ADMMQ_OK: return "ok";
+    case ADMMQ_ERR_INVALID_ARG: return "invalid argument";
+    case ADMMQ_ERR_SHAPE: return "unsupported shape";
+    case ADMMQ_ERR_STATE: return "call out of order";
+    case ADMMQ_ERR_WORKSPACE: return "workspace too small";
+    case ADMMQ_ERR_NOT_SPD: return "Hessian not positive definite";
+    case ADMMQ_ERR_NONFINITE: return "non-finite value in the input";
+    case ADMMQ_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case ADMMQ_ERR_CUDA: return "CUDA call failed";
+    case ADMMQ_ERR_UNSUPPORTED: return "not implemented in this build";
+    case ADMMQ_WARN_MOVE_CAP: return "local search stopped at the move cap";
+  }
+  return "unknown status";
+}
+
+size_t admmq_workspace_bytes(int d_in, int d_out_max, int T_max) {
+  if (!sizes_ok(d_in, d_out_max, T_max)) return 0;
+  return carve(nullptr, nullptr, d_in, d_out_max, T_max);
+}
+
+admmq_status admmq_create(admmq_ctx** ctx, int d_in, int d_out_max, int T_max, void* d_workspace,
+                          size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx || !d_workspace) return ADMMQ_ERR_INVALID_ARG;
+  *ctx = nullptr;
+  if (!sizes_ok(d_in, d_out_max, T_max)) return ADMMQ_ERR_SHAPE;
+  if (reinterpret_cast<uintptr_t>(d_workspace) & 255u) return ADMMQ_ERR_INVALID_ARG;
+  if (workspace_bytes < admmq_workspace_bytes(d_in, d_out_max, T_max)) return ADMMQ_ERR_WORKSPACE;
+  admmq_ctx* a = new (std::nothrow) admmq_ctx();
+  if (!a) return ADMMQ_ERR_CUDA;
+  a->c.n = d_in;
+  a->c.p_max = d_out_max;
+  a->c.T_max = T_max;
+  a->c.stream = (cudaStream_t)cuda_stream;
+  a->c.ws = (char*)d_workspace;
+  a->c.ws_bytes = workspace_bytes;
+  carve(a, (char*)d_workspace, d_in, d_out_max, T_max);
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+    delete a;
+    return ADMMQ_ERR_CUDA;
+  }
+  a->c.num_sms = sms;
+  if (cudaMemsetAsync(a->c.status, 0, 256, a->c.stream) != cudaSuccess) {
+    delete a;
+    return ADMMQ_ERR_CUDA;
+  }
+  *ctx = a;
+  return ADMMQ_OK;
+}
+
+admmq_status admmq_destroy(admmq_ctx* ctx) {
+  if (!ctx) return ADMMQ_ERR_INVALID_ARG;
+  delete ctx;
+  return ADMMQ_OK;
+}
+
+admmq_status admmq_set_gemm_kind(admmq_ctx* ctx, admmq_gemm_kind kind) {
+  if (!ctx || (kind != ADMMQ_GEMM_TENSOR && kind != ADMMQ_GEMM_SIMT)) return ADMMQ_ERR_INVALID_ARG;
+  ctx->c.gemm_kind = (int)kind;
+  return ADMMQ_OK;
+}
+
+admmq_status admmq_last_device_status(admmq_ctx* ctx) {
+  if (!ctx) return ADMMQ_ERR_INVALID_ARG;
+  return read_status(ctx);
+}
+
+long long admmq_launch_count(const admmq_ctx* ctx) { return ctx ? ctx->c.launches : 0; }
+
+admmq_status admmq_hessian_reset(admmq_ctx* ctx) {
+  if (!ctx) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  launch_zero(c, c->H_raw, (size_t)c->n * c->n * sizeof(float));
+  launch_zero(c, c->status, 256);
+  c->n_tokens = 0;
+  c->state = 1;
+  return cudaGetLastError() == cudaSuccess ? ADMMQ_OK : ADMMQ_ERR_CUDA;
+}
+
+admmq_status admmq_hessian_accumulate(admmq_ctx* ctx, const void* d_X, admmq_dtype dtype,
+                                      long long n_tokens, long long ldx) {
+  if (!ctx || !d_X || !aligned16(d_X)) return ADMMQ_ERR_INVALID_ARG;
+  if (dtype != ADMMQ_F32 && dtype != ADMMQ_BF16) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (c->state != 1) return ADMMQ_ERR_STATE;
+  const size_t esz = dtype == ADMMQ_BF16 ? 2 : 4;
+  if (n_tokens < 0 || ldx < c->n || ((size_t)ldx * esz) % 16 != 0) return ADMMQ_ERR_SHAPE;
+  const int n = c->n;
+  for (long long r0 = 0; r0 < n_tokens; r0 += XT_ROWS) {
+    const long long rows = (n_tokens - r0 < XT_ROWS) ? (n_tokens - r0) : XT_ROWS;
+    const char* xp = (const char*)d_X + (size_t)r0 * ldx * esz;
+    bf16* lo = dtype == ADMMQ_BF16 ? nullptr : c->XT_lo;
+    launch_transpose_split(c, xp, dtype == ADMMQ_BF16, rows, ldx, n, c->XT_hi, lo, XT_ROWS);
+    EpiParams e{};
+    e.kind = EPI_ACCUM;
+    e.C = c->H_raw;
+    e.ldc = n;
+    e.lower_only = 1;
+    Planes P{c->XT_hi, lo, XT_ROWS};
+    if (product(c, P, P, n, n, (int)rows, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  }
+  c->n_tokens += n_tokens;
+  return cudaGetLastError() == cudaSuccess ? ADMMQ_OK : ADMMQ_ERR_CUDA;
+}
+
+admmq_status admmq_hessian_set(admmq_ctx* ctx, const float* d_H) {
+  if (!ctx || !d_H || !aligned16(d_H)) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (cudaMemcpyAsync(c->H_raw, d_H, (size_t)c->n * c->n * sizeof(float), cudaMemcpyDeviceToDevice,
+                      c->stream) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  launch_zero(c, c->status, 256);
+  c->n_tokens = 1;
+  c->state = 1;
+  return ADMMQ_OK;
+}
+
+admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg) {
+  if (!ctx || !cfg || cfg->struct_size != sizeof(admmq_factor_cfg)) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (c->state < 1 || c->n_tokens < 1) return ADMMQ_ERR_STATE;
+  if (cfg->kind == ADMMQ_FACTOR_CHOLESKY || cfg->kind == ADMMQ_FACTOR_EIG) return ADMMQ_ERR_UNSUPPORTED;
+  if (cfg->kind != ADMMQ_FACTOR_TRIDIAG) return ADMMQ_ERR_INVALID_ARG;
+  if (cfg->T < 1 || cfg->T > c->T_max) return ADMMQ_ERR_SHAPE;
+  if (!(cfg->damp_frac >= 0.0) || !isfinite(cfg->damp_frac)) return ADMMQ_ERR_INVALID_ARG;
+  for (int t = 0; t < cfg->T; ++t) {
+    const double r = cfg->h_rho ? cfg->h_rho[t] : cfg->rho0 * pow(cfg->gamma, (double)t);
+    if (!(r > 0.0) || !isfinite(r)) return ADMMQ_ERR_INVALID_ARG;
+    c->rho_host[t] = r;
+  }
+  c->T = cfg->T;
+  c->precondition = cfg->precondition ? 1 : 0;
+  const int n = c->n;
+  launch_finalize(c, cfg->damp_frac, c->precondition);
+  launch_split_f32(c, c->H, (long long)n * n, c->H_hi, c->H_lo);
+  if (tridiag_reduce(c) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  if (tridiag_form_qt(c) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  launch_split_f64(c, c->P64, n, c->QT_hi, c->QT_lo, c->Q_hi, c->Q_lo);
+  if (cudaMemcpyAsync(ctx->rho_dev, c->rho_host, sizeof(double) * c->T, cudaMemcpyHostToDevice,
+                      c->stream) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  launch_stage_factors(c, ctx->rho_dev, 0, c->T);
+  if (cudaGetLastError() != cudaSuccess) return ADMMQ_ERR_CUDA;
+  c->state = 2;
+  return ADMMQ_OK;
+}
+
+static admmq_status check_layer_args(admmq_ctx* ctx, const float* d_W0, int d_out, int bits, int group_size,
+                                     const void* codes, const void* scale, const void* zero) {
+  if (!ctx || !d_W0 || !codes || !scale || !zero) return ADMMQ_ERR_INVALID_ARG;
+  if (!aligned16(d_W0) || !aligned16(codes) || !aligned16(scale) || !aligned16(zero))
+    return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (c->state != 2) return ADMMQ_ERR_STATE;
+  if (d_out < 1 || d_out > c->p_max) return ADMMQ_ERR_SHAPE;
+  if (bits < 2 || bits > ADMMQ_MAX_BITS) return ADMMQ_ERR_SHAPE;
+  if (group_size < 0 || group_size > c->n) return ADMMQ_ERR_SHAPE;
+  const int gs = group_of(c->n, group_size);
+  if (c->n % gs != 0) return ADMMQ_ERR_SHAPE;
+  return ADMMQ_OK;
+}
+
+// One W-update in the error form of Eq. 7:  W - W_hat' = Q (T/rho + I)^{-1} Q^T R,
+// R = D - V/rho - W_hat'.  Product 1 -> solve -> product 2 (whose epilogue is `epi`).
+static cudaError_t w_update_products(Ctx* c, int p, int stage, const EpiParams& epi) {
+  const int n = c->n;
+  EpiParams e1{};
+  e1.kind = EPI_STORE;
+  e1.C = c->Y;
+  e1.ldc = n;
+  cudaError_t err = product(c, Planes{c->R_hi, c->R_lo, n}, Planes{c->QT_hi, c->QT_lo, n}, p, n, n, e1);
+  if (err != cudaSuccess) return err;
+  launch_tridiag_solve(c, p, stage);
+  return product(c, Planes{c->Y_hi, c->Y_lo, n}, Planes{c->Q_hi, c->Q_lo, n}, p, n, n, epi);
+}
+
+admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, const admmq_quant_cfg* cfg,
+                                  unsigned char* d_codes, float* d_scale, float* d_zero, float* d_Wq,
+                                  float* d_resid, admmq_report* h_report) {
+  if (!cfg || cfg->struct_size != sizeof(admmq_quant_cfg)) return ADMMQ_ERR_INVALID_ARG;
+  admmq_status st = check_layer_args(ctx, d_W0, d_out, cfg->bits, cfg->group_size, d_codes, d_scale, d_zero);
+  if (st != ADMMQ_OK) return st;
+  if ((d_Wq && !aligned16(d_Wq)) || (d_resid && !aligned16(d_resid))) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  const int n = c->n, p = d_out, gs = group_of(n, cfg->group_size), T = c->T;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  if (h_report) {
+    if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return ADMMQ_ERR_CUDA;
+    cudaEventRecord(ev0, c->stream);
+  }
+  if (!cfg->use_caller_grid) launch_grid_fit(c, d_W0, p, cfg->bits, gs, cfg->symmetric, d_scale, d_zero);
+  launch_scale_weights(c, d_W0, p);                        // W_hat', V = 0, R = 0 (Algorithm 1 l.2, l.4)
+  launch_zero(c, c->partials, (size_t)T * c->partial_slots * 2 * sizeof(float));
+  EpiParams e{};
+  e.kind = EPI_ADMM;
+  e.Whs = c->Whs;
+  e.V = c->V;
+  e.codes = d_codes;
+  e.s = c->s;
+  e.delta = d_scale;
+  e.zero = d_zero;
+  e.group_size = gs;
+  e.n_groups = n / gs;
+  e.kmax = (1 << cfg->bits) - 1;
+  e.Rhi = c->R_hi;
+  e.Rlo = c->R_lo;
+  for (int t = 0; t < T; ++t) {
+    const double rho = c->rho_host[t];
+    const double rho_next = (t + 1 < T) ? c->rho_host[t + 1] : rho;
+    e.first_iter = (t == 0);
+    e.rho = (float)rho;
+    e.inv_rho = (float)(1.0 / rho);
+    e.inv_rho_next = (float)(1.0 / rho_next);
+    e.partials = c->partials + (size_t)t * c->partial_slots * 2;
+    if (w_update_products(c, p, t, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  }
+  if (d_resid) launch_reduce_partials(c, T, d_resid);
+  if (d_Wq) launch_dequant(c, p, gs, d_codes, d_scale, d_zero, d_Wq);
+  if (cudaGetLastError() != cudaSuccess) return ADMMQ_ERR_CUDA;
+  if (!h_report) return ADMMQ_OK;
+  cudaEventRecord(ev1, c->stream);
+  memset(h_report, 0, sizeof(*h_report));
+  if (gradient(ctx, d_W0, p, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 1);
+  st = read_status(ctx);
+  double err = 0.0;
+  cudaMemcpy(&err, c->scal + 1, sizeof(double), cudaMemcpyDeviceToHost);
+  cudaEventElapsedTime(&h_report->ms, ev0, ev1);
+  cudaEventDestroy(ev0);
+  cudaEventDestroy(ev1);
+  h_report->err_before = err;
+  h_report->err_after = err;
+  h_report->iters_run = T;
+  return st;
+}
+
+admmq_status admmq_w_update(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
+                            const unsigned char* d_codes, const float* d_scale, const float* d_zero,
+                            const float* d_V, double rho, float* d_W_out) {
+  admmq_status st = check_layer_args(ctx, d_W0, d_out, 2, group_size, d_codes, d_scale, d_zero);
+  if (st != ADMMQ_OK) return st;
+  if (!d_V || !d_W_out || !aligned16(d_V) || !aligned16(d_W_out)) return ADMMQ_ERR_INVALID_ARG;
+  if (!(rho > 0.0) || !isfinite(rho)) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  const int n = c->n, p = d_out, gs = group_of(n, group_size);
+  launch_scale_weights(c, d_W0, p);
+  launch_init_rhs(c, p, gs, d_codes, d_scale, d_zero, d_V, (float)(1.0 / rho));
+  const int stage = c->T_max;                              // spare slot for an ad-hoc penalty
+  ctx->rho_adhoc = rho;
+  if (cudaMemcpyAsync(ctx->rho_dev + stage, &ctx->rho_adhoc, sizeof(double), cudaMemcpyHostToDevice,
+                      c->stream) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  launch_stage_factors(c, ctx->rho_dev, stage, 1);
+  EpiParams e{};
+  e.kind = EPI_WOUT;
+  e.C = d_W_out;
+  e.ldc = n;
+  e.Whs = c->Whs;
+  if (w_update_products(c, p, stage, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? ADMMQ_OK : ADMMQ_ERR_CUDA;
+}
+
+admmq_status admmq_local_search(admmq_ctx* ctx, const float* d_W0, int d_out, const admmq_ls_cfg* cfg,
+                                unsigned char* d_codes, const float* d_scale, const float* d_zero,
+                                float* d_Wq, admmq_report* h_report) {
+  if (!cfg || cfg->struct_size != sizeof(admmq_ls_cfg)) return ADMMQ_ERR_INVALID_ARG;
+  admmq_status st = check_layer_args(ctx, d_W0, d_out, cfg->bits, cfg->group_size, d_codes, d_scale, d_zero);
+  if (st != ADMMQ_OK) return st;
+  if (d_Wq && !aligned16(d_Wq)) return ADMMQ_ERR_INVALID_ARG;
+  if (cfg->max_moves_per_col < 0 || !(cfg->accept_tol >= 0.0)) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  const int n = c->n, p = d_out, gs = group_of(n, cfg->group_size);
+  const long long cap = cfg->max_moves_per_col > 0 ? cfg->max_moves_per_col : 8LL * n;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  if (h_report) {
+    if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return ADMMQ_ERR_CUDA;
+    cudaEventRecord(ev0, c->stream);
+  }
+  if (gradient(ctx, d_W0, p, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  if (h_report) launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 1);
+  launch_zero(c, ctx->d_moves, 64);
+  launch_zero(c, ctx->d_capped, 64);
+  if (launch_local_search(c, d_W0, p, cfg->bits, gs, cap, (float)cfg->accept_tol, d_codes, d_scale, d_zero,
+                          d_Wq, c->Y, ctx->d_moves, ctx->d_capped) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  if (!h_report) return ADMMQ_OK;
+  cudaEventRecord(ev1, c->stream);
+  memset(h_report, 0, sizeof(*h_report));
+  if (gradient(ctx, d_W0, p, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 2);
+  st = read_status(ctx);
+  double errs[2] = {0, 0};
+  long long moves = 0;
+  int capped = 0;
+  cudaMemcpy(errs, c->scal + 1, 2 * sizeof(double), cudaMemcpyDeviceToHost);
+  cudaMemcpy(&moves, ctx->d_moves, sizeof(long long), cudaMemcpyDeviceToHost);
+  cudaMemcpy(&capped, ctx->d_capped, sizeof(int), cudaMemcpyDeviceToHost);
+  cudaEventElapsedTime(&h_report->ms, ev0, ev1);
+  cudaEventDestroy(ev0);
+  cudaEventDestroy(ev1);
+  h_report->err_before = errs[0];
+  h_report->err_after = errs[1];
+  h_report->moves = moves;
+  h_report->capped_columns = capped;
+  if (st == ADMMQ_OK && capped > 0) st = ADMMQ_WARN_MOVE_CAP;
+  return st;
+}
+
+admmq_status admmq_objective(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
+                             const unsigned char* d_codes, const float* d_scale, const float* d_zero,
+                             double* h_err) {
+  admmq_status st = check_layer_args(ctx, d_W0, d_out, 2, group_size, d_codes, d_scale, d_zero);
+  if (st != ADMMQ_OK) return st;
+  if (!h_err) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  const int gs = group_of(c->n, group_size);
+  if (gradient(ctx, d_W0, d_out, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  launch_objective_dot(c, d_W0, d_out, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 1);
+  st = read_status(ctx);
+  if (cudaMemcpy(h_err, c->scal + 1, sizeof(double), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  return st;
+}
+
+admmq_status admmq_get_hessian(admmq_ctx* ctx, float* d_H_out, float* d_s_out) {
+  if (!ctx) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (c->state != 2) return ADMMQ_ERR_STATE;
+  if (d_H_out && cudaMemcpyAsync(d_H_out, c->H, (size_t)c->n * c->n * sizeof(float),
+                                 cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  if (d_s_out && cudaMemcpyAsync(d_s_out, c->s, (size_t)c->n * sizeof(float), cudaMemcpyDeviceToDevice,
+                                 c->stream) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  return read_status(ctx);
+}
+
+}  // extern "C"

@@ -1,0 +1,364 @@
+// Bandwidth-bound kernels of the ADMM-Q path: layout changes, Hessian finalisation (damping, diagonal
+// scaling), grid fit, operand splitting and the small reductions.
+#include "internal.h"
+
+namespace admmq {
+
+#define LAUNCH(c) ((c)->launches++)
+
+void launch_zero(Ctx* c, void* ptr, size_t bytes) { cudaMemsetAsync(ptr, 0, bytes, c->stream); }
+
+// ------------------------------------------------------------------------------------------------
+// X chunk [rows][ldx] -> X^T planes [n][ldt] (token index contiguous), so that the Hessian product
+// H_raw += X^T X contracts over a contiguous index.  fp32 input is split into two bf16 planes.
+// ------------------------------------------------------------------------------------------------
+template <typename TIn>
+__global__ void transpose_split_kernel(const TIn* __restrict__ X, long long rows, long long ldx, int n,
+                                       bf16* __restrict__ Thi, bf16* __restrict__ Tlo, long long ldt) {
+  __shared__ float tile[32][33];
+  const long long r0 = (long long)blockIdx.x * 32;
+  const int c0 = blockIdx.y * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const long long r = r0 + i;
+    const int cc = c0 + threadIdx.x;
+    float v = 0.f;
+    if (r < rows && cc < n) {
+      if constexpr (sizeof(TIn) == 2) v = __bfloat162float(X[r * ldx + cc]);
+      else v = X[r * ldx + cc];
+    }
+    tile[i][threadIdx.x] = v;
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int cc = c0 + i;
+    const long long r = r0 + threadIdx.x;
+    if (cc < n && r < rows) {
+      const float v = tile[threadIdx.x][i];
+      if (Tlo) {
+        bf16 hi, lo;
+        split_bf16(v, hi, lo);
+        Thi[(long long)cc * ldt + r] = hi;
+        Tlo[(long long)cc * ldt + r] = lo;
+      } else {
+        Thi[(long long)cc * ldt + r] = __float2bfloat16_rn(v);
+      }
+    }
+  }
+}
+
+void launch_transpose_split(Ctx* c, const void* X, int is_bf16, long long rows, long long ldx, int n,
+                            bf16* XT_hi, bf16* XT_lo, long long ldt) {
+  dim3 grid((unsigned)((rows + 31) / 32), (unsigned)((n + 31) / 32)), block(32, 8);
+  if (is_bf16)
+    transpose_split_kernel<bf16><<<grid, block, 0, c->stream>>>((const bf16*)X, rows, ldx, n, XT_hi,
+                                                                nullptr, ldt);
+  else
+    transpose_split_kernel<float><<<grid, block, 0, c->stream>>>((const float*)X, rows, ldx, n, XT_hi,
+                                                                 XT_lo, ldt);
+  LAUNCH(c);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Finalisation: H = H_raw/N + damp * mean(diag(H_raw/N)) I (App. D), s_i = sqrt(H_ii),
+// H~ = diag(1/s) H diag(1/s) in fp64 (Sec. 3.2).  H_raw holds the lower triangle.
+// ------------------------------------------------------------------------------------------------
+__global__ void diag_sum_kernel(const float* __restrict__ Hraw, int n, double inv_N, double* out) {
+  __shared__ double scratch[32];
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) acc += (double)Hraw[(long long)i * n + i] * inv_N;
+  acc = block_sum(acc, scratch);
+  if (threadIdx.x == 0) out[0] = acc;
+}
+
+__global__ void finalize_diag_kernel(const float* __restrict__ Hraw, int n, double inv_N,
+                                     double damp_frac, int precondition, const double* __restrict__ dsum,
+                                     float* __restrict__ hdiag, float* __restrict__ s, double* s64,
+                                     int* status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const double lam = damp_frac * dsum[0] / n;
+  const float hii = (float)((double)Hraw[(long long)i * n + i] * inv_N + lam);
+  hdiag[i] = hii;
+  if (!(hii > 0.f) || !isfinite(hii)) {
+    raise_status(status, isfinite(hii) ? ST_NOT_SPD : ST_NONFINITE);
+    s[i] = 1.f;
+    s64[i] = 1.0;
+    return;
+  }
+  const double sv = precondition ? sqrt((double)hii) : 1.0;
+  s64[i] = sv;
+  s[i] = (float)sv;
+}
+
+__global__ void finalize_full_kernel(const float* __restrict__ Hraw, int n, double inv_N,
+                                     const float* __restrict__ hdiag, const double* __restrict__ s64,
+                                     float* __restrict__ H, double* __restrict__ A64, int* status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  const int a = blockIdx.y;
+  if (b >= n) return;
+  const int lo = min(a, b), hi = max(a, b);
+  float h = (float)((double)Hraw[(long long)hi * n + lo] * inv_N);
+  if (a == b) h = hdiag[a];
+  if (!isfinite(h)) raise_status(status, ST_NONFINITE);
+  H[(long long)a * n + b] = h;
+  A64[(long long)a * n + b] = (double)h / (s64[a] * s64[b]);
+}
+
+void launch_finalize(Ctx* c, double damp_frac, int precondition) {
+  const int n = c->n;
+  const double inv_N = 1.0 / (double)c->n_tokens;
+  double* s64 = c->pvec;  // scratch [n]; consumed before the reduction starts
+  diag_sum_kernel<<<1, 1024, 0, c->stream>>>(c->H_raw, n, inv_N, c->scal);
+  LAUNCH(c);
+  finalize_diag_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(c->H_raw, n, inv_N, damp_frac,
+                                                              precondition, c->scal, c->hdiag, c->s,
+                                                              s64, c->status);
+  LAUNCH(c);
+  dim3 grid((n + 255) / 256, n);
+  finalize_full_kernel<<<grid, 256, 0, c->stream>>>(c->H_raw, n, inv_N, c->hdiag, s64, c->H, c->A64,
+                                                    c->status);
+  LAUNCH(c);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Grid fit (Sec. 3.4: Delta = (max - min)/(2^b - 1); Sec. 3.5: levels z0 + k Delta): one warp per
+// (output channel, group) of the unscaled weights.
+// ------------------------------------------------------------------------------------------------
+__global__ void grid_fit_kernel(const float* __restrict__ W0, int p, int n, int gs, int levels,
+                                int symmetric, float* __restrict__ delta, float* __restrict__ zero) {
+  const int ng = n / gs;
+  const long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (gw >= (long long)p * ng) return;
+  const int j = (int)(gw / ng), g = (int)(gw % ng);
+  const float* w = W0 + (long long)j * n + (long long)g * gs;
+  float lo = INFINITY, hi = -INFINITY;
+  for (int i = lane; i < gs; i += 32) {
+    const float v = w[i];
+    lo = fminf(lo, v);
+    hi = fmaxf(hi, v);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+  }
+  if (lane == 0) {
+    if (symmetric) {
+      hi = fmaxf(fabsf(lo), fabsf(hi));
+      lo = -hi;
+    }
+    float d = (hi - lo) / (float)levels;
+    if (hi - lo == 0.f) d = 1.f;
+    delta[gw] = d;
+    zero[gw] = lo;
+  }
+}
+
+void launch_grid_fit(Ctx* c, const float* W0, int p, int bits, int gs, int symmetric, float* delta,
+                     float* zero) {
+  const long long warps = (long long)p * (c->n / gs);
+  const int threads = 256;
+  const long long blocks = (warps * 32 + threads - 1) / threads;
+  grid_fit_kernel<<<(unsigned)blocks, threads, 0, c->stream>>>(W0, p, c->n, gs, (1 << bits) - 1,
+                                                                symmetric, delta, zero);
+  LAUNCH(c);
+}
+
+// W_hat' = Sigma^{-1} W_hat (Algorithm 1 line 2); V^(0) = 0; first right-hand side R = D^(0) - W_hat' = 0.
+__global__ void scale_weights_kernel(const float* __restrict__ W0, const float* __restrict__ s,
+                                     long long total, int n, float* __restrict__ Whs,
+                                     float* __restrict__ V, bf16* __restrict__ Rhi,
+                                     bf16* __restrict__ Rlo, int* status) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const float w = W0[i];
+  if (!isfinite(w)) raise_status(status, ST_NONFINITE);
+  Whs[i] = s[i % n] * w;
+  V[i] = 0.f;
+  Rhi[i] = __float2bfloat16_rn(0.f);
+  Rlo[i] = __float2bfloat16_rn(0.f);
+}
+
+void launch_scale_weights(Ctx* c, const float* W0, int p) {
+  const long long total = (long long)p * c->n;
+  scale_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
+      W0, c->s, total, c->n, c->Whs, c->V, c->R_hi, c->R_lo, c->status);
+  LAUNCH(c);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Operand splitting: fp64 / fp32 matrices -> (hi, lo) bf16 planes, optionally also transposed.
+// ------------------------------------------------------------------------------------------------
+__global__ void split_f64_kernel(const double* __restrict__ src, int n, bf16* __restrict__ hi,
+                                 bf16* __restrict__ lo, bf16* __restrict__ thi, bf16* __restrict__ tlo) {
+  __shared__ float tile[32][33];
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int r = r0 + i, cc = c0 + threadIdx.x;
+    float v = 0.f;
+    if (r < n && cc < n) {
+      v = (float)src[(long long)r * n + cc];
+      bf16 h, l;
+      split_bf16(v, h, l);
+      hi[(long long)r * n + cc] = h;
+      lo[(long long)r * n + cc] = l;
+    }
+    tile[i][threadIdx.x] = v;
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int cc = c0 + i, r = r0 + threadIdx.x;   // element (r, cc) of src -> (cc, r) of the transpose
+    if (cc < n && r < n) {
+      bf16 h, l;
+      split_bf16(tile[threadIdx.x][i], h, l);
+      thi[(long long)cc * n + r] = h;
+      tlo[(long long)cc * n + r] = l;
+    }
+  }
+}
+
+void launch_split_f64(Ctx* c, const double* src, int n, bf16* hi, bf16* lo, bf16* thi, bf16* tlo) {
+  dim3 grid((n + 31) / 32, (n + 31) / 32), block(32, 8);
+  split_f64_kernel<<<grid, block, 0, c->stream>>>(src, n, hi, lo, thi, tlo);
+  LAUNCH(c);
+}
+
+__global__ void split_f32_kernel(const float* __restrict__ src, long long count, bf16* __restrict__ hi,
+                                 bf16* __restrict__ lo) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  bf16 h, l;
+  split_bf16(src[i], h, l);
+  hi[i] = h;
+  lo[i] = l;
+}
+
+void launch_split_f32(Ctx* c, const float* src, long long count, bf16* hi, bf16* lo) {
+  split_f32_kernel<<<(unsigned)((count + 255) / 256), 256, 0, c->stream>>>(src, count, hi, lo);
+  LAUNCH(c);
+}
+
+// Right-hand side of the error-form W-update from a caller-supplied state:
+// R = D - V/rho - W_hat', D = s (z0 + Delta k).
+__global__ void init_rhs_kernel(long long total, int n, int gs, int ng,
+                                const unsigned char* __restrict__ codes,
+                                const float* __restrict__ delta, const float* __restrict__ zero,
+                                const float* __restrict__ V, float inv_rho, const float* __restrict__ s,
+                                const float* __restrict__ Whs, bf16* __restrict__ Rhi,
+                                bf16* __restrict__ Rlo) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int col = (int)(idx % n);
+  const long long row = idx / n;
+  const long long gi = row * ng + col / gs;
+  const float d = s[col] * (zero[gi] + delta[gi] * (float)codes[idx]);
+  const float r = d - V[idx] * inv_rho - Whs[idx];
+  bf16 h, l;
+  split_bf16(r, h, l);
+  Rhi[idx] = h;
+  Rlo[idx] = l;
+}
+
+void launch_init_rhs(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
+                     const float* zero, const float* V_in, float inv_rho) {
+  const long long total = (long long)p * c->n;
+  init_rhs_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
+      total, c->n, gs, c->n / gs, codes, delta, zero, V_in, inv_rho, c->s, c->Whs, c->R_hi, c->R_lo);
+  LAUNCH(c);
+}
+
+// Fixed-order second stage of the residual sums: resid[t] = (sqrt(sum (W-D)^2), sqrt(sum (D-D_old)^2)).
+__global__ void reduce_partials_kernel(const float* __restrict__ partials, int slots, int T,
+                                       float* __restrict__ resid) {
+  __shared__ double scratch[32];
+  const int t = blockIdx.x;
+  if (t >= T) return;
+  double a = 0.0, b = 0.0;
+  for (int i = threadIdx.x; i < slots; i += blockDim.x) {
+    a += (double)partials[((long long)t * slots + i) * 2 + 0];
+    b += (double)partials[((long long)t * slots + i) * 2 + 1];
+  }
+  a = block_sum(a, scratch);
+  b = block_sum(b, scratch);
+  if (threadIdx.x == 0) {
+    resid[2 * t + 0] = (float)sqrt(a);
+    resid[2 * t + 1] = (float)sqrt(b);
+  }
+}
+
+void launch_reduce_partials(Ctx* c, int T, float* resid) {
+  reduce_partials_kernel<<<T, 128, 0, c->stream>>>(c->partials, c->partial_slots, T, resid);
+  LAUNCH(c);
+}
+
+// W_q = z0 + Delta k (Algorithm 1 line 11, unscaled coordinates).
+__global__ void dequant_kernel(long long total, int n, int gs, int ng,
+                               const unsigned char* __restrict__ codes, const float* __restrict__ delta,
+                               const float* __restrict__ zero, float* __restrict__ Wq) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const long long gi = (idx / n) * ng + (idx % n) / gs;
+  Wq[idx] = zero[gi] + delta[gi] * (float)codes[idx];
+}
+
+void launch_dequant(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
+                    const float* zero, float* Wq) {
+  const long long total = (long long)p * c->n;
+  dequant_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(total, c->n, gs, c->n / gs,
+                                                                         codes, delta, zero, Wq);
+  LAUNCH(c);
+}
+
+// E = W_q - W_hat as two bf16 planes (operand of the gradient product g = E H, Sec. 3.5).
+__global__ void error_planes_kernel(long long total, int n, int gs, int ng, const float* __restrict__ W0,
+                                    const unsigned char* __restrict__ codes,
+                                    const float* __restrict__ delta, const float* __restrict__ zero,
+                                    bf16* __restrict__ Ehi, bf16* __restrict__ Elo) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const long long gi = (idx / n) * ng + (idx % n) / gs;
+  const float e = (zero[gi] + delta[gi] * (float)codes[idx]) - W0[idx];
+  bf16 h, l;
+  split_bf16(e, h, l);
+  Ehi[idx] = h;
+  Elo[idx] = l;
+}
+
+void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes,
+                         const float* delta, const float* zero, bf16* Ehi, bf16* Elo) {
+  const long long total = (long long)p * c->n;
+  error_planes_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
+      total, c->n, gs, c->n / gs, W0, codes, delta, zero, Ehi, Elo);
+  LAUNCH(c);
+}
+
+// sum_j eps_j . g_j  =  Tr(E^T H E)  when g = H E  (fp64 accumulation).
+__global__ void objective_dot_kernel(long long total, int n, int gs, int ng, const float* __restrict__ W0,
+                                     const unsigned char* __restrict__ codes,
+                                     const float* __restrict__ delta, const float* __restrict__ zero,
+                                     const float* __restrict__ g, double* out) {
+  __shared__ double scratch[32];
+  double acc = 0.0;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const long long gi = (idx / n) * ng + (idx % n) / gs;
+    const float e = (zero[gi] + delta[gi] * (float)codes[idx]) - W0[idx];
+    acc += (double)e * (double)g[idx];
+  }
+  acc = block_sum(acc, scratch);
+  if (threadIdx.x == 0) atomicAdd(out, acc);
+}
+
+void launch_objective_dot(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes,
+                          const float* delta, const float* zero, const float* g, double* out) {
+  const long long total = (long long)p * c->n;
+  cudaMemsetAsync(out, 0, sizeof(double), c->stream);
+  long long blocks = (total + 255) / 256;
+  if (blocks > 4 * 148) blocks = 4 * 148;
+  objective_dot_kernel<<<(unsigned)blocks, 256, 0, c->stream>>>(total, c->n, gs, c->n / gs, W0, codes,
+                                                                delta, zero, g, out);
+  LAUNCH(c);
+}
+
+}  // namespace admmq

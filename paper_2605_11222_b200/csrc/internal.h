@@ -1,0 +1,103 @@
+// Host-side declarations shared by the translation units of libadmmq.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "epilogue.cuh"
+
+namespace admmq {
+
+typedef __nv_bfloat16 bf16;
+
+// One operand of a product C = A * B^T: up to two bf16 planes (hi, lo) whose sum is the value.
+// Row-major [rows][ld], the contraction index contiguous ("K-major").
+struct Planes {
+  const bf16* hi;
+  const bf16* lo;   // nullptr: single plane
+  long long ld;
+};
+
+struct Ctx {
+  int n = 0, p_max = 0, T_max = 0;
+  cudaStream_t stream = nullptr;
+  int num_sms = 148;
+  int gemm_kind = 0;
+  int state = 0;            // 0 created, 1 hessian open, 2 factored
+  long long n_tokens = 0;
+  int T = 0;
+  int precondition = 1;
+  double rho_host[4096];
+  long long launches = 0;
+  // ---- workspace carve-up (device) ----
+  char* ws = nullptr;
+  size_t ws_bytes = 0;
+  int* status = nullptr;        // device status word (+ padding)
+  float* H_raw = nullptr;       // [n][n] fp32 accumulator of X^T X (lower triangle valid until finalize)
+  float* H = nullptr;           // [n][n] fp32 damped, unscaled
+  float* s = nullptr;           // [n]
+  float* hdiag = nullptr;       // [n] diag of damped H
+  double* A64 = nullptr;        // [n][n] fp64 working copy of H~, reflectors afterwards
+  double* P64 = nullptr;        // [n][n] fp64 Q^T
+  double* td = nullptr;         // [n] tridiagonal diagonal
+  double* te = nullptr;         // [n] tridiagonal off-diagonal
+  double* beta = nullptr;       // [n] reflector scalars
+  double* pvec = nullptr;       // [n] matrix-vector scratch of the reduction
+  double* stage_l = nullptr;    // [T_max+1][n] LDL^T multipliers per penalty
+  double* stage_invd = nullptr; // [T_max+1][n] LDL^T inverse pivots per penalty
+  bf16 *Q_hi = nullptr, *Q_lo = nullptr;    // [n][n] Q   (row i, col m)
+  bf16 *QT_hi = nullptr, *QT_lo = nullptr;  // [n][n] Q^T (row m, col k)
+  bf16 *H_hi = nullptr, *H_lo = nullptr;    // [n][n] split planes of the damped unscaled H
+  float* Whs = nullptr;         // [p][n] scaled weights
+  float* V = nullptr;           // [p][n]
+  bf16 *R_hi = nullptr, *R_lo = nullptr;    // [p][n]
+  float* Y = nullptr;           // [p][n] (also the local-search gradient g)
+  bf16 *Y_hi = nullptr, *Y_lo = nullptr;    // [p][n]
+  float* partials = nullptr;    // [T_max][slots][2]
+  int partial_slots = 0;
+  double* scal = nullptr;       // small fp64 scalars (objective, counters)
+  bf16 *XT_hi = nullptr, *XT_lo = nullptr;  // [n][XT_ROWS] transposed chunk of X
+  void* tmaps = nullptr;        // reserved
+};
+
+constexpr int XT_ROWS = 16384;   // calibration rows handled per Hessian launch
+
+// ---- elem.cu ----
+void launch_zero(Ctx* c, void* ptr, size_t bytes);
+void launch_transpose_split(Ctx* c, const void* X, int is_bf16, long long rows, long long ldx, int n,
+                            bf16* XT_hi, bf16* XT_lo, long long ldt);
+void launch_finalize(Ctx* c, double damp_frac, int precondition);
+void launch_grid_fit(Ctx* c, const float* W0, int p, int bits, int gs, int symmetric, float* delta,
+                     float* zero);
+void launch_scale_weights(Ctx* c, const float* W0, int p);
+void launch_split_f64(Ctx* c, const double* src, int n, bf16* hi, bf16* lo, bf16* thi, bf16* tlo);
+void launch_split_f32(Ctx* c, const float* src, long long count, bf16* hi, bf16* lo);
+void launch_init_rhs(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
+                     const float* zero, const float* V_in, float inv_rho);
+void launch_reduce_partials(Ctx* c, int T, float* resid);
+void launch_dequant(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
+                    const float* zero, float* Wq);
+void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes,
+                         const float* delta, const float* zero, bf16* Ehi, bf16* Elo);
+void launch_objective_dot(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes,
+                          const float* delta, const float* zero, const float* g, double* out);
+
+// ---- gemm_simt.cu / gemm_tc.cu:  C[M][N] (epilogue)= A[M][K] * B[N][K]^T ----
+cudaError_t gemm_simt(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiParams& epi);
+cudaError_t gemm_tc(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiParams& epi);
+int gemm_tc_partial_slots(int num_sms);
+
+// ---- tridiag.cu ----
+cudaError_t tridiag_reduce(Ctx* c);                 // A64 -> td, te, reflectors, beta
+cudaError_t tridiag_form_qt(Ctx* c);                // reflectors -> P64 = Q^T
+void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count);
+void launch_tridiag_solve(Ctx* c, int p, int stage);
+
+// ---- local_search.cu ----
+cudaError_t launch_local_search(Ctx* c, const float* W0, int p, int bits, int gs, long long max_moves,
+                                float tau, unsigned char* codes, const float* delta,
+                                const float* zero, float* Wq, float* g, long long* d_moves,
+                                int* d_capped);
+
+}  // namespace admmq

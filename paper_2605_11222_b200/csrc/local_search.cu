@@ -1,0 +1,119 @@
+// Greedy single-entry local search (Sec. 3.5; Eq. 11 with the second perturbation zero).
+// One CTA per output channel: its gradient g = H (w_q - w_hat), its codes and diag(H) stay in shared
+// memory; every step scans the 2 n candidate moves, a block-wide argmin picks the best one, and the
+// gradient takes the rank-1 correction g += d H[:, i] (row i of the symmetric H, contiguous).
+#include "internal.h"
+
+namespace admmq {
+
+struct Cand {
+  float cost;
+  int idx;   // 2 * i + (0 for +Delta, 1 for -Delta); ties resolve to the smallest idx
+};
+
+__device__ __forceinline__ Cand better(Cand a, Cand b) {
+  if (b.cost < a.cost || (b.cost == a.cost && b.idx < a.idx)) return b;
+  return a;
+}
+
+__global__ void __launch_bounds__(256)
+local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag, int n, int p, int gs,
+                    int kmax, long long max_moves, float tau, const float* __restrict__ W0,
+                    unsigned char* __restrict__ codes, const float* __restrict__ delta,
+                    const float* __restrict__ zero, float* __restrict__ Wq, float* __restrict__ g_glob,
+                    long long* __restrict__ moves_out, int* __restrict__ capped_out) {
+  extern __shared__ float smf[];
+  float* g = smf;                  // [n]
+  float* hd = smf + n;             // [n]
+  unsigned char* kc = (unsigned char*)(smf + 2 * n);   // [n]
+  __shared__ Cand wbest[8];
+  __shared__ Cand chosen;
+  const int j = blockIdx.x;
+  if (j >= p) return;
+  const int ng = n / gs;
+  const float* dl = delta + (long long)j * ng;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    g[i] = g_glob[(long long)j * n + i];
+    hd[i] = hdiag[i];
+    kc[i] = codes[(long long)j * n + i];
+  }
+  __syncthreads();
+  long long moves = 0;
+  int capped = 0;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  while (true) {
+    Cand best;
+    best.cost = INFINITY;
+    best.idx = 0x7fffffff;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      const float d = dl[i / gs];
+      const float quad = d * d * hd[i];
+      const float lin = 2.0f * d * g[i];
+      const int k = kc[i];
+      if (k < kmax) best = better(best, Cand{lin + quad, 2 * i});
+      if (k > 0) best = better(best, Cand{-lin + quad, 2 * i + 1});
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      Cand other;
+      other.cost = __shfl_xor_sync(0xffffffffu, best.cost, o);
+      other.idx = __shfl_xor_sync(0xffffffffu, best.idx, o);
+      best = better(best, other);
+    }
+    if (lane == 0) wbest[wid] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      Cand b = wbest[0];
+      for (int w = 1; w < nw; ++w) b = better(b, wbest[w]);
+      if (b.idx != 0x7fffffff) {
+        const int i = b.idx >> 1;
+        const float d = dl[i / gs];
+        if (!(b.cost < -tau * hd[i] * d * d)) b.idx = -1;   // no improving move: stop
+      } else {
+        b.idx = -1;
+      }
+      chosen = b;
+    }
+    __syncthreads();
+    const Cand c = chosen;
+    if (c.idx < 0) break;
+    const int i = c.idx >> 1;
+    const float sgn = (c.idx & 1) ? -1.0f : 1.0f;
+    const float d = sgn * dl[i / gs];
+    const float* hrow = H + (long long)i * n;
+    for (int t = threadIdx.x; t < n; t += blockDim.x) g[t] = fmaf(d, hrow[t], g[t]);
+    if (threadIdx.x == 0) kc[i] = (unsigned char)((int)kc[i] + ((c.idx & 1) ? -1 : 1));
+    ++moves;
+    __syncthreads();
+    if (moves >= max_moves) {
+      capped = 1;
+      break;
+    }
+  }
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const long long idx = (long long)j * n + i;
+    codes[idx] = kc[i];
+    g_glob[idx] = g[i];
+    if (Wq) Wq[idx] = zero[(long long)j * ng + i / gs] + dl[i / gs] * (float)kc[i];
+  }
+  if (threadIdx.x == 0) {
+    atomicAdd((unsigned long long*)moves_out, (unsigned long long)moves);
+    if (capped) atomicAdd(capped_out, 1);
+  }
+}
+
+cudaError_t launch_local_search(Ctx* c, const float* W0, int p, int bits, int gs, long long max_moves,
+                                float tau, unsigned char* codes, const float* delta, const float* zero,
+                                float* Wq, float* g, long long* d_moves, int* d_capped) {
+  const int n = c->n;
+  const size_t smem = (size_t)n * 9 + 16;
+  cudaError_t e = cudaFuncSetAttribute(local_search_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) return e;
+  local_search_kernel<<<p, 256, smem, c->stream>>>(c->H, c->hdiag, n, p, gs, (1 << bits) - 1, max_moves,
+                                                   tau, W0, codes, delta, zero, Wq, g, d_moves, d_capped);
+  c->launches++;
+  return cudaGetLastError();
+}
+
+}  // namespace admmq
