@@ -90,7 +90,7 @@ admmq_status admmq_last_device_status(admmq_ctx* ctx);
 /* ---- Step 1: Hessian accumulation, H_raw += X^T X, N += n_tokens  (Sec. 3.1: H = X^T X). ----------
  * d_X: [n_tokens][ldx] row-major, dtype fp32 or bf16; the first d_in columns of each row are used;
  * ldx >= d_in, and ldx * sizeof(element) a multiple of 16.  Only read.  May be called any number of
- * times after admmq_hessian_reset; accumulation is in fp32. */
+ * times after admmq_hessian_reset; accumulation is in fp32.  n_tokens == 0 is a no-op. */
 admmq_status admmq_hessian_reset(admmq_ctx* ctx);
 admmq_status admmq_hessian_accumulate(admmq_ctx* ctx, const void* d_X, admmq_dtype dtype,
                                       long long n_tokens, long long ldx);
@@ -182,6 +182,24 @@ admmq_status admmq_get_hessian(admmq_ctx* ctx, float* d_H_out, float* d_s_out);
 
 /* Number of kernels this context has launched so far (host counter). */
 long long admmq_launch_count(const admmq_ctx* ctx);
+
+/* Per-kernel device timing for measurement.  With timing on, the library brackets each launch of the
+ * kinds below with CUDA events on its stream.  admmq_get_timing synchronises, adds up the elapsed time
+ * and the number of launches of one kind since the last admmq_reset_timing, and keeps the records. */
+typedef enum {
+  ADMMQ_T_HESSIAN_PRODUCT = 0,  /* X^T X product kernel                                   (step 1) */
+  ADMMQ_T_TRANSPOSE = 1,        /* X chunk -> K-major planes                              (step 1) */
+  ADMMQ_T_FACTOR = 2,           /* finalisation + tridiagonal reduction + Q + stage factors (step 2) */
+  ADMMQ_T_WUPDATE_PRODUCT1 = 3, /* Y = R Q                                                (step 3) */
+  ADMMQ_T_TRIDIAG_SOLVE = 4,    /* (T/rho + I)^{-1} row solve                             (step 3) */
+  ADMMQ_T_WUPDATE_PRODUCT2 = 5, /* Z = Y' Q^T with the fused projection/dual/residual epilogue */
+  ADMMQ_T_GRADIENT_PRODUCT = 6, /* g = E H                                                (step 4) */
+  ADMMQ_T_LOCAL_SEARCH = 7,     /* move loop kernel                                       (step 4) */
+  ADMMQ_T_KINDS = 8
+} admmq_timing_kind;
+admmq_status admmq_set_timing(admmq_ctx* ctx, int on);
+admmq_status admmq_reset_timing(admmq_ctx* ctx);
+admmq_status admmq_get_timing(admmq_ctx* ctx, int kind, double* h_total_ms, long long* h_count);
 
 #ifdef __cplusplus
 }

@@ -26,8 +26,12 @@ EXPORTS = [
     "admmq_set_gemm_kind", "admmq_last_device_status", "admmq_hessian_reset",
     "admmq_hessian_accumulate", "admmq_hessian_set", "admmq_factor", "admmq_quantize_layer",
     "admmq_w_update", "admmq_local_search", "admmq_objective", "admmq_get_hessian",
-    "admmq_launch_count",
+    "admmq_launch_count", "admmq_set_timing", "admmq_reset_timing", "admmq_get_timing",
 ]
+T_HESSIAN_PRODUCT, T_TRANSPOSE, T_FACTOR, T_WUPDATE_PRODUCT1, T_TRIDIAG_SOLVE, T_WUPDATE_PRODUCT2, \
+    T_GRADIENT_PRODUCT, T_LOCAL_SEARCH = range(8)
+TIMING_NAMES = ["hessian_product", "transpose", "factor", "wupdate_product1", "tridiag_solve",
+                "wupdate_product2", "gradient_product", "local_search"]
 
 
 class FactorCfg(C.Structure):
@@ -90,6 +94,9 @@ def load_library(path: Optional[str] = None):
     lib.admmq_local_search.argtypes = [vp, vp, ci, C.POINTER(LsCfg), vp, vp, vp, vp, C.POINTER(Report)]
     lib.admmq_objective.argtypes = [vp, vp, ci, ci, vp, vp, vp, C.POINTER(cd)]
     lib.admmq_get_hessian.argtypes = [vp, vp, vp]
+    lib.admmq_set_timing.argtypes = [vp, ci]
+    lib.admmq_reset_timing.argtypes = [vp]
+    lib.admmq_get_timing.argtypes = [vp, ci, C.POINTER(cd), C.POINTER(cll)]
     lib.admmq_launch_count.restype = cll
     lib.admmq_launch_count.argtypes = [vp]
     for name in EXPORTS:
@@ -233,6 +240,21 @@ class Solver:
         s = torch.empty(self.d_in, dtype=torch.float32, device=self.device)
         _check(self.lib.admmq_get_hessian(self.h, _ptr(H), _ptr(s)), "admmq_get_hessian")
         return H, s
+
+    def set_timing(self, on: bool):
+        _check(self.lib.admmq_set_timing(self.h, int(on)), "admmq_set_timing")
+
+    def reset_timing(self):
+        _check(self.lib.admmq_reset_timing(self.h), "admmq_reset_timing")
+
+    def get_timing(self) -> dict:
+        """{kind name: (total ms, launches)} since the last reset (synchronises)."""
+        out = {}
+        for k, name in enumerate(TIMING_NAMES):
+            ms, cnt = C.c_double(0.0), C.c_longlong(0)
+            _check(self.lib.admmq_get_timing(self.h, k, C.byref(ms), C.byref(cnt)), "admmq_get_timing")
+            out[name] = (ms.value, cnt.value)
+        return out
 
     def launch_count(self) -> int:
         return int(self.lib.admmq_launch_count(self.h))

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <new>
 #include <string.h>
+#include <vector>
 
 #include "../../include/admmq.h"
 #include "internal.h"
@@ -16,6 +17,11 @@ struct admmq_ctx {
   int* d_capped = nullptr;
   int slots_cap = 0;
   double rho_adhoc = 0.0;
+  // ---- optional per-kernel timing ----
+  int timing_on = 0;
+  struct Rec { cudaEvent_t a, b; int kind; };
+  std::vector<Rec> recs;          // records in use
+  std::vector<Rec> pool;          // created events available for reuse
 };
 
 namespace {
@@ -108,6 +114,30 @@ admmq_status read_status(admmq_ctx* a) {
   return (admmq_status)st;
 }
 
+// Brackets a region of launches with events when timing is on.
+struct Timed {
+  admmq_ctx* a;
+  bool live = false;
+  admmq_ctx::Rec r{};
+  Timed(admmq_ctx* ctx, int kind) : a(ctx) {
+    if (!a->timing_on) return;
+    if (!a->pool.empty()) {
+      r = a->pool.back();
+      a->pool.pop_back();
+    } else if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) {
+      return;
+    }
+    r.kind = kind;
+    live = true;
+    cudaEventRecord(r.a, a->c.stream);
+  }
+  ~Timed() {
+    if (!live) return;
+    cudaEventRecord(r.b, a->c.stream);
+    a->recs.push_back(r);
+  }
+};
+
 int group_of(int d_in, int gs) { return (gs == 0 || gs == d_in) ? d_in : gs; }
 
 // g = E H with E = W_q - W_hat, into c->Y; E planes go through the R buffers.
@@ -119,6 +149,7 @@ cudaError_t gradient(admmq_ctx* a, const float* W0, int p, int gs, const unsigne
   e.kind = EPI_STORE;
   e.C = c->Y;
   e.ldc = c->n;
+  Timed t(a, ADMMQ_T_GRADIENT_PRODUCT);
   return product(c, Planes{c->R_hi, c->R_lo, c->n}, Planes{c->H_hi, c->H_lo, c->n}, p, c->n, c->n, e);
 }
 
@@ -181,6 +212,11 @@ admmq_status admmq_create(admmq_ctx** ctx, int d_in, int d_out_max, int T_max, v
 
 admmq_status admmq_destroy(admmq_ctx* ctx) {
   if (!ctx) return ADMMQ_ERR_INVALID_ARG;
+  for (auto* v : {&ctx->recs, &ctx->pool})
+    for (auto& r : *v) {
+      cudaEventDestroy(r.a);
+      cudaEventDestroy(r.b);
+    }
   delete ctx;
   return ADMMQ_OK;
 }
@@ -210,10 +246,12 @@ admmq_status admmq_hessian_reset(admmq_ctx* ctx) {
 
 admmq_status admmq_hessian_accumulate(admmq_ctx* ctx, const void* d_X, admmq_dtype dtype,
                                       long long n_tokens, long long ldx) {
-  if (!ctx || !d_X || !aligned16(d_X)) return ADMMQ_ERR_INVALID_ARG;
+  if (!ctx) return ADMMQ_ERR_INVALID_ARG;
   if (dtype != ADMMQ_F32 && dtype != ADMMQ_BF16) return ADMMQ_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
   if (c->state != 1) return ADMMQ_ERR_STATE;
+  if (n_tokens == 0) return ADMMQ_OK;                    // an empty chunk adds nothing
+  if (!d_X || !aligned16(d_X)) return ADMMQ_ERR_INVALID_ARG;
   const size_t esz = dtype == ADMMQ_BF16 ? 2 : 4;
   if (n_tokens < 0 || ldx < c->n || ((size_t)ldx * esz) % 16 != 0) return ADMMQ_ERR_SHAPE;
   const int n = c->n;
@@ -221,13 +259,17 @@ admmq_status admmq_hessian_accumulate(admmq_ctx* ctx, const void* d_X, admmq_dty
     const long long rows = (n_tokens - r0 < XT_ROWS) ? (n_tokens - r0) : XT_ROWS;
     const char* xp = (const char*)d_X + (size_t)r0 * ldx * esz;
     bf16* lo = dtype == ADMMQ_BF16 ? nullptr : c->XT_lo;
-    launch_transpose_split(c, xp, dtype == ADMMQ_BF16, rows, ldx, n, c->XT_hi, lo, XT_ROWS);
+    {
+      Timed t(ctx, ADMMQ_T_TRANSPOSE);
+      launch_transpose_split(c, xp, dtype == ADMMQ_BF16, rows, ldx, n, c->XT_hi, lo, XT_ROWS);
+    }
     EpiParams e{};
     e.kind = EPI_ACCUM;
     e.C = c->H_raw;
     e.ldc = n;
     e.lower_only = 1;
     Planes P{c->XT_hi, lo, XT_ROWS};
+    Timed t(ctx, ADMMQ_T_HESSIAN_PRODUCT);
     if (product(c, P, P, n, n, (int)rows, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
   }
   c->n_tokens += n_tokens;
@@ -262,6 +304,7 @@ admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg) {
   c->T = cfg->T;
   c->precondition = cfg->precondition ? 1 : 0;
   const int n = c->n;
+  Timed tfac(ctx, ADMMQ_T_FACTOR);
   launch_finalize(c, cfg->damp_frac, c->precondition);
   launch_split_f32(c, c->H, (long long)n * n, c->H_hi, c->H_lo);
   if (tridiag_reduce(c) != cudaSuccess) return ADMMQ_ERR_CUDA;
@@ -293,15 +336,24 @@ static admmq_status check_layer_args(admmq_ctx* ctx, const float* d_W0, int d_ou
 
 // One W-update in the error form of Eq. 7:  W - W_hat' = Q (T/rho + I)^{-1} Q^T R,
 // R = D - V/rho - W_hat'.  Product 1 -> solve -> product 2 (whose epilogue is `epi`).
-static cudaError_t w_update_products(Ctx* c, int p, int stage, const EpiParams& epi) {
+static cudaError_t w_update_products(admmq_ctx* a, int p, int stage, const EpiParams& epi) {
+  Ctx* c = &a->c;
   const int n = c->n;
   EpiParams e1{};
   e1.kind = EPI_STORE;
   e1.C = c->Y;
   e1.ldc = n;
-  cudaError_t err = product(c, Planes{c->R_hi, c->R_lo, n}, Planes{c->QT_hi, c->QT_lo, n}, p, n, n, e1);
+  cudaError_t err;
+  {
+    Timed t(a, ADMMQ_T_WUPDATE_PRODUCT1);
+    err = product(c, Planes{c->R_hi, c->R_lo, n}, Planes{c->QT_hi, c->QT_lo, n}, p, n, n, e1);
+  }
   if (err != cudaSuccess) return err;
-  launch_tridiag_solve(c, p, stage);
+  {
+    Timed t(a, ADMMQ_T_TRIDIAG_SOLVE);
+    launch_tridiag_solve(c, p, stage);
+  }
+  Timed t(a, ADMMQ_T_WUPDATE_PRODUCT2);
   return product(c, Planes{c->Y_hi, c->Y_lo, n}, Planes{c->Q_hi, c->Q_lo, n}, p, n, n, epi);
 }
 
@@ -343,7 +395,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     e.inv_rho = (float)(1.0 / rho);
     e.inv_rho_next = (float)(1.0 / rho_next);
     e.partials = c->partials + (size_t)t * c->partial_slots * 2;
-    if (w_update_products(c, p, t, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
+    if (w_update_products(ctx, p, t, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
   }
   if (d_resid) launch_reduce_partials(c, T, d_resid);
   if (d_Wq) launch_dequant(c, p, gs, d_codes, d_scale, d_zero, d_Wq);
@@ -387,7 +439,7 @@ admmq_status admmq_w_update(admmq_ctx* ctx, const float* d_W0, int d_out, int gr
   e.C = d_W_out;
   e.ldc = n;
   e.Whs = c->Whs;
-  if (w_update_products(c, p, stage, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  if (w_update_products(ctx, p, stage, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? ADMMQ_OK : ADMMQ_ERR_CUDA;
 }
 
@@ -411,9 +463,12 @@ admmq_status admmq_local_search(admmq_ctx* ctx, const float* d_W0, int d_out, co
   if (h_report) launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 1);
   launch_zero(c, ctx->d_moves, 64);
   launch_zero(c, ctx->d_capped, 64);
-  if (launch_local_search(c, d_W0, p, cfg->bits, gs, cap, (float)cfg->accept_tol, d_codes, d_scale, d_zero,
-                          d_Wq, c->Y, ctx->d_moves, ctx->d_capped) != cudaSuccess)
-    return ADMMQ_ERR_CUDA;
+  {
+    Timed t(ctx, ADMMQ_T_LOCAL_SEARCH);
+    if (launch_local_search(c, d_W0, p, cfg->bits, gs, cap, (float)cfg->accept_tol, d_codes, d_scale,
+                            d_zero, d_Wq, c->Y, ctx->d_moves, ctx->d_capped) != cudaSuccess)
+      return ADMMQ_ERR_CUDA;
+  }
   if (!h_report) return ADMMQ_OK;
   cudaEventRecord(ev1, c->stream);
   memset(h_report, 0, sizeof(*h_report));
@@ -451,6 +506,37 @@ admmq_status admmq_objective(admmq_ctx* ctx, const float* d_W0, int d_out, int g
   if (cudaMemcpy(h_err, c->scal + 1, sizeof(double), cudaMemcpyDeviceToHost) != cudaSuccess)
     return ADMMQ_ERR_CUDA;
   return st;
+}
+
+admmq_status admmq_set_timing(admmq_ctx* ctx, int on) {
+  if (!ctx) return ADMMQ_ERR_INVALID_ARG;
+  ctx->timing_on = on ? 1 : 0;
+  return ADMMQ_OK;
+}
+
+admmq_status admmq_reset_timing(admmq_ctx* ctx) {
+  if (!ctx) return ADMMQ_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(ctx->c.stream) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  for (auto& r : ctx->recs) ctx->pool.push_back(r);
+  ctx->recs.clear();
+  return ADMMQ_OK;
+}
+
+admmq_status admmq_get_timing(admmq_ctx* ctx, int kind, double* h_total_ms, long long* h_count) {
+  if (!ctx || !h_total_ms || !h_count || kind < 0 || kind >= ADMMQ_T_KINDS) return ADMMQ_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(ctx->c.stream) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  double total = 0.0;
+  long long count = 0;
+  for (auto& r : ctx->recs) {
+    if (r.kind != kind) continue;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, r.a, r.b) != cudaSuccess) return ADMMQ_ERR_CUDA;
+    total += ms;
+    ++count;
+  }
+  *h_total_ms = total;
+  *h_count = count;
+  return ADMMQ_OK;
 }
 
 admmq_status admmq_get_hessian(admmq_ctx* ctx, float* d_H_out, float* d_s_out) {

@@ -1,0 +1,359 @@
+"""GPU parity: every step of the CUDA path, called through the C ABI, against the fp64 oracle
+on the same seeded inputs.  Tolerances (derivation in the design notes):
+  * integer codes: exact on the tiny / brute-force cases, >= 99.9 % equal on larger layers;
+  * layer reconstruction error within 1e-3 relative of the oracle's;
+  * one W-update from identical (D, V): 1e-4 relative Frobenius;
+  * Hessian entries: 1e-4 relative to the Frobenius norm (fp32 accumulation of bf16 products).
+"""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import admmq_oracle as O
+from paper_2605_11222_b200 import binding as B
+from paper_2605_11222_b200 import workloads as wl
+from tests.helpers import np64, oracle_hessian, to_dev
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+W_UPDATE_TOL = 1e-4
+CODE_AGREEMENT = 0.999
+ERR_TOL = 1e-3
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2605_11222_b200 import build
+    build.build()
+    B.load_library()
+
+
+def _solve_gpu(spec, gemm_kind=B.GEMM_TENSOR, local_search=True, precondition=True):
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(spec.d_in, spec.d_out, T_max=max(spec.T, 2))
+    sol.set_gemm_kind(gemm_kind)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=spec.rho(), precondition=precondition)
+    resid = torch.zeros(spec.T, 2, device=DEV)
+    Wq = torch.empty_like(W)
+    codes, scale, zero, rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, Wq=Wq,
+                                                 resid=resid)
+    out = dict(sol=sol, W=W, codes_admm=codes.clone(), scale=scale, zero=zero, rep=rep,
+               resid=resid.cpu().numpy(), Wq_admm=Wq.clone())
+    if local_search:
+        rep2, st = sol.local_search(W, spec.bits, spec.group_size, codes, scale, zero, Wq=Wq)
+        out.update(codes_final=codes, rep_ls=rep2, st_ls=st, Wq_final=Wq)
+    assert sol.last_device_status() == B.OK
+    return out
+
+
+def _solve_oracle(spec, H=None, cols=None):
+    Wn = np64(wl.gen_weight(spec, DEV))
+    if cols is not None:
+        Wn = Wn[cols]
+    H = oracle_hessian(spec, DEV) if H is None else H
+    res = O.quantize_layer(H, Wn, spec.bits, spec.group_size, spec.symmetric, np.array(spec.rho()))
+    return H, Wn, res
+
+
+# ------------------------------------------------------------------ step 1-2: Hessian, damping, scaling
+@pytest.mark.parametrize("x_dtype,n,N", [("bf16", 520, 6000), ("f32", 264, 9000), ("bf16", 64, 100)])
+@pytest.mark.parametrize("kind", [B.GEMM_TENSOR, B.GEMM_SIMT])
+def test_hessian_parity(x_dtype, n, N, kind):
+    spec = wl.small_case(n, 16, N, x_dtype=x_dtype, group_size=0, T=2)
+    sol = B.Solver(n, 16, T_max=2)
+    sol.set_gemm_kind(kind)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=[0.1, 0.2])
+    Hg, sg = sol.get_hessian()
+    Ho = oracle_hessian(spec, DEV)
+    Hg = np64(Hg)
+    assert np.array_equal(Hg, Hg.T)
+    assert np.linalg.norm(Hg - Ho) <= 1e-4 * np.linalg.norm(Ho)
+    assert np.abs(np64(sg) - np.sqrt(np.diag(Ho))).max() <= 1e-4 * np.sqrt(np.diag(Ho)).max()
+    # sampled entries against the entry-wise definition H_ab = sum_t X_ta X_tb / N (+ damping on a = b)
+    X = torch.cat([wl.gen_x_chunk(spec, c, DEV) for c in range(spec.n_chunks)]).double()
+    lam = 0.01 * float((X * X).sum(0).mean() / N)
+    for a, b in [(0, 0), (n - 1, 3), (n // 2, n // 2 + 1), (n - 1, n - 1)]:
+        ref = float((X[:, a] * X[:, b]).sum() / N) + (lam if a == b else 0.0)
+        assert abs(Hg[a, b] - ref) <= 1e-4 * max(abs(ref), np.sqrt(Ho[a, a] * Ho[b, b]) * 1e-2)
+    assert sol.last_device_status() == B.OK
+
+
+def test_hessian_chunking_is_immaterial():
+    spec = wl.small_case(256, 16, 5000, group_size=0, T=2)
+    X = torch.cat([wl.gen_x_chunk(spec, c, DEV) for c in range(spec.n_chunks)])
+    outs = []
+    for pieces in ([5000], [1234, 3766], [100] * 50):
+        sol = B.Solver(256, 16, T_max=2)
+        sol.hessian_reset()
+        a = 0
+        for m in pieces:
+            sol.hessian_accumulate(X[a:a + m])
+            a += m
+        sol.factor(rho=[0.1, 0.2])
+        outs.append(np64(sol.get_hessian()[0]))
+    for o in outs[1:]:
+        assert np.linalg.norm(o - outs[0]) <= 2e-5 * np.linalg.norm(outs[0])
+
+
+# ------------------------------------------------------------------ step 5-6: one W-update from identical (D, V)
+@pytest.mark.parametrize("n,p,gs", [(512, 384, 128), (328, 130, 0)])
+@pytest.mark.parametrize("kind", [B.GEMM_TENSOR, B.GEMM_SIMT])
+def test_w_update_parity(n, p, gs, kind):
+    spec = wl.small_case(n, p, 4096, group_size=gs, T=2)
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(n, p, T_max=2)
+    sol.set_gemm_kind(kind)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=[0.1, 0.2])
+    Ho = oracle_hessian(spec, DEV)
+    Wn = np64(W)
+    delta, z0 = O.grid_fit(Wn, spec.bits, gs, False)
+    s, Ht, Ws = O.precondition(Ho, Wn)
+    lam, U = O.eig_factor(Ht)
+    rng = np.random.default_rng(5)
+    codes = rng.integers(0, 1 << spec.bits, size=Wn.shape).astype(np.uint8)
+    V = (0.01 * np.abs(Ws).mean() * rng.standard_normal(Wn.shape)).astype(np.float32)
+    D = s[None, :] * O.dequantize(codes, delta, z0)
+    for rho in (0.05, 0.1, 1.0, 37.0, 1e4):
+        Wo = O.w_update(lam, U, Ws @ Ht, D, V.astype(np.float64), rho)
+        Wg = sol.w_update(W, gs, to_dev(codes, torch.uint8, DEV), to_dev(delta, torch.float32, DEV),
+                          to_dev(z0, torch.float32, DEV), to_dev(V, torch.float32, DEV), rho)
+        rel = np.linalg.norm(np64(Wg) - Wo) / np.linalg.norm(Wo)
+        assert rel <= W_UPDATE_TOL, (rho, rel)
+    assert sol.last_device_status() == B.OK
+
+
+# ------------------------------------------------------------------ whole layer, mid size
+@pytest.mark.parametrize("kw", [
+    dict(d_in=512, d_out=384, n_tokens=6144),                                   # g128, asym, 3 bit
+    dict(d_in=328, d_out=130, n_tokens=3000, group_size=0, bits=4),             # ragged tiles, per-channel
+    dict(d_in=256, d_out=200, n_tokens=3000, group_size=0, bits=2, symmetric=True, rotate=True),
+    dict(d_in=384, d_out=64, n_tokens=2048, group_size=64, x_kind="silu_like"),
+])
+def test_layer_parity_mid_size(kw):
+    spec = wl.small_case(**kw)
+    g = _solve_gpu(spec)
+    H, Wn, res = _solve_oracle(spec)
+    a = res.admm
+    assert np.allclose(g["scale"].cpu().numpy(), a.delta, rtol=2e-7, atol=0)
+    assert np.allclose(g["zero"].cpu().numpy(), a.z0, rtol=1e-7, atol=0)
+    cg = g["codes_admm"].cpu().numpy()
+    assert cg.max() <= (1 << spec.bits) - 1
+    assert (cg == a.codes).mean() >= CODE_AGREEMENT
+    # reconstruction error of the GPU's codes, evaluated by the oracle, against the oracle's own
+    e_g = O.objective(H, Wn, O.dequantize(cg, a.delta, a.z0))
+    assert abs(e_g - res.err_admm) <= ERR_TOL * res.err_admm
+    assert abs(g["rep"].err_before - e_g) <= ERR_TOL * e_g                   # the GPU's own error report
+    # dequantised output is the grid point of its codes
+    assert np.allclose(g["Wq_admm"].cpu().numpy(), O.dequantize(cg, a.delta, a.z0), rtol=1e-6, atol=3e-8)
+    # residual traces (Theorem 1 quantities); the fp32 floor shows only once they are ~1e-6 of the start
+    r = g["resid"]
+    assert np.abs(r[:, 0] - a.r).max() <= 1e-3 * a.r.max()
+    assert np.abs(r[:, 1] - a.sres).max() <= 2e-2 * a.sres.max()
+    # after local search
+    cf = g["codes_final"].cpu().numpy()
+    assert (cf == res.ls.codes).mean() >= CODE_AGREEMENT
+    e_f = O.objective(H, Wn, O.dequantize(cf, a.delta, a.z0))
+    assert abs(e_f - res.err_final) <= ERR_TOL * res.err_final
+    assert e_f <= e_g * (1 + 1e-9)
+    assert abs(g["rep_ls"].err_after - e_f) <= ERR_TOL * e_f
+    # the GPU's final point is a 1-move local optimum in the oracle's fp64 arithmetic, up to fp32 slack
+    again = O.local_search(H, Wn, cf, a.delta, a.z0, spec.bits, tau=1e-6)
+    assert again.moves.sum() <= 1e-3 * cf.size
+    assert O.objective(H, Wn, again.Wq) >= e_f * (1 - 1e-5)
+
+
+def test_local_search_from_identical_codes():
+    spec = wl.small_case(512, 96, 4096, bits=3)
+    g = _solve_gpu(spec, local_search=False)
+    H, Wn, _ = _solve_oracle(spec)
+    codes = g["codes_admm"].clone()
+    cg = codes.cpu().numpy()
+    delta, z0 = O.grid_fit(Wn, spec.bits, spec.group_size, spec.symmetric)
+    ls = O.local_search(H, Wn, cg, delta, z0, spec.bits)
+    rep, st = g["sol"].local_search(g["W"], spec.bits, spec.group_size, codes, g["scale"], g["zero"])
+    assert st == B.OK
+    assert (codes.cpu().numpy() == ls.codes).mean() >= 0.9999
+    assert abs(rep.moves - int(ls.moves.sum())) <= max(3, 1e-3 * ls.moves.sum())
+    e = O.objective(H, Wn, ls.Wq)
+    assert abs(rep.err_after - e) <= ERR_TOL * e
+    # move cap: a warning status, never more than the cap per column
+    codes2 = g["codes_admm"].clone()
+    rep2, st2 = g["sol"].local_search(g["W"], spec.bits, spec.group_size, codes2, g["scale"], g["zero"],
+                                      max_moves_per_col=2)
+    assert st2 == B.WARN_MOVE_CAP and rep2.capped_columns > 0 and rep2.moves <= 2 * spec.d_out
+    ls2 = O.local_search(H, Wn, cg, delta, z0, spec.bits, max_moves=2)
+    assert (codes2.cpu().numpy() == ls2.codes).mean() >= 0.9999
+
+
+def test_tensor_and_simt_products_agree():
+    spec = wl.small_case(512, 256, 4096)
+    a = _solve_gpu(spec, B.GEMM_TENSOR)
+    b = _solve_gpu(spec, B.GEMM_SIMT)
+    assert (a["codes_admm"] == b["codes_admm"]).float().mean().item() >= CODE_AGREEMENT
+    assert abs(a["rep"].err_before - b["rep"].err_before) <= ERR_TOL * b["rep"].err_before
+
+
+# ------------------------------------------------------------------ config 1 in full
+def test_config1_full():
+    spec = wl.config1()
+    g = _solve_gpu(spec)
+    H, Wn, res = _solve_oracle(spec)
+    cg = g["codes_admm"].cpu().numpy()
+    assert (cg == res.admm.codes).mean() >= CODE_AGREEMENT
+    cf = g["codes_final"].cpu().numpy()
+    assert (cf == res.ls.codes).mean() >= CODE_AGREEMENT
+    e_f = O.objective(H, Wn, O.dequantize(cf, res.admm.delta, res.admm.z0))
+    assert abs(e_f - res.err_final) <= ERR_TOL * res.err_final
+    rtn = O.dequantize(O.project(Wn, np.ones(spec.d_in), res.admm.delta, res.admm.z0, spec.bits)[0],
+                       res.admm.delta, res.admm.z0)
+    assert e_f < O.objective(H, Wn, rtn)
+
+
+# ------------------------------------------------------------------ tiny cases: exact codes, brute force
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_tiny_exact_and_brute_force(seed):
+    n, p, bits = 8, 5, 2
+    rng = np.random.default_rng(200 + seed)
+    X = rng.standard_normal((64, n))
+    X[:, seed % n] *= 5.0
+    Hn = (X.T @ X / 64).astype(np.float32)                       # undamped Hessian, handed over directly
+    Wn = (0.02 * rng.standard_normal((p, n))).astype(np.float32)
+    rho = O.rho_schedule(40, 0.05, 1.3)
+    sol = B.Solver(n, p, T_max=40)
+    sol.hessian_set(to_dev(Hn, torch.float32, DEV))
+    sol.factor(rho=list(rho))
+    W = to_dev(Wn, torch.float32, DEV)
+    codes, scale, zero, rep = sol.quantize_layer(W, bits, 0, False)
+    H = O.hessian_finalize(Hn.astype(np.float64), 1)
+    res = O.quantize_layer(H, Wn.astype(np.float64), bits, 0, False, rho)
+    assert np.array_equal(codes.cpu().numpy(), res.admm.codes)
+    sol.local_search(W, bits, 0, codes, scale, zero)
+    mine = codes.cpu().numpy()
+    assert np.array_equal(mine, res.ls.codes)
+    # brute force over all 4^8 assignments per column: 1-move local optimum
+    all_codes = np.array(list(itertools.product(range(4), repeat=n)))
+    delta, z0 = res.admm.delta, res.admm.z0
+    for j in range(p):
+        E = z0[j, 0] + delta[j, 0] * all_codes - Wn[j].astype(np.float64)[None, :]
+        loss = np.einsum("ci,ik,ck->c", E, H, E)
+        w = 4 ** np.arange(n - 1, -1, -1)
+        my = loss[int(mine[j].astype(int) @ w)]
+        assert my >= loss.min() - 1e-15
+        for i in range(n):
+            for sg in (1, -1):
+                nb = mine[j].astype(int).copy()
+                nb[i] += sg
+                if 0 <= nb[i] <= 3:
+                    assert loss[int(nb @ w)] >= my - 1e-6 * H[i, i] * delta[j, 0] ** 2 - 1e-12
+    assert sol.last_device_status() == B.OK
+
+
+def test_diagonal_hessian_gives_rtn():
+    n, p, bits = 64, 24, 3
+    rng = np.random.default_rng(12)
+    Wn = (0.02 * rng.standard_normal((p, n))).astype(np.float32)
+    Hn = np.diag(np.exp(rng.standard_normal(n))).astype(np.float32)
+    W = to_dev(Wn, torch.float32, DEV)
+    delta, z0 = O.grid_fit(Wn.astype(np.float64), bits, 0, False)
+    rtn = O.project(Wn.astype(np.float64), np.ones(n), delta, z0, bits)[0]
+    for rho in ([1.0 * 1.2 ** t for t in range(30)], [0.05]):                 # rho >= 1 always; T = 1
+        sol = B.Solver(n, p, T_max=30)
+        sol.hessian_set(to_dev(Hn, torch.float32, DEV))
+        sol.factor(rho=rho, damp_frac=0.0)
+        codes, scale, zero, _ = sol.quantize_layer(W, bits, 0, False)
+        assert np.array_equal(codes.cpu().numpy(), rtn)
+    sol = B.Solver(n, p, T_max=60)                                           # any schedule + local search
+    sol.hessian_set(to_dev(Hn, torch.float32, DEV))
+    sol.factor(rho=[0.01 * 1.2 ** t for t in range(60)], damp_frac=0.0)
+    codes, scale, zero, _ = sol.quantize_layer(W, bits, 0, False)
+    sol.local_search(W, bits, 0, codes, scale, zero)
+    assert np.array_equal(codes.cpu().numpy(), rtn)
+
+
+# ------------------------------------------------------------------ edge cases and error paths (no GPU fault)
+def test_degenerate_inputs():
+    n, p = 64, 3
+    spec = wl.small_case(n, p, 512, group_size=16, T=5)
+    W = wl.gen_weight(spec, DEV)
+    W[1, 16:32] = 0.0125                                          # a constant group: Delta = 1, codes 0
+    W[2, :] = 0.0                                                 # a constant channel
+    sol = B.Solver(n, p, T_max=5)
+    sol.hessian_reset()
+    sol.hessian_accumulate(wl.gen_x_chunk(spec, 0, DEV))
+    sol.hessian_accumulate(wl.gen_x_chunk(spec, 0, DEV)[:0])      # an empty chunk is a no-op
+    sol.factor(rho=spec.rho())
+    codes, scale, zero, rep = sol.quantize_layer(W, 3, 16, False)
+    assert scale[1, 1].item() == 1.0 and zero[1, 1].item() == pytest.approx(0.0125)
+    assert codes[1, 16:32].max().item() == 0 and codes[2].max().item() == 0
+    sol.local_search(W, 3, 16, codes, scale, zero)
+    assert codes[1, 16:32].max().item() == 0 and codes[2].max().item() == 0
+    assert sol.last_device_status() == B.OK
+    # caller-supplied grid is honoured
+    Hh, _ = sol.get_hessian()
+    sc = torch.full((p, n // 16), 0.01, device=DEV)
+    zr = torch.full((p, n // 16), -0.035, device=DEV)
+    c2, s2, z2, _ = sol.quantize_layer(W, 3, 16, False, scale=sc, zero=zr, use_caller_grid=True)
+    assert torch.equal(s2, sc) and torch.equal(z2, zr) and c2.max().item() <= 7
+
+
+def test_error_paths():
+    n, p = 64, 4
+    spec = wl.small_case(n, p, 256, group_size=0, T=3)
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(n, p, T_max=3)
+    lib = sol.lib
+    with pytest.raises(B.AdmmqError) as e:                        # factor before any Hessian
+        sol.factor(rho=[0.1])
+    assert e.value.status == B.ERR_STATE
+    with pytest.raises(B.AdmmqError) as e:                        # accumulate before reset
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, 0, DEV))
+    assert e.value.status == B.ERR_STATE
+    sol.hessian_reset()
+    sol.hessian_accumulate(wl.gen_x_chunk(spec, 0, DEV))
+    with pytest.raises(B.AdmmqError) as e:                        # quantize before factor
+        sol.quantize_layer(W, 3)
+    assert e.value.status == B.ERR_STATE
+    for bad in (dict(rho=[0.1, -1.0]), dict(rho=[0.1] * 4), dict(rho=[0.1], kind=B.FACTOR_EIG)):
+        with pytest.raises(B.AdmmqError) as e:
+            sol.factor(**bad)
+        assert e.value.status in (B.ERR_INVALID_ARG, B.ERR_SHAPE, B.ERR_UNSUPPORTED)
+    sol.factor(rho=[0.1, 0.2, 0.4])
+    for kw in (dict(bits=1), dict(bits=9), dict(bits=3, group_size=48)):
+        with pytest.raises(B.AdmmqError) as e:
+            sol.quantize_layer(W, **kw)
+        assert e.value.status == B.ERR_SHAPE
+    with pytest.raises(B.AdmmqError) as e:                        # more output channels than the context holds
+        sol.quantize_layer(torch.zeros(p + 1, n, device=DEV), 3)
+    assert e.value.status == B.ERR_SHAPE
+    with pytest.raises(B.AdmmqError) as e:                        # misaligned pointer
+        sol.quantize_layer(torch.zeros(p * n + 1, device=DEV)[1:].view(p, n), 3)
+    assert e.value.status == B.ERR_INVALID_ARG
+    # non-finite weights: reported through the device status word, nothing faults
+    Wbad = W.clone()
+    Wbad[0, 0] = float("nan")
+    with pytest.raises(B.AdmmqError) as e:
+        sol.quantize_layer(Wbad, 3)
+    assert e.value.status == B.ERR_NONFINITE
+    # a Hessian with a non-positive diagonal entry: NOT_SPD through the status word
+    sol2 = B.Solver(n, p, T_max=3)
+    Hbad = torch.eye(n, device=DEV)
+    Hbad[5, 5] = -1.0
+    sol2.hessian_set(Hbad)
+    sol2.factor(rho=[0.1], damp_frac=0.0)
+    assert sol2.last_device_status() == B.ERR_NOT_SPD
+    # the context is still usable afterwards
+    sol2.hessian_set(torch.eye(n, device=DEV))
+    sol2.factor(rho=[0.1], damp_frac=0.0)
+    assert sol2.last_device_status() == B.OK
