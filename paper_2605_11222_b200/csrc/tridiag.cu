@@ -211,7 +211,9 @@ void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count) {
 // Y' = (T/rho + I)^{-1} Y row by row (one warp per output channel).  Both substitutions are first-
 // order linear recurrences x_i = y_i - l x_{i-1}; each lane runs its contiguous segment once to get
 // the segment's affine map, the 32 maps are combined by a warp scan, and a second run applies the
-// carry.  fp64 registers, fp32 shared-memory row, result written as two bf16 planes.
+// carry.  The factor (l, 1/d) of this penalty is staged once per CTA in shared memory in the same
+// padded layout as the rows, so every lane's walk through its segment is bank-conflict free.
+// fp64 registers, fp32 shared memory, result written as two bf16 planes.
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ int pad_index(int i, int seg, int stride) { return (i / seg) * stride + (i % seg); }
 
@@ -219,71 +221,91 @@ __global__ void tridiag_solve_kernel(const float* __restrict__ Y, int p, int n,
                                      const double* __restrict__ L, const double* __restrict__ invD,
                                      bf16* __restrict__ Yhi, bf16* __restrict__ Ylo, int seg, int stride) {
   extern __shared__ float smf[];
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  const int j = blockIdx.x * (blockDim.x >> 5) + wid;
-  if (j >= p) return;
-  float* rs = smf + (size_t)wid * stride * 32;
-  const float* y = Y + (long long)j * n;
-  for (int i = lane; i < n; i += 32) rs[pad_index(i, seg, stride)] = y[i];
-  __syncwarp();
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+  float* sl = smf;                         // l_i,     padded
+  float* sd = smf + stride * 32;           // 1 / d_i, padded
+  float* rs = smf + (size_t)(2 + wid) * stride * 32;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int q = pad_index(i, seg, stride);
+    sl[q] = (float)L[i];
+    sd[q] = (float)invD[i];
+  }
+  __syncthreads();
   const int a = min(n, lane * seg), b = min(n, (lane + 1) * seg);
-  float* mine = rs + lane * stride - a;            // mine[i] is element i for a <= i < b
-  // ---- forward substitution  x_i = y_i - l_{i-1} x_{i-1} ----
-  {
-    double cc = 0.0, mm = 1.0;
-    for (int i = a; i < b; ++i) {
-      const double li = (i > 0) ? L[i - 1] : 0.0;
-      cc = (double)mine[i] - li * cc;
-      mm *= -li;
-    }
+  const int len = b - a;
+  float* mine = rs + lane * stride;        // mine[t] is element a + t
+  const float* ml = sl + lane * stride;    // ml[t] = l_{a+t}
+  const float* md = sd + lane * stride;
+  // l_{a-1}: the multiplier that couples this segment to the previous one
+  const double l_prev = (a > 0 && a < n) ? (double)sl[pad_index(a - 1, seg, stride)] : 0.0;
+
+  for (int j = blockIdx.x * wpb + wid; j < p; j += gridDim.x * wpb) {
+    const float* y = Y + (long long)j * n;
+    for (int i = lane; i < n; i += 32) rs[pad_index(i, seg, stride)] = y[i];
+    __syncwarp();
+    // ---- forward substitution  x_i = y_i - l_{i-1} x_{i-1} ----
+    {
+      double cc = 0.0, mm = 1.0, lp = l_prev;
+#pragma unroll 4
+      for (int t = 0; t < len; ++t) {
+        cc = (double)mine[t] - lp * cc;
+        mm *= -lp;
+        lp = (double)ml[t];
+      }
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const double c2 = __shfl_up_sync(0xffffffffu, cc, off);
-      const double m2 = __shfl_up_sync(0xffffffffu, mm, off);
-      if (lane >= off) {
-        cc = cc + mm * c2;
-        mm = mm * m2;
+      for (int off = 1; off < 32; off <<= 1) {
+        const double c2 = __shfl_up_sync(0xffffffffu, cc, off);
+        const double m2 = __shfl_up_sync(0xffffffffu, mm, off);
+        if (lane >= off) {
+          cc = cc + mm * c2;
+          mm = mm * m2;
+        }
+      }
+      double x = __shfl_up_sync(0xffffffffu, cc, 1);
+      if (lane == 0) x = 0.0;
+      lp = l_prev;
+#pragma unroll 4
+      for (int t = 0; t < len; ++t) {
+        x = (double)mine[t] - lp * x;
+        lp = (double)ml[t];
+        mine[t] = (float)(x * (double)md[t]);
       }
     }
-    double x = __shfl_up_sync(0xffffffffu, cc, 1);
-    if (lane == 0) x = 0.0;
-    for (int i = a; i < b; ++i) {
-      const double li = (i > 0) ? L[i - 1] : 0.0;
-      x = (double)mine[i] - li * x;
-      mine[i] = (float)(x * invD[i]);
-    }
-  }
-  __syncwarp();
-  // ---- backward substitution  z_i = x_i - l_i z_{i+1} ----
-  {
-    double cc = 0.0, mm = 1.0;
-    for (int i = b - 1; i >= a; --i) {
-      const double li = L[i];
-      cc = (double)mine[i] - li * cc;
-      mm *= -li;
-    }
+    __syncwarp();
+    // ---- backward substitution  z_i = x_i - l_i z_{i+1} ----
+    {
+      double cc = 0.0, mm = 1.0;
+#pragma unroll 4
+      for (int t = len - 1; t >= 0; --t) {
+        const double li = (double)ml[t];
+        cc = (double)mine[t] - li * cc;
+        mm *= -li;
+      }
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const double c2 = __shfl_down_sync(0xffffffffu, cc, off);
-      const double m2 = __shfl_down_sync(0xffffffffu, mm, off);
-      if (lane + off < 32) {
-        cc = cc + mm * c2;
-        mm = mm * m2;
+      for (int off = 1; off < 32; off <<= 1) {
+        const double c2 = __shfl_down_sync(0xffffffffu, cc, off);
+        const double m2 = __shfl_down_sync(0xffffffffu, mm, off);
+        if (lane + off < 32) {
+          cc = cc + mm * c2;
+          mm = mm * m2;
+        }
+      }
+      double z = __shfl_down_sync(0xffffffffu, cc, 1);
+      if (lane == 31) z = 0.0;
+#pragma unroll 4
+      for (int t = len - 1; t >= 0; --t) {
+        z = (double)mine[t] - (double)ml[t] * z;
+        mine[t] = (float)z;
       }
     }
-    double z = __shfl_down_sync(0xffffffffu, cc, 1);
-    if (lane == 31) z = 0.0;
-    for (int i = b - 1; i >= a; --i) {
-      z = (double)mine[i] - L[i] * z;
-      mine[i] = (float)z;
+    __syncwarp();
+    for (int i = lane; i < n; i += 32) {
+      bf16 h, l;
+      split_bf16(rs[pad_index(i, seg, stride)], h, l);
+      Yhi[(long long)j * n + i] = h;
+      Ylo[(long long)j * n + i] = l;
     }
-  }
-  __syncwarp();
-  for (int i = lane; i < n; i += 32) {
-    bf16 h, l;
-    split_bf16(rs[pad_index(i, seg, stride)], h, l);
-    Yhi[(long long)j * n + i] = h;
-    Ylo[(long long)j * n + i] = l;
+    __syncwarp();
   }
 }
 
@@ -291,17 +313,19 @@ void launch_tridiag_solve(Ctx* c, int p, int stage) {
   const int n = c->n;
   const int seg = (n + 31) / 32;
   const int stride = seg | 1;
-  const size_t per_warp = (size_t)stride * 32 * sizeof(float);
-  int wpb = (int)((200 * 1024) / per_warp);
-  if (wpb > 8) wpb = 8;
+  const size_t per_row = (size_t)stride * 32 * sizeof(float);
+  int wpb = (int)((200 * 1024) / per_row) - 2;
+  if (wpb > 16) wpb = 16;
   if (wpb < 1) wpb = 1;
-  const size_t smem = per_warp * wpb;
+  const size_t smem = per_row * (wpb + 2);
   static bool attr_set = false;
   if (!attr_set) {
     cudaFuncSetAttribute(tridiag_solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
     attr_set = true;
   }
-  tridiag_solve_kernel<<<(p + wpb - 1) / wpb, wpb * 32, smem, c->stream>>>(
+  int blocks = (p + wpb - 1) / wpb;
+  if (blocks > c->num_sms) blocks = c->num_sms;
+  tridiag_solve_kernel<<<blocks, wpb * 32, smem, c->stream>>>(
       c->Y, p, n, c->stage_l + (long long)stage * n, c->stage_invd + (long long)stage * n, c->Y_hi,
       c->Y_lo, seg, stride);
   c->launches++;
