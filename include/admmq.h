@@ -201,6 +201,30 @@ admmq_status admmq_set_timing(admmq_ctx* ctx, int on);
 admmq_status admmq_reset_timing(admmq_ctx* ctx);
 admmq_status admmq_get_timing(admmq_ctx* ctx, int kind, double* h_total_ms, long long* h_count);
 
+/* ---- Error report without a context, a workspace or any allocation. ---------------------------------
+ * (The paper has no counterpart: this entry point exists for deployment, not for the method.)
+ * Computes Tr(E^T H E), E = (z0 + Delta k) - W_hat, like admmq_objective, for callers that cannot obtain
+ * device memory of their own: a job sharing the GPU with an engine that has already claimed all free
+ * HBM for its pool, code hosted by a framework that forbids allocations outside its arena, or a thread
+ * that must not cause the device-wide synchronisation an allocation may imply.  The caller passes only
+ * inputs and the output; the per-channel scratch of the reduction is a fixed array inside the library
+ * (ADMMQ_STATIC_MAX_D_OUT doubles = 128 KiB on every GPU that loads the library, until process exit).
+ *   d_H [d_in][d_in] fp32  damped unscaled Hessian (e.g. from admmq_get_hessian), symmetric
+ *   d_W0, d_codes [d_out][d_in]; d_scale, d_zero [d_out][d_in/group]; d_err: one DEVICE double (output)
+ *   cuda_stream: stream to enqueue on (NULL = default).  Asynchronous: read *d_err after the stream
+ *   has finished.
+ * Limits: d_out <= ADMMQ_STATIC_MAX_D_OUT and d_in <= ADMMQ_MAX_D_IN, otherwise ADMMQ_ERR_SHAPE and
+ * nothing is enqueued.  The call makes no cudaMalloc/cudaFree and calls no allocating routine.
+ * The scratch is shared by all calls and keeps the last call's contents (each call overwrites the
+ * entries it later reads, so nothing needs clearing): calls that overlap on the GPU -- different
+ * streams or threads without an ordering between them -- race; serialise them.  The first call on a
+ * device also looks up the scratch address and raises the kernel's shared-memory limit; make that first
+ * call outside any stream capture. */
+#define ADMMQ_STATIC_MAX_D_OUT 16384
+admmq_status admmq_objective_static(const float* d_H, int d_in, const float* d_W0, int d_out,
+                                    int group_size, const unsigned char* d_codes, const float* d_scale,
+                                    const float* d_zero, double* d_err, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif
