@@ -173,6 +173,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--tokens", type=int, default=262144)
+    ap.add_argument("--iters", type=int, default=0, help="ADMM iterations T (0: the workload's own, 300)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -185,6 +186,8 @@ def main():
     base = wl.config2(args.tokens)
     import dataclasses
     spec = dataclasses.replace(base, seed=base.seed + rank)
+    if args.iters > 0:
+        spec = dataclasses.replace(spec, T=args.iters)
 
     if args.impl == "reference":
         return run_reference(args, spec, wl)
