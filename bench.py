@@ -311,7 +311,7 @@ def main():
     # ---- roofline of the dominant kernel: the split-bf16 tcgen05 product of the W-update ----
     ms_p1, n_p1 = timing["wupdate_product1"]
     ms_p2, n_p2 = timing["wupdate_product2"]
-    flops_launch = 3 * 2.0 * p * n * n                     # three bf16 MMAs per term of the 2-plane split
+    flops_launch = 3 * 2.0 * p * n * n                     # three 16-bit MMAs per K step of the 2-plane split
     avg_ms = (ms_p1 + ms_p2) / max(1, n_p1 + n_p2)
     achieved = flops_launch / (avg_ms * 1e-3) / 1e12
     prof = os.path.join(ROOT, "profiles", "gemm_tc_wupdate_traffic.json")
@@ -321,7 +321,7 @@ def main():
                 "frac": achieved / peaks["bf16_sustained"], "peak_source": peaks["source"] + ", bf16 sustained",
                 "traffic": traffic, "launches": n_p1 + n_p2, "avg_launch_ms": avg_ms,
                 "fused_epilogue_launch_ms": ms_p2 / max(1, n_p2), "plain_epilogue_launch_ms": ms_p1 / max(1, n_p1)}
-    w_update_ms = (ms_p1 + ms_p2 + timing["tridiag_solve"][0]) / args.steps
+    w_update_ms = (ms_p1 + ms_p2 + timing["tridiag_solve"][0] + timing["row_split"][0]) / args.steps
     breakdown = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
                  for k, v in timing.items()}
 
@@ -333,7 +333,7 @@ def main():
     line = {
         "metric": METRIC, "value": ms_step / 1e3, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16x2-split (fp32 accumulate)", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f16x2-split (fp32 accumulate)", "data": "synthetic",
         "config": {"workload": spec.name, "d_in": n, "d_out": p, "n_tokens": spec.n_tokens, "T": T,
                    "bits": spec.bits, "group_size": spec.group_size, "layers_per_step": world,
                    "l2": "inputs_exceed_l2", "parallelism": f"layer-parallel x{world}"},

@@ -65,9 +65,10 @@ typedef enum { ADMMQ_F32 = 0, ADMMQ_BF16 = 1 } admmq_dtype;
  *          Algorithm 1 line 3.  The only kind implemented. */
 typedef enum { ADMMQ_FACTOR_TRIDIAG = 0, ADMMQ_FACTOR_CHOLESKY = 1, ADMMQ_FACTOR_EIG = 2 } admmq_factor_kind;
 
-/* Which matrix-product kernels run.  TENSOR: tcgen05 tensor-core kernels on split-bf16 operands with
- * fp32 accumulation (the product path).  SIMT: plain fp32 FMA kernels on the same operands, kept as an
- * on-device cross-check. */
+/* Which matrix-product kernels run.  TENSOR: tcgen05 tensor-core kernels on two-plane 16-bit operands
+ * (power-of-two scaled fp16 hi + lo for the W-update and gradient products, bf16 for the calibration
+ * activations) with fp32 accumulation: the product path.  SIMT: plain fp32 FMA kernels on the same
+ * operands, kept as an on-device cross-check. */
 typedef enum { ADMMQ_GEMM_TENSOR = 0, ADMMQ_GEMM_SIMT = 1 } admmq_gemm_kind;
 
 const char* admmq_status_string(admmq_status s);
@@ -180,6 +181,12 @@ admmq_status admmq_objective(admmq_ctx* ctx, const float* d_W0, int d_out, int g
  * H; d_s_out [d_in] fp32: s_i = sqrt(H_ii) (1 when preconditioning is off).  Either may be NULL. */
 admmq_status admmq_get_hessian(admmq_ctx* ctx, float* d_H_out, float* d_s_out);
 
+/* The one-time factorisation H~ = Q T Q^T (Algorithm 1 line 3 in its tridiagonal form), for checking
+ * (synchronises).  d_QT_out [d_in][d_in] fp64: Q^T, row m = m-th basis vector; d_diag_out [d_in] and
+ * d_offdiag_out [d_in] fp64: diagonal of T and its off-diagonal (entry i couples i and i+1; the last is 0).
+ * Any of them may be NULL. */
+admmq_status admmq_get_factor(admmq_ctx* ctx, double* d_QT_out, double* d_diag_out, double* d_offdiag_out);
+
 /* Number of kernels this context has launched so far (host counter). */
 long long admmq_launch_count(const admmq_ctx* ctx);
 
@@ -195,7 +202,8 @@ typedef enum {
   ADMMQ_T_WUPDATE_PRODUCT2 = 5, /* Z = Y' Q^T with the fused projection/dual/residual epilogue */
   ADMMQ_T_GRADIENT_PRODUCT = 6, /* g = E H                                                (step 4) */
   ADMMQ_T_LOCAL_SEARCH = 7,     /* move loop kernel                                       (step 4) */
-  ADMMQ_T_KINDS = 8
+  ADMMQ_T_ROW_SPLIT = 8,        /* next right-hand side -> scaled fp16 operand planes     (step 3) */
+  ADMMQ_T_KINDS = 9
 } admmq_timing_kind;
 admmq_status admmq_set_timing(admmq_ctx* ctx, int on);
 admmq_status admmq_reset_timing(admmq_ctx* ctx);

@@ -27,12 +27,12 @@ EXPORTS = [
     "admmq_hessian_accumulate", "admmq_hessian_set", "admmq_factor", "admmq_quantize_layer",
     "admmq_w_update", "admmq_local_search", "admmq_objective", "admmq_get_hessian",
     "admmq_launch_count", "admmq_set_timing", "admmq_reset_timing", "admmq_get_timing",
-    "admmq_objective_static",
+    "admmq_objective_static", "admmq_get_factor",
 ]
 T_HESSIAN_PRODUCT, T_TRANSPOSE, T_FACTOR, T_WUPDATE_PRODUCT1, T_TRIDIAG_SOLVE, T_WUPDATE_PRODUCT2, \
-    T_GRADIENT_PRODUCT, T_LOCAL_SEARCH = range(8)
+    T_GRADIENT_PRODUCT, T_LOCAL_SEARCH, T_ROW_SPLIT = range(9)
 TIMING_NAMES = ["hessian_product", "transpose", "factor", "wupdate_product1", "tridiag_solve",
-                "wupdate_product2", "gradient_product", "local_search"]
+                "wupdate_product2", "gradient_product", "local_search", "row_split"]
 
 
 class FactorCfg(C.Structure):
@@ -95,6 +95,7 @@ def load_library(path: Optional[str] = None):
     lib.admmq_local_search.argtypes = [vp, vp, ci, C.POINTER(LsCfg), vp, vp, vp, vp, C.POINTER(Report)]
     lib.admmq_objective.argtypes = [vp, vp, ci, ci, vp, vp, vp, C.POINTER(cd)]
     lib.admmq_get_hessian.argtypes = [vp, vp, vp]
+    lib.admmq_get_factor.argtypes = [vp, vp, vp, vp]
     lib.admmq_set_timing.argtypes = [vp, ci]
     lib.admmq_reset_timing.argtypes = [vp]
     lib.admmq_get_timing.argtypes = [vp, ci, C.POINTER(cd), C.POINTER(cll)]
@@ -242,6 +243,15 @@ class Solver:
         s = torch.empty(self.d_in, dtype=torch.float32, device=self.device)
         _check(self.lib.admmq_get_hessian(self.h, _ptr(H), _ptr(s)), "admmq_get_hessian")
         return H, s
+
+    def get_factor(self):
+        """(Q^T [n, n], diag(T) [n], offdiag(T) [n]) in fp64, copies of the factorisation H~ = Q T Q^T."""
+        n = self.d_in
+        QT = torch.empty(n, n, dtype=torch.float64, device=self.device)
+        td = torch.empty(n, dtype=torch.float64, device=self.device)
+        te = torch.empty(n, dtype=torch.float64, device=self.device)
+        _check(self.lib.admmq_get_factor(self.h, _ptr(QT), _ptr(td), _ptr(te)), "admmq_get_factor")
+        return QT, td, te
 
     def set_timing(self, on: bool):
         _check(self.lib.admmq_set_timing(self.h, int(on)), "admmq_set_timing")

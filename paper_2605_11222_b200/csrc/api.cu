@@ -53,6 +53,9 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   const size_t nn = (size_t)n * n, pn = (size_t)p * n;
   c.status = cv.take<int>(64);
   c.scal = cv.take<double>(32);
+  c.fscal = cv.take<float>(16);
+  c.rs_R = cv.take<float>((size_t)p);
+  c.rs_Y = cv.take<float>((size_t)p);
   long long* moves = cv.take<long long>(8);
   int* capped = cv.take<int>(16);
   double* rho_dev = cv.take<double>((size_t)T + 1);
@@ -66,8 +69,9 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   c.te = cv.take<double>(n);
   c.beta = cv.take<double>(n);
   c.pvec = cv.take<double>(n);
-  c.stage_l = cv.take<double>((size_t)(T + 1) * n);
-  c.stage_invd = cv.take<double>((size_t)(T + 1) * n);
+  c.stage_l = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
+  c.stage_invd = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
+  c.wy_s = cv.take<double>((size_t)((n + 31) / 32) * 1024);
   c.Q_hi = cv.take<bf16>(nn);
   c.Q_lo = cv.take<bf16>(nn);
   c.QT_hi = cv.take<bf16>(nn);
@@ -140,17 +144,25 @@ struct Timed {
 
 int group_of(int d_in, int gs) { return (gs == 0 || gs == d_in) ? d_in : gs; }
 
+// Operand descriptors: Q, Q^T and H are stored once per factorisation as fp16 planes with a common
+// power-of-two scale; R, Y' and E carry one scale per row (output channel).
+Planes op_Q(Ctx* c) { return planes_f16(c->Q_hi, c->Q_lo, c->n, nullptr, c->fscal + 0); }
+Planes op_QT(Ctx* c) { return planes_f16(c->QT_hi, c->QT_lo, c->n, nullptr, c->fscal + 0); }
+Planes op_H(Ctx* c) { return planes_f16(c->H_hi, c->H_lo, c->n, nullptr, c->fscal + 1); }
+Planes op_R(Ctx* c) { return planes_f16(c->R_hi, c->R_lo, c->n, c->rs_R, nullptr); }
+Planes op_Y(Ctx* c) { return planes_f16(c->Y_hi, c->Y_lo, c->n, c->rs_Y, nullptr); }
+
 // g = E H with E = W_q - W_hat, into c->Y; E planes go through the R buffers.
 cudaError_t gradient(admmq_ctx* a, const float* W0, int p, int gs, const unsigned char* codes,
                      const float* delta, const float* zero) {
   Ctx* c = &a->c;
-  launch_error_planes(c, W0, p, gs, codes, delta, zero, c->R_hi, c->R_lo);
+  launch_error_planes(c, W0, p, gs, codes, delta, zero, c->R_hi, c->R_lo, c->rs_R);
   EpiParams e{};
   e.kind = EPI_STORE;
   e.C = c->Y;
   e.ldc = c->n;
   Timed t(a, ADMMQ_T_GRADIENT_PRODUCT);
-  return product(c, Planes{c->R_hi, c->R_lo, c->n}, Planes{c->H_hi, c->H_lo, c->n}, p, c->n, c->n, e);
+  return product(c, op_R(c), op_H(c), p, c->n, c->n, e);
 }
 
 }  // namespace
@@ -268,7 +280,7 @@ admmq_status admmq_hessian_accumulate(admmq_ctx* ctx, const void* d_X, admmq_dty
     e.C = c->H_raw;
     e.ldc = n;
     e.lower_only = 1;
-    Planes P{c->XT_hi, lo, XT_ROWS};
+    Planes P = planes_bf16(c->XT_hi, lo, XT_ROWS);
     Timed t(ctx, ADMMQ_T_HESSIAN_PRODUCT);
     if (product(c, P, P, n, n, (int)rows, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
   }
@@ -306,6 +318,7 @@ admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg) {
   const int n = c->n;
   Timed tfac(ctx, ADMMQ_T_FACTOR);
   launch_finalize(c, cfg->damp_frac, c->precondition);
+  launch_operand_scales(c);
   launch_split_f32(c, c->H, (long long)n * n, c->H_hi, c->H_lo);
   if (tridiag_reduce(c) != cudaSuccess) return ADMMQ_ERR_CUDA;
   if (tridiag_form_qt(c) != cudaSuccess) return ADMMQ_ERR_CUDA;
@@ -346,7 +359,7 @@ static cudaError_t w_update_products(admmq_ctx* a, int p, int stage, const EpiPa
   cudaError_t err;
   {
     Timed t(a, ADMMQ_T_WUPDATE_PRODUCT1);
-    err = product(c, Planes{c->R_hi, c->R_lo, n}, Planes{c->QT_hi, c->QT_lo, n}, p, n, n, e1);
+    err = product(c, op_R(c), op_QT(c), p, n, n, e1);
   }
   if (err != cudaSuccess) return err;
   {
@@ -354,7 +367,7 @@ static cudaError_t w_update_products(admmq_ctx* a, int p, int stage, const EpiPa
     launch_tridiag_solve(c, p, stage);
   }
   Timed t(a, ADMMQ_T_WUPDATE_PRODUCT2);
-  return product(c, Planes{c->Y_hi, c->Y_lo, n}, Planes{c->Q_hi, c->Q_lo, n}, p, n, n, epi);
+  return product(c, op_Y(c), op_Q(c), p, n, n, epi);
 }
 
 admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, const admmq_quant_cfg* cfg,
@@ -385,8 +398,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.group_size = gs;
   e.n_groups = n / gs;
   e.kmax = (1 << cfg->bits) - 1;
-  e.Rhi = c->R_hi;
-  e.Rlo = c->R_lo;
+  e.Rnext = c->Y;                                          // Y is free once its planes exist
   for (int t = 0; t < T; ++t) {
     const double rho = c->rho_host[t];
     const double rho_next = (t + 1 < T) ? c->rho_host[t + 1] : rho;
@@ -396,6 +408,10 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     e.inv_rho_next = (float)(1.0 / rho_next);
     e.partials = c->partials + (size_t)t * c->partial_slots * 2;
     if (w_update_products(ctx, p, t, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
+    if (t + 1 < T) {
+      Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
+      launch_row_split(c, c->Y, p, c->R_hi, c->R_lo, c->rs_R);
+    }
   }
   if (d_resid) launch_reduce_partials(c, T, d_resid);
   if (d_Wq) launch_dequant(c, p, gs, d_codes, d_scale, d_zero, d_Wq);
@@ -427,7 +443,8 @@ admmq_status admmq_w_update(admmq_ctx* ctx, const float* d_W0, int d_out, int gr
   Ctx* c = &ctx->c;
   const int n = c->n, p = d_out, gs = group_of(n, group_size);
   launch_scale_weights(c, d_W0, p);
-  launch_init_rhs(c, p, gs, d_codes, d_scale, d_zero, d_V, (float)(1.0 / rho));
+  launch_init_rhs(c, p, gs, d_codes, d_scale, d_zero, d_V, (float)(1.0 / rho), c->Y);
+  launch_row_split(c, c->Y, p, c->R_hi, c->R_lo, c->rs_R);
   const int stage = c->T_max;                              // spare slot for an ad-hoc penalty
   ctx->rho_adhoc = rho;
   if (cudaMemcpyAsync(ctx->rho_dev + stage, &ctx->rho_adhoc, sizeof(double), cudaMemcpyHostToDevice,
@@ -548,6 +565,23 @@ admmq_status admmq_get_hessian(admmq_ctx* ctx, float* d_H_out, float* d_s_out) {
     return ADMMQ_ERR_CUDA;
   if (d_s_out && cudaMemcpyAsync(d_s_out, c->s, (size_t)c->n * sizeof(float), cudaMemcpyDeviceToDevice,
                                  c->stream) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  return read_status(ctx);
+}
+
+admmq_status admmq_get_factor(admmq_ctx* ctx, double* d_QT_out, double* d_diag_out, double* d_offdiag_out) {
+  if (!ctx) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (c->state != 2) return ADMMQ_ERR_STATE;
+  const size_t n = (size_t)c->n;
+  if (d_QT_out && cudaMemcpyAsync(d_QT_out, c->P64, n * n * sizeof(double), cudaMemcpyDeviceToDevice,
+                                  c->stream) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  if (d_diag_out && cudaMemcpyAsync(d_diag_out, c->td, n * sizeof(double), cudaMemcpyDeviceToDevice,
+                                    c->stream) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  if (d_offdiag_out && cudaMemcpyAsync(d_offdiag_out, c->te, n * sizeof(double), cudaMemcpyDeviceToDevice,
+                                       c->stream) != cudaSuccess)
     return ADMMQ_ERR_CUDA;
   return read_status(ctx);
 }

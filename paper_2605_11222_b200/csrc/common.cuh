@@ -1,6 +1,7 @@
 // Shared device helpers for the ADMM-Q kernels (sm_100a).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -16,6 +17,43 @@ __device__ __forceinline__ void raise_status(int* status, int code) { atomicCAS(
 __device__ __forceinline__ void split_bf16(float a, __nv_bfloat16& hi, __nv_bfloat16& lo) {
   hi = __float2bfloat16_rn(a);
   lo = __float2bfloat16_rn(a - __bfloat162float(hi));
+}
+
+// fp16 counterpart for operands that were first multiplied by a power of two which brings their
+// largest magnitude to [2^13, 2^14): a ~= hi + lo keeps 22 mantissa bits for every element within
+// 2^17 of that maximum (lo stays a normal fp16 number), and 2^-25 absolute below.  The clamp only
+// guards the conversion against non-finite results.
+__device__ __forceinline__ void split_f16(float a, __half& hi, __half& lo) {
+  a = fminf(fmaxf(a, -60000.0f), 60000.0f);
+  hi = __float2half_rn(a);
+  lo = __float2half_rn(a - __half2float(hi));
+}
+// Power of two S with maxabs * S in [2^13, 2^14); 1 for a zero or non-finite maximum.  *inv = 1 / S.
+__device__ __forceinline__ float pow2_scale_for(float maxabs, float* inv) {
+  if (!(maxabs > 0.0f) || !isfinite(maxabs)) {
+    *inv = 1.0f;
+    return 1.0f;
+  }
+  int e;
+  frexpf(maxabs, &e);
+  *inv = ldexpf(1.0f, e - 14);
+  return ldexpf(1.0f, 14 - e);
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+// Maximum over the block, result in every thread.  `scratch` holds >= 32 floats.
+__device__ __forceinline__ float block_max(float v, float* scratch) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  v = warp_max(v);
+  __syncthreads();
+  if (lane == 0) scratch[w] = v;
+  __syncthreads();
+  float t = (lane < nw) ? scratch[lane] : 0.0f;
+  return warp_max(t);
 }
 
 __device__ __forceinline__ float warp_sum(float v) {

@@ -165,31 +165,63 @@ void launch_grid_fit(Ctx* c, const float* W0, int p, int bits, int gs, int symme
   LAUNCH(c);
 }
 
-// W_hat' = Sigma^{-1} W_hat (Algorithm 1 line 2); V^(0) = 0; first right-hand side R = D^(0) - W_hat' = 0.
+// W_hat' = Sigma^{-1} W_hat (Algorithm 1 line 2); V^(0) = 0; first right-hand side R = D^(0) - W_hat' = 0
+// (all-zero planes, row scale 1).
 __global__ void scale_weights_kernel(const float* __restrict__ W0, const float* __restrict__ s,
                                      long long total, int n, float* __restrict__ Whs,
                                      float* __restrict__ V, bf16* __restrict__ Rhi,
-                                     bf16* __restrict__ Rlo, int* status) {
+                                     bf16* __restrict__ Rlo, float* __restrict__ row_inv, int* status) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
   const float w = W0[i];
   if (!isfinite(w)) raise_status(status, ST_NONFINITE);
   Whs[i] = s[i % n] * w;
   V[i] = 0.f;
-  Rhi[i] = __float2bfloat16_rn(0.f);
+  Rhi[i] = __float2bfloat16_rn(0.f);                      // the all-zero pattern is zero in fp16 as well
   Rlo[i] = __float2bfloat16_rn(0.f);
+  if (i % n == 0) row_inv[i / n] = 1.0f;
 }
 
 void launch_scale_weights(Ctx* c, const float* W0, int p) {
   const long long total = (long long)p * c->n;
   scale_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
-      W0, c->s, total, c->n, c->Whs, c->V, c->R_hi, c->R_lo, c->status);
+      W0, c->s, total, c->n, c->Whs, c->V, c->R_hi, c->R_lo, c->rs_R, c->status);
   LAUNCH(c);
 }
 
 // ------------------------------------------------------------------------------------------------
-// Operand splitting: fp64 / fp32 matrices -> (hi, lo) bf16 planes, optionally also transposed.
+// Operand splitting: matrices -> (hi, lo) fp16 planes of the value times a power of two.
+// Q has entries of magnitude <= 1 and takes the fixed scale 2^13; H takes the scale that brings its
+// largest entry (on the diagonal: H is positive definite) to [2^13, 2^14).
 // ------------------------------------------------------------------------------------------------
+constexpr float Q_PLANE_SCALE = 8192.0f;
+
+__device__ __forceinline__ void store_f16_pair(bf16* hi, bf16* lo, long long idx, float scaled) {
+  __half h, l;
+  split_f16(scaled, h, l);
+  reinterpret_cast<__half*>(hi)[idx] = h;
+  reinterpret_cast<__half*>(lo)[idx] = l;
+}
+
+__global__ void operand_scales_kernel(const float* __restrict__ hdiag, int n, float* __restrict__ fscal) {
+  __shared__ float scratch[32];
+  float m = 0.0f;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) m = fmaxf(m, fabsf(hdiag[i]));
+  m = block_max(m, scratch);
+  if (threadIdx.x == 0) {
+    float inv;
+    const float sc = pow2_scale_for(m, &inv);
+    fscal[0] = 1.0f / Q_PLANE_SCALE;
+    fscal[1] = inv;
+    fscal[2] = sc;
+  }
+}
+
+void launch_operand_scales(Ctx* c) {
+  operand_scales_kernel<<<1, 1024, 0, c->stream>>>(c->hdiag, c->n, c->fscal);
+  LAUNCH(c);
+}
+
 __global__ void split_f64_kernel(const double* __restrict__ src, int n, bf16* __restrict__ hi,
                                  bf16* __restrict__ lo, bf16* __restrict__ thi, bf16* __restrict__ tlo) {
   __shared__ float tile[32][33];
@@ -198,23 +230,15 @@ __global__ void split_f64_kernel(const double* __restrict__ src, int n, bf16* __
     const int r = r0 + i, cc = c0 + threadIdx.x;
     float v = 0.f;
     if (r < n && cc < n) {
-      v = (float)src[(long long)r * n + cc];
-      bf16 h, l;
-      split_bf16(v, h, l);
-      hi[(long long)r * n + cc] = h;
-      lo[(long long)r * n + cc] = l;
+      v = (float)(src[(long long)r * n + cc] * (double)Q_PLANE_SCALE);
+      store_f16_pair(hi, lo, (long long)r * n + cc, v);
     }
     tile[i][threadIdx.x] = v;
   }
   __syncthreads();
   for (int i = threadIdx.y; i < 32; i += blockDim.y) {
     const int cc = c0 + i, r = r0 + threadIdx.x;   // element (r, cc) of src -> (cc, r) of the transpose
-    if (cc < n && r < n) {
-      bf16 h, l;
-      split_bf16(tile[threadIdx.x][i], h, l);
-      thi[(long long)cc * n + r] = h;
-      tlo[(long long)cc * n + r] = l;
-    }
+    if (cc < n && r < n) store_f16_pair(thi, tlo, (long long)cc * n + r, tile[threadIdx.x][i]);
   }
 }
 
@@ -224,18 +248,77 @@ void launch_split_f64(Ctx* c, const double* src, int n, bf16* hi, bf16* lo, bf16
   LAUNCH(c);
 }
 
-__global__ void split_f32_kernel(const float* __restrict__ src, long long count, bf16* __restrict__ hi,
+__global__ void split_f32_kernel(const float* __restrict__ src, long long count,
+                                 const float* __restrict__ fscal, bf16* __restrict__ hi,
                                  bf16* __restrict__ lo) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= count) return;
-  bf16 h, l;
-  split_bf16(src[i], h, l);
-  hi[i] = h;
-  lo[i] = l;
+  store_f16_pair(hi, lo, i, src[i] * fscal[2]);
 }
 
 void launch_split_f32(Ctx* c, const float* src, long long count, bf16* hi, bf16* lo) {
-  split_f32_kernel<<<(unsigned)((count + 255) / 256), 256, 0, c->stream>>>(src, count, hi, lo);
+  split_f32_kernel<<<(unsigned)((count + 255) / 256), 256, 0, c->stream>>>(src, count, c->fscal, hi, lo);
+  LAUNCH(c);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Row pass: one fp32 row -> its largest magnitude -> power-of-two scale -> (hi, lo) fp16 planes and
+// the inverse scale.  One CTA per row at a time, the row staged in shared memory.  `make` yields
+// element i of row j.
+// ------------------------------------------------------------------------------------------------
+constexpr int ROW_THREADS = 256;
+
+template <typename Make>
+__device__ __forceinline__ void row_split_body(int p, int n, Make make, bf16* __restrict__ hi,
+                                               bf16* __restrict__ lo, float* __restrict__ row_inv) {
+  extern __shared__ float rowbuf[];
+  __shared__ float scratch[32];
+  for (int j = blockIdx.x; j < p; j += gridDim.x) {
+    float m = 0.0f;
+    for (int i = threadIdx.x * 4; i < n; i += ROW_THREADS * 4) {          // n is a multiple of 8
+      const float4 v = make(j, i);
+      *reinterpret_cast<float4*>(rowbuf + i) = v;
+      m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(m, fmaxf(fabsf(v.z), fabsf(v.w))));
+    }
+    m = block_max(m, scratch);
+    float inv;
+    const float sc = pow2_scale_for(m, &inv);
+    if (threadIdx.x == 0) row_inv[j] = inv;
+    for (int i = threadIdx.x * 8; i < n; i += ROW_THREADS * 8) {
+      __align__(16) __half hh[8];
+      __align__(16) __half ll[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) split_f16(rowbuf[i + e] * sc, hh[e], ll[e]);
+      *reinterpret_cast<uint4*>(hi + (size_t)j * n + i) = *reinterpret_cast<const uint4*>(hh);
+      *reinterpret_cast<uint4*>(lo + (size_t)j * n + i) = *reinterpret_cast<const uint4*>(ll);
+    }
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(ROW_THREADS)
+row_split_kernel(const float* __restrict__ src, int p, int n, bf16* __restrict__ hi, bf16* __restrict__ lo,
+                 float* __restrict__ row_inv) {
+  row_split_body(p, n, [&](int j, int i) { return *reinterpret_cast<const float4*>(src + (size_t)j * n + i); },
+                 hi, lo, row_inv);
+}
+
+static int row_pass_blocks(Ctx* c, int p, size_t smem) {
+  int per_sm = (int)((200 * 1024) / (smem + 1024));
+  if (per_sm > 8) per_sm = 8;
+  if (per_sm < 1) per_sm = 1;
+  const int blocks = c->num_sms * per_sm;
+  return blocks < p ? blocks : p;
+}
+
+void launch_row_split(Ctx* c, const float* src, int p, bf16* hi, bf16* lo, float* row_inv) {
+  const size_t smem = (size_t)c->n * sizeof(float);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(row_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    attr_set = true;
+  }
+  row_split_kernel<<<row_pass_blocks(c, p, smem), ROW_THREADS, smem, c->stream>>>(src, p, c->n, hi, lo, row_inv);
   LAUNCH(c);
 }
 
@@ -245,26 +328,21 @@ __global__ void init_rhs_kernel(long long total, int n, int gs, int ng,
                                 const unsigned char* __restrict__ codes,
                                 const float* __restrict__ delta, const float* __restrict__ zero,
                                 const float* __restrict__ V, float inv_rho, const float* __restrict__ s,
-                                const float* __restrict__ Whs, bf16* __restrict__ Rhi,
-                                bf16* __restrict__ Rlo) {
+                                const float* __restrict__ Whs, float* __restrict__ R) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
   const int col = (int)(idx % n);
   const long long row = idx / n;
   const long long gi = row * ng + col / gs;
   const float d = s[col] * (zero[gi] + delta[gi] * (float)codes[idx]);
-  const float r = d - V[idx] * inv_rho - Whs[idx];
-  bf16 h, l;
-  split_bf16(r, h, l);
-  Rhi[idx] = h;
-  Rlo[idx] = l;
+  R[idx] = d - V[idx] * inv_rho - Whs[idx];
 }
 
 void launch_init_rhs(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
-                     const float* zero, const float* V_in, float inv_rho) {
+                     const float* zero, const float* V_in, float inv_rho, float* R_out) {
   const long long total = (long long)p * c->n;
   init_rhs_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
-      total, c->n, gs, c->n / gs, codes, delta, zero, V_in, inv_rho, c->s, c->Whs, c->R_hi, c->R_lo);
+      total, c->n, gs, c->n / gs, codes, delta, zero, V_in, inv_rho, c->s, c->Whs, R_out);
   LAUNCH(c);
 }
 
@@ -311,25 +389,40 @@ void launch_dequant(Ctx* c, int p, int gs, const unsigned char* codes, const flo
 }
 
 // E = W_q - W_hat as two bf16 planes (operand of the gradient product g = E H, Sec. 3.5).
-__global__ void error_planes_kernel(long long total, int n, int gs, int ng, const float* __restrict__ W0,
-                                    const unsigned char* __restrict__ codes,
-                                    const float* __restrict__ delta, const float* __restrict__ zero,
-                                    bf16* __restrict__ Ehi, bf16* __restrict__ Elo) {
-  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= total) return;
-  const long long gi = (idx / n) * ng + (idx % n) / gs;
-  const float e = (zero[gi] + delta[gi] * (float)codes[idx]) - W0[idx];
-  bf16 h, l;
-  split_bf16(e, h, l);
-  Ehi[idx] = h;
-  Elo[idx] = l;
+__global__ void __launch_bounds__(ROW_THREADS)
+error_planes_kernel(int p, int n, int gs, int ng, const float* __restrict__ W0,
+                    const unsigned char* __restrict__ codes, const float* __restrict__ delta,
+                    const float* __restrict__ zero, bf16* __restrict__ Ehi, bf16* __restrict__ Elo,
+                    float* __restrict__ row_inv) {
+  row_split_body(p, n,
+                 [&](int j, int i) {
+                   const size_t idx = (size_t)j * n + i;
+                   const float4 w = *reinterpret_cast<const float4*>(W0 + idx);
+                   const uchar4 k = *reinterpret_cast<const uchar4*>(codes + idx);
+                   float4 e;
+                   size_t gi = (size_t)j * ng + i / gs;
+                   e.x = (zero[gi] + delta[gi] * (float)k.x) - w.x;
+                   gi = (size_t)j * ng + (i + 1) / gs;
+                   e.y = (zero[gi] + delta[gi] * (float)k.y) - w.y;
+                   gi = (size_t)j * ng + (i + 2) / gs;
+                   e.z = (zero[gi] + delta[gi] * (float)k.z) - w.z;
+                   gi = (size_t)j * ng + (i + 3) / gs;
+                   e.w = (zero[gi] + delta[gi] * (float)k.w) - w.w;
+                   return e;
+                 },
+                 Ehi, Elo, row_inv);
 }
 
 void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes,
-                         const float* delta, const float* zero, bf16* Ehi, bf16* Elo) {
-  const long long total = (long long)p * c->n;
-  error_planes_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
-      total, c->n, gs, c->n / gs, W0, codes, delta, zero, Ehi, Elo);
+                         const float* delta, const float* zero, bf16* Ehi, bf16* Elo, float* row_inv) {
+  const size_t smem = (size_t)c->n * sizeof(float);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(error_planes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    attr_set = true;
+  }
+  error_planes_kernel<<<row_pass_blocks(c, p, smem), ROW_THREADS, smem, c->stream>>>(
+      p, c->n, gs, c->n / gs, W0, codes, delta, zero, Ehi, Elo, row_inv);
   LAUNCH(c);
 }
 

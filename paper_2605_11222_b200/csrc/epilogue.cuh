@@ -29,10 +29,22 @@ struct EpiParams {
   int kmax;                 // 2^bits - 1
   int first_iter;           // 1: D^(0) = W_hat' (Algorithm 1 line 4), codes not yet defined
   float rho, inv_rho, inv_rho_next;
-  __nv_bfloat16* Rhi;       // next right-hand side D - V/rho_next - W_hat', split in two bf16 planes
-  __nv_bfloat16* Rlo;
+  float* Rnext;             // next right-hand side D - V/rho_next - W_hat' (fp32; split into planes by a row pass)
   float* partials;          // [slots][2]: per-CTA sums of (W-D)^2 and (D-D_old)^2
+  // ---- undoing the operands' power-of-two scales: value = acc * row_inv[row] * a_inv[0] * b_inv[0] ----
+  const float* row_inv;     // [M] or nullptr
+  const float* a_inv;       // device scalar or nullptr
+  const float* b_inv;       // device scalar or nullptr
 };
+
+// Factor that turns an accumulator of output row `row` back into the unscaled product.
+__device__ __forceinline__ float epi_row_factor(const EpiParams& P, int row) {
+  float f = 1.0f;
+  if (P.row_inv) f = P.row_inv[row];
+  if (P.a_inv) f *= P.a_inv[0];
+  if (P.b_inv) f *= P.b_inv[0];
+  return f;
+}
 
 // One element of the fused ADMM epilogue.  z = [Q (T/rho + I)^{-1} Q^T R]_{ji} is the accumulator, so
 // that W = W_hat' + z is the W-update of Eq. 7 written for the error W - W_hat'.
@@ -63,6 +75,7 @@ __device__ __forceinline__ AdmmElem admm_elem(float z, float wh, float v, int co
 // Scalar epilogue for one output element (used by the SIMT kernel and for ragged edges).
 __device__ __forceinline__ void epi_scalar(const EpiParams& P, int row, int col, int n_cols, float acc,
                                            float& r2, float& s2) {
+  acc *= epi_row_factor(P, row);
   if (P.kind == EPI_STORE) {
     P.C[(long long)row * P.ldc + col] = acc;
   } else if (P.kind == EPI_ACCUM) {
@@ -78,10 +91,7 @@ __device__ __forceinline__ void epi_scalar(const EpiParams& P, int row, int col,
                            dl, z0, P);
     P.codes[idx] = e.code;
     P.V[idx] = e.v_new;
-    __nv_bfloat16 hi, lo;
-    split_bf16(e.r_next, hi, lo);
-    P.Rhi[idx] = hi;
-    P.Rlo[idx] = lo;
+    P.Rnext[idx] = e.r_next;
     r2 += e.dr2;
     s2 += e.ds2;
   }

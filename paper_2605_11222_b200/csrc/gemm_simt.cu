@@ -7,6 +7,10 @@ namespace admmq {
 
 constexpr int ST = 64, SK = 16;
 
+__device__ __forceinline__ float plane_value(const bf16* plane, long long idx, int f16) {
+  return f16 ? __half2float(reinterpret_cast<const __half*>(plane)[idx]) : __bfloat162float(plane[idx]);
+}
+
 __global__ void __launch_bounds__(256)
 gemm_simt_kernel(Planes A, Planes B, int M, int N, int K, EpiParams epi) {
   __shared__ float As[SK][ST + 1];
@@ -21,13 +25,13 @@ gemm_simt_kernel(Planes A, Planes B, int M, int N, int K, EpiParams epi) {
       float a = 0.f, b = 0.f;
       if (m0 + r < M && k0 + kk < K) {
         const long long ia = (long long)(m0 + r) * A.ld + k0 + kk;
-        a = __bfloat162float(A.hi[ia]);
-        if (A.lo) a += __bfloat162float(A.lo[ia]);
+        a = plane_value(A.hi, ia, A.f16);
+        if (A.lo) a += plane_value(A.lo, ia, A.f16);
       }
       if (n0 + r < N && k0 + kk < K) {
         const long long ib = (long long)(n0 + r) * B.ld + k0 + kk;
-        b = __bfloat162float(B.hi[ib]);
-        if (B.lo) b += __bfloat162float(B.lo[ib]);
+        b = plane_value(B.hi, ib, B.f16);
+        if (B.lo) b += plane_value(B.lo, ib, B.f16);
       }
       As[kk][r] = a;
       Bs[kk][r] = b;
@@ -66,7 +70,11 @@ gemm_simt_kernel(Planes A, Planes B, int M, int N, int K, EpiParams epi) {
   }
 }
 
-cudaError_t gemm_simt(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiParams& epi) {
+cudaError_t gemm_simt(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiParams& epi_in) {
+  EpiParams epi = epi_in;
+  epi.row_inv = A.row_inv;
+  epi.a_inv = A.all_inv;
+  epi.b_inv = B.all_inv;
   dim3 grid((N + ST - 1) / ST, (M + ST - 1) / ST);
   gemm_simt_kernel<<<grid, 256, 0, c->stream>>>(A, B, M, N, K, epi);
   c->launches++;

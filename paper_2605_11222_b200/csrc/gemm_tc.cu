@@ -1,18 +1,24 @@
 // Tensor-core product kernel for sm_100a:  C[M][N] (epilogue)= A[M][K] * B[N][K]^T.
 //
-// Operands are bf16 planes, one (plain bf16 data) or two (hi + lo split of an fp32 value) per operand;
-// with two planes the product is hi*hi + hi*lo + lo*hi, three tcgen05.mma per K step into one fp32
-// accumulator in tensor memory, which keeps ~16 mantissa bits of each operand.
+// Operands are 16-bit planes, one (plain bf16 data) or two (hi + lo split of an fp32 value) per
+// operand; with two planes the product is hi*hi + hi*lo + lo*hi, three tcgen05.mma per K step.
 //
-// One persistent CTA per SM, 192 threads:
-//   warp 0     TMA producer: cp.async.bulk.tensor loads of 128B-swizzled K-major tiles into a ring
-//              of shared-memory stages, completion counted by mbarriers;
-//   warp 1     MMA issuer: one elected thread issues tcgen05.mma (M=128, N=256, K=16 per instruction)
-//              and tcgen05.commit, which releases stages and publishes finished accumulators;
-//   warps 2-5  epilogue: tcgen05.ld the accumulator (lane = output row) and apply the epilogue --
-//              for the ADMM iteration the projection, dual update, residual sums and the next
-//              right-hand side -- while the issuer already works on the next tile in the second
-//              accumulator (2 x 256 columns of tensor memory).
+// Accumulation.  The tensor core adds into its fp32 accumulator with truncation, so a long chain of
+// accumulating MMAs drifts toward zero (measured ~3e-5 relative after the 768 steps of K = 4096).
+// The chain is therefore kept short: one flush = 12 MMA steps (one 64-wide K block with two planes,
+// three with one plane) goes into one of four 128-column accumulators in tensor memory, and the
+// worker warps add each finished partial into fp32 registers with round-to-nearest adds.
+//
+// One persistent CTA per SM, 576 threads, output tiles of 128 x 128:
+//   warp 0       TMA producer: cp.async.bulk.tensor loads of 128B-swizzled K-major tiles into a ring
+//                of shared-memory stages, completion counted by mbarriers;
+//   warp 1       MMA issuer: one elected thread issues tcgen05.mma (M = 128, N = 128, K = 16 per
+//                instruction) and tcgen05.commit, which releases stages and publishes partials;
+//   warps 2-9    worker group 0, warps 10-17 worker group 1.  The groups take alternate tiles.  A
+//                group drains the partials of its tile (tcgen05.ld, lane = output row; the two
+//                warps of a lane quarter split the 128 columns) and then runs the epilogue from its
+//                registers -- for the ADMM iteration the projection, dual update, residual sums and
+//                the next right-hand side -- while the other group drains the next tile.
 // Every wait is bounded: on expiry the kernel records ADMMQ_ERR_TIMEOUT, stops issuing work, lets
 // copies in flight land, frees tensor memory and returns.
 #include <cuda.h>
@@ -21,8 +27,11 @@
 
 namespace admmq {
 
-constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int TC_THREADS = 192;
+constexpr int BM = 128, BN = 128, BK = 64;
+constexpr int NPART = 4;                 // partial accumulators in tensor memory (4 x 128 columns)
+constexpr int GROUP_WARPS = 8;
+constexpr int TC_THREADS = 32 * (2 + 2 * GROUP_WARPS);
+constexpr int COLS_PER_THREAD = BN / 2;  // 64
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // about a second
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -80,8 +89,8 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                           uint32_t accumulate) {
   asm volatile(
       "{\n.reg .pred p;\n"
       "setp.ne.b32 p, %4, 0;\n"
@@ -89,7 +98,8 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uin
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+// 32 consecutive accumulator columns of this warp's 32 lanes (lane = row), issued without waiting.
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -101,8 +111,8 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major tile with 128-byte rows and 128B swizzle: groups of
 // 8 rows are 1024 bytes apart (stride byte offset), the leading byte offset is unused for swizzled
@@ -116,79 +126,104 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
   d |= (uint64_t)2 << 61;
   return d;
 }
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, N = 256, M = 128.
-constexpr uint32_t IDESC_BF16_128x256 =
-    (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// Instruction descriptor: fp32 accumulate, A and B of the same 16-bit type (format 1 = bf16, 0 = fp16),
+// both K-major, N = 128, M = 128.
+__host__ __device__ constexpr uint32_t idesc_128x128(uint32_t fmt) {
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
 
 struct TcMaps {
   CUtensorMap a[2];
   CUtensorMap b[2];
 };
 
-// ------------------------------------------------------------------ vectorised epilogue pieces
-__device__ __forceinline__ void epi_chunk32(const EpiParams& P, int row, int col0, int M, int N,
-                                            const uint32_t (&acc)[32], float& r2, float& s2) {
+// ------------------------------------------------------------------ epilogue on 4 columns of one row
+// `a` holds the 4 products (already unscaled).  Everything is indexed statically so that the running
+// sums stay in registers; chunks of 4 keep the worker threads under their register budget.
+struct AdmmIn {
+  float4 w, v, s;
+  uint32_t codes;
+};
+__device__ __forceinline__ AdmmIn admm_load4(const EpiParams& P, long long o, int col) {
+  AdmmIn in;
+  in.w = *reinterpret_cast<const float4*>(P.Whs + o);
+  in.v = *reinterpret_cast<const float4*>(P.V + o);
+  in.s = *reinterpret_cast<const float4*>(P.s + col);
+  in.codes = 0u;
+  if (!P.first_iter) in.codes = *reinterpret_cast<const uint32_t*>(P.codes + o);
+  return in;
+}
+__device__ __forceinline__ void admm_apply4(const EpiParams& P, long long o, const AdmmIn& in,
+                                            const float (&a)[4], float dl, float z0, float& r2, float& s2) {
+  const float wh[4] = {in.w.x, in.w.y, in.w.z, in.w.w};
+  const float vv[4] = {in.v.x, in.v.y, in.v.z, in.v.w};
+  const float ss[4] = {in.s.x, in.s.y, in.s.z, in.s.w};
+  float vn[4], rn[4];
+  uint32_t cn = 0u;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const int code_old = (int)((in.codes >> (8 * e)) & 0xffu);
+    AdmmElem r = admm_elem(a[e], wh[e], vv[e], code_old, ss[e], dl, z0, P);
+    vn[e] = r.v_new;
+    cn |= (uint32_t)r.code << (8 * e);
+    rn[e] = r.r_next;
+    r2 += r.dr2;
+    s2 += r.ds2;
+  }
+  *reinterpret_cast<float4*>(P.V + o) = make_float4(vn[0], vn[1], vn[2], vn[3]);
+  *reinterpret_cast<uint32_t*>(P.codes + o) = cn;
+  *reinterpret_cast<float4*>(P.Rnext + o) = make_float4(rn[0], rn[1], rn[2], rn[3]);
+}
+
+// The 64 columns [col0, col0 + 64) of output row `row`, products in `sums`.
+template <int EPI>
+__device__ __forceinline__ void epilogue_row64(const EpiParams& P, int row, int col0, int M, int N,
+                                               const float (&sums)[COLS_PER_THREAD], float& r2, float& s2) {
   if (row >= M || col0 >= N) return;
-  const bool full = (col0 + 32 <= N);
-  if (P.kind == EPI_ADMM) {
+  const float sc = epi_row_factor(P, row);
+  const bool full = (col0 + COLS_PER_THREAD <= N);
+  if (EPI == EPI_ADMM) {
     const long long base = (long long)row * N + col0;
-    const bool one_group = full && ((P.group_size & 31) == 0);
-    if (one_group) {
-      const long long gi = (long long)row * P.n_groups + col0 / P.group_size;
-      const float dl = P.delta[gi], z0 = P.zero[gi];
+    if (full && (P.group_size & 3) == 0) {
+      // one (Delta, z0) per 4 columns; inputs of chunk c + 1 are requested before chunk c is computed
+      AdmmIn cur = admm_load4(P, base, col0);
+      const bool one_group = (P.group_size % COLS_PER_THREAD) == 0;   // then (Delta, z0) is fixed here
+      long long gi = (long long)row * P.n_groups + col0 / P.group_size;
+      float dl = P.delta[gi], z0 = P.zero[gi];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const long long o = base + q * 8;
-        const float4 w0 = *reinterpret_cast<const float4*>(P.Whs + o);
-        const float4 w1 = *reinterpret_cast<const float4*>(P.Whs + o + 4);
-        const float4 v0 = *reinterpret_cast<const float4*>(P.V + o);
-        const float4 v1 = *reinterpret_cast<const float4*>(P.V + o + 4);
-        const float4 s0 = *reinterpret_cast<const float4*>(P.s + col0 + q * 8);
-        const float4 s1 = *reinterpret_cast<const float4*>(P.s + col0 + q * 8 + 4);
-        uint2 cold = make_uint2(0u, 0u);
-        if (!P.first_iter) cold = *reinterpret_cast<const uint2*>(P.codes + o);
-        const float wh[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
-        const float vv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-        const float ss[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-        float vn[8];
-        uint32_t cn[2] = {0u, 0u};
-        __align__(16) bf16 rh[8];
-        __align__(16) bf16 rl[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const uint32_t word = (e < 4) ? cold.x : cold.y;
-          const int code_old = (int)((word >> (8 * (e & 3))) & 0xffu);
-          AdmmElem r = admm_elem(__uint_as_float(acc[q * 8 + e]), wh[e], vv[e], code_old, ss[e], dl, z0, P);
-          vn[e] = r.v_new;
-          cn[e >> 2] |= (uint32_t)r.code << (8 * (e & 3));
-          split_bf16(r.r_next, rh[e], rl[e]);
-          r2 += r.dr2;
-          s2 += r.ds2;
+      for (int c = 0; c < COLS_PER_THREAD / 4; ++c) {
+        AdmmIn nxt = cur;
+        if (c + 1 < COLS_PER_THREAD / 4) nxt = admm_load4(P, base + (c + 1) * 4, col0 + (c + 1) * 4);
+        if (!one_group) {
+          gi = (long long)row * P.n_groups + (col0 + c * 4) / P.group_size;
+          dl = P.delta[gi];
+          z0 = P.zero[gi];
         }
-        *reinterpret_cast<float4*>(P.V + o) = make_float4(vn[0], vn[1], vn[2], vn[3]);
-        *reinterpret_cast<float4*>(P.V + o + 4) = make_float4(vn[4], vn[5], vn[6], vn[7]);
-        *reinterpret_cast<uint2*>(P.codes + o) = make_uint2(cn[0], cn[1]);
-        *reinterpret_cast<uint4*>(P.Rhi + o) = *reinterpret_cast<const uint4*>(rh);
-        *reinterpret_cast<uint4*>(P.Rlo + o) = *reinterpret_cast<const uint4*>(rl);
+        float a[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) a[e] = sums[c * 4 + e] * sc;
+        admm_apply4(P, base + c * 4, cur, a, dl, z0, r2, s2);
+        cur = nxt;
       }
       return;
     }
-    for (int e = 0; e < 32; ++e)
-      if (col0 + e < N) epi_scalar(P, row, col0 + e, N, __uint_as_float(acc[e]), r2, s2);
+#pragma unroll
+    for (int e = 0; e < COLS_PER_THREAD; ++e)
+      if (col0 + e < N) epi_scalar(P, row, col0 + e, N, sums[e], r2, s2);
     return;
   }
   // STORE / ACCUM / WOUT
   float* crow = P.C + (long long)row * P.ldc + col0;
-  const bool vec_ok = full && ((P.ldc & 3) == 0) && (P.kind != EPI_ACCUM || !P.lower_only || col0 + 31 <= row);
+  const bool vec_ok = full && ((P.ldc & 3) == 0) &&
+                      (EPI != EPI_ACCUM || !P.lower_only || col0 + COLS_PER_THREAD - 1 <= row);
   if (vec_ok) {
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      float4 o = make_float4(__uint_as_float(acc[4 * q]), __uint_as_float(acc[4 * q + 1]),
-                             __uint_as_float(acc[4 * q + 2]), __uint_as_float(acc[4 * q + 3]));
-      if (P.kind == EPI_ACCUM) {
+    for (int q = 0; q < COLS_PER_THREAD / 4; ++q) {
+      float4 o = make_float4(sums[4 * q] * sc, sums[4 * q + 1] * sc, sums[4 * q + 2] * sc, sums[4 * q + 3] * sc);
+      if (EPI == EPI_ACCUM) {
         const float4 c = *reinterpret_cast<const float4*>(crow + 4 * q);
         o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
-      } else if (P.kind == EPI_WOUT) {
+      } else if (EPI == EPI_WOUT) {
         const float4 c = *reinterpret_cast<const float4*>(P.Whs + (long long)row * N + col0 + 4 * q);
         o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
       }
@@ -196,22 +231,26 @@ __device__ __forceinline__ void epi_chunk32(const EpiParams& P, int row, int col
     }
     return;
   }
-  for (int e = 0; e < 32; ++e)
-    if (col0 + e < N) epi_scalar(P, row, col0 + e, N, __uint_as_float(acc[e]), r2, s2);
+#pragma unroll
+  for (int e = 0; e < COLS_PER_THREAD; ++e)
+    if (col0 + e < N) epi_scalar(P, row, col0 + e, N, sums[e], r2, s2);
 }
 
 // ------------------------------------------------------------------ the kernel
-template <int NA, int NB>
+// NP: planes per operand (1 or 2).  EPI: epilogue kind (compile-time copy of epi.kind).
+template <int NP, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, EpiParams epi, int* status) {
+gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_t idesc, EpiParams epi,
+               int* status) {
   constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
-  constexpr int STAGE_BYTES = NA * A_BYTES + NB * B_BYTES;
-  constexpr int STAGES = (NA + NB == 2) ? 4 : 2;
+  constexpr int STAGE_BYTES = NP * (A_BYTES + B_BYTES);
+  constexpr int STAGES = (NP == 1) ? 6 : 3;
+  constexpr int KB_PER_FLUSH = (NP == 1) ? 3 : 1;        // 12 accumulating MMA steps per flush either way
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 2 * NPART + 2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
-  __shared__ float red[8];
+  __shared__ float red[2 * GROUP_WARPS * 2];
 
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -219,8 +258,9 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, EpiPara
 
   const uint32_t full0 = smem_u32(&bars[0]);
   const uint32_t empty0 = smem_u32(&bars[STAGES]);
-  const uint32_t tfull0 = smem_u32(&bars[2 * STAGES]);
-  const uint32_t tempty0 = smem_u32(&bars[2 * STAGES + 2]);
+  const uint32_t pfull0 = smem_u32(&bars[2 * STAGES]);
+  const uint32_t pempty0 = smem_u32(&bars[2 * STAGES + NPART]);
+  const uint32_t drained0 = smem_u32(&bars[2 * STAGES + 2 * NPART]);   // [group]: that group has drained a tile
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
@@ -228,10 +268,11 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, EpiPara
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
     }
-    for (int a = 0; a < 2; ++a) {
-      mbar_init(tfull0 + 8 * a, 1);
-      mbar_init(tempty0 + 8 * a, 4);
+    for (int a = 0; a < NPART; ++a) {
+      mbar_init(pfull0 + 8 * a, 1);
+      mbar_init(pempty0 + 8 * a, GROUP_WARPS);
     }
+    for (int a = 0; a < 2; ++a) mbar_init(drained0 + 8 * a, GROUP_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -248,7 +289,8 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, EpiPara
   const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
   const int num_tiles = tiles_m * tiles_n;
   const int num_kb = (K + BK - 1) / BK;
-  const bool lower = (epi.kind == EPI_ACCUM) && epi.lower_only;
+  const int num_flush = (num_kb + KB_PER_FLUSH - 1) / KB_PER_FLUSH;
+  const bool lower = (EPI == EPI_ACCUM) && epi.lower_only;
 
   if (warp == 0) {
     // ===================== TMA producer =====================
@@ -266,10 +308,10 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, EpiPara
           const uint32_t fb = full0 + 8 * stage;
           mbar_expect_tx(fb, STAGE_BYTES);
 #pragma unroll
-          for (int pl = 0; pl < NA; ++pl) tma_load_2d(sbase + pl * A_BYTES, &maps.a[pl], fb, kb * BK, tm * BM);
+          for (int pl = 0; pl < NP; ++pl) tma_load_2d(sbase + pl * A_BYTES, &maps.a[pl], fb, kb * BK, tm * BM);
 #pragma unroll
-          for (int pl = 0; pl < NB; ++pl)
-            tma_load_2d(sbase + NA * A_BYTES + pl * B_BYTES, &maps.b[pl], fb, kb * BK, tn * BN);
+          for (int pl = 0; pl < NP; ++pl)
+            tma_load_2d(sbase + NP * A_BYTES + pl * B_BYTES, &maps.b[pl], fb, kb * BK, tn * BN);
           if (++stage == STAGES) {
             stage = 0;
             phase ^= 1u;
@@ -282,77 +324,114 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, EpiPara
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      int it = 0;
+      uint32_t g = 0;                        // flush counter, shared sequence with the workers
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         const int tm = tile / tiles_n, tn = tile % tiles_n;
         if (lower && tn * BN > tm * BM + BM - 1) continue;
-        const int acc = it & 1;
-        ok = mbar_wait(tempty0 + 8 * acc, (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag, status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
-        uint32_t accumulate = 0;
+        uint32_t d_tmem = 0, accumulate = 0;
+        int pb = 0;
         for (int kb = 0; kb < num_kb; ++kb) {
+          if (kb % KB_PER_FLUSH == 0) {
+            pb = (int)(g % NPART);
+            ok = mbar_wait(pempty0 + 8 * pb, ((g / NPART) & 1u) ^ 1u, abort_flag, status);
+            if (!ok) break;
+            tc_fence_after();
+            d_tmem = tmem_base + (uint32_t)pb * BN;
+            accumulate = 0;
+          }
           ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, status);
           if (!ok) break;
           tc_fence_after();
           const uint32_t sbase = tiles_base + stage * STAGE_BYTES;
           const uint64_t a_hi = make_kmajor_sw128_desc(sbase);
           const uint64_t a_lo = make_kmajor_sw128_desc(sbase + A_BYTES);
-          const uint64_t b_hi = make_kmajor_sw128_desc(sbase + NA * A_BYTES);
-          const uint64_t b_lo = make_kmajor_sw128_desc(sbase + NA * A_BYTES + B_BYTES);
+          const uint64_t b_hi = make_kmajor_sw128_desc(sbase + NP * A_BYTES);
+          const uint64_t b_lo = make_kmajor_sw128_desc(sbase + NP * A_BYTES + B_BYTES);
 #pragma unroll
           for (int k16 = 0; k16 < BK / 16; ++k16) {
-            const uint64_t koff = (uint64_t)((k16 * 32) >> 4);   // 16 bf16 = 32 bytes along K
-            tc_mma_bf16(d_tmem, a_hi + koff, b_hi + koff, IDESC_BF16_128x256, accumulate);
+            const uint64_t koff = (uint64_t)((k16 * 32) >> 4);   // 16 elements = 32 bytes along K
+            // small terms first, so that they meet a small accumulator
+            if (NP == 2) {
+              tc_mma_f16(d_tmem, a_hi + koff, b_lo + koff, idesc, accumulate);
+              tc_mma_f16(d_tmem, a_lo + koff, b_hi + koff, idesc, 1);
+              accumulate = 1;
+            }
+            tc_mma_f16(d_tmem, a_hi + koff, b_hi + koff, idesc, accumulate);
             accumulate = 1;
-            if (NB == 2) tc_mma_bf16(d_tmem, a_hi + koff, b_lo + koff, IDESC_BF16_128x256, 1);
-            if (NA == 2) tc_mma_bf16(d_tmem, a_lo + koff, b_hi + koff, IDESC_BF16_128x256, 1);
           }
           tc_commit(empty0 + 8 * stage);     // stage reusable once these MMAs have read it
           if (++stage == STAGES) {
             stage = 0;
             phase ^= 1u;
           }
+          if (kb % KB_PER_FLUSH == KB_PER_FLUSH - 1 || kb == num_kb - 1) {
+            tc_commit(pfull0 + 8 * pb);      // partial complete
+            ++g;
+          }
         }
-        if (!ok) break;
-        tc_commit(tfull0 + 8 * acc);         // accumulator complete
-        ++it;
       }
     }
   } else {
-    // ===================== epilogue warps =====================
-    const int q = warp & 3;                  // tensor-memory lane quarter this warp may read
+    // ===================== worker groups =====================
+    const int gsel = (warp - 2) / GROUP_WARPS;             // 0 or 1
+    const int wi = (warp - 2) % GROUP_WARPS;
+    const int q = warp & 3;                                // tensor-memory lane quarter this warp may read
+    const int half = wi >> 2;                              // which 64 of the 128 columns
     float r2 = 0.f, s2 = 0.f;
+    uint32_t g = 0;
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
       const int tm = tile / tiles_n, tn = tile % tiles_n;
       if (lower && tn * BN > tm * BM + BM - 1) continue;
-      const int acc = it & 1;
-      ok = mbar_wait(tfull0 + 8 * acc, ((uint32_t)it >> 1) & 1u, abort_flag, status);
-      if (!ok) break;
-      tc_fence_after();
-      const int row = tm * BM + q * 32 + lane;
-      const uint32_t taddr = tmem_base + (uint32_t)acc * BN + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
-      for (int cchunk = 0; cchunk < BN / 32; ++cchunk) {
-        uint32_t v[32];
-        tc_ld32(taddr + cchunk * 32, v);
-        epi_chunk32(epi, row, tn * BN + cchunk * 32, M, N, v, r2, s2);
+      if ((it & 1) != gsel) {                              // the other group's tile
+        g += (uint32_t)num_flush;
+        ++it;
+        continue;
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+      // A parity wait cannot tell a phase from the one two completions later, so a group starts
+      // watching the partial barriers only once the other group has drained the tile before this one.
+      if (it > 0) {
+        ok = mbar_wait(drained0 + 8 * (1 - gsel), (uint32_t)((it - 1) >> 1) & 1u, abort_flag, status);
+        if (!ok) break;
+      }
+      float sums[COLS_PER_THREAD];
+#pragma unroll
+      for (int e = 0; e < COLS_PER_THREAD; ++e) sums[e] = 0.f;
+      for (int f = 0; f < num_flush; ++f) {
+        const int pb = (int)(g % NPART);
+        ok = mbar_wait(pfull0 + 8 * pb, (g / NPART) & 1u, abort_flag, status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + (uint32_t)pb * BN + (uint32_t)(half * COLS_PER_THREAD) +
+                               ((uint32_t)(q * 32) << 16);
+        uint32_t v[32];
+        tc_ld32_issue(taddr, v);
+        tc_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) sums[e] += __uint_as_float(v[e]);
+        tc_ld32_issue(taddr + 32, v);
+        tc_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pempty0 + 8 * pb);      // the partial is in registers: buffer free
+#pragma unroll
+        for (int e = 0; e < 32; ++e) sums[32 + e] += __uint_as_float(v[e]);
+        ++g;
+      }
+      if (!ok) break;
+      if (lane == 0) mbar_arrive(drained0 + 8 * gsel);
+      const int row = tm * BM + q * 32 + lane;
+      epilogue_row64<EPI>(epi, row, tn * BN + half * COLS_PER_THREAD, M, N, sums, r2, s2);
       ++it;
     }
-    if (epi.kind == EPI_ADMM) {
+    if (EPI == EPI_ADMM) {
       r2 = warp_sum(r2);
       s2 = warp_sum(s2);
       if (lane == 0) {
-        red[2 * q] = r2;
-        red[2 * q + 1] = s2;
+        red[2 * (warp - 2)] = r2;
+        red[2 * (warp - 2) + 1] = s2;
       }
     }
   }
@@ -364,10 +443,14 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, EpiPara
     }
     __syncthreads();
   }
-  if (epi.kind == EPI_ADMM && threadIdx.x == 0) {
-    // fixed order over the four lane quarters (warps 2,3,4,5 hold quarters 2,3,0,1)
-    epi.partials[2 * blockIdx.x + 0] = ((red[0] + red[2]) + red[4]) + red[6];
-    epi.partials[2 * blockIdx.x + 1] = ((red[1] + red[3]) + red[5]) + red[7];
+  if (EPI == EPI_ADMM && threadIdx.x == 0) {
+    float a = 0.f, b = 0.f;                  // fixed order over the worker warps
+    for (int w = 0; w < 2 * GROUP_WARPS; ++w) {
+      a += red[2 * w];
+      b += red[2 * w + 1];
+    }
+    epi.partials[2 * blockIdx.x + 0] = a;
+    epi.partials[2 * blockIdx.x + 1] = b;
   }
   if (warp == 1) {
     tc_fence_after();
@@ -393,56 +476,73 @@ static EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// Row-major bf16 matrix [rows][ld], K = `cols` contiguous; box = box_rows x 64 elements, 128B swizzle;
+// Row-major 16-bit matrix [rows][ld], K = `cols` contiguous; box = box_rows x 64 elements, 128B swizzle;
 // out-of-range elements read as zero.
 static bool encode_plane(CUtensorMap* map, const bf16* ptr, long long rows, long long cols, long long ld,
-                         int box_rows) {
+                         int box_rows, int f16) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(bf16)};
   cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr, dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = fn(map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr,
+                  dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
 int gemm_tc_partial_slots(int num_sms) { return num_sms; }
 
-template <int NA, int NB>
-static cudaError_t launch_tc(Ctx* c, const TcMaps& maps, int M, int N, int K, const EpiParams& epi) {
-  constexpr int STAGE_BYTES = NA * BM * BK * 2 + NB * BN * BK * 2;
-  constexpr int STAGES = (NA + NB == 2) ? 4 : 2;
+template <int NP, int EPI>
+static cudaError_t launch_tc(Ctx* c, const TcMaps& maps, int M, int N, int K, uint32_t idesc,
+                             const EpiParams& epi) {
+  constexpr int STAGE_BYTES = NP * (BM * BK * 2 + BN * BK * 2);
+  constexpr int STAGES = (NP == 1) ? 6 : 3;
   const size_t smem = (size_t)STAGES * STAGE_BYTES + 1024;
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<NA, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem);
-  if (e != cudaSuccess) return e;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<NP, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
   const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = tiles < c->num_sms ? tiles : c->num_sms;
-  gemm_tc_kernel<NA, NB><<<grid, TC_THREADS, smem, c->stream>>>(maps, M, N, K, epi, c->status);
+  gemm_tc_kernel<NP, EPI><<<grid, TC_THREADS, smem, c->stream>>>(maps, M, N, K, idesc, epi, c->status);
   c->launches++;
   return cudaGetLastError();
 }
 
-cudaError_t gemm_tc(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiParams& epi) {
+cudaError_t gemm_tc(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiParams& epi_in) {
   const int na = A.lo ? 2 : 1, nb = B.lo ? 2 : 1;
-  if (na != nb) return cudaErrorInvalidValue;
+  if (na != nb || A.f16 != B.f16) return cudaErrorInvalidValue;   // one MMA takes A and B of one type
   if ((A.ld & 7) || (B.ld & 7)) return cudaErrorInvalidValue;
   TcMaps maps;
-  bool ok = encode_plane(&maps.a[0], A.hi, M, K, A.ld, BM) && encode_plane(&maps.b[0], B.hi, N, K, B.ld, BN);
-  if (na == 2) ok = ok && encode_plane(&maps.a[1], A.lo, M, K, A.ld, BM);
+  bool ok = encode_plane(&maps.a[0], A.hi, M, K, A.ld, BM, A.f16) &&
+            encode_plane(&maps.b[0], B.hi, N, K, B.ld, BN, B.f16);
+  if (na == 2) ok = ok && encode_plane(&maps.a[1], A.lo, M, K, A.ld, BM, A.f16);
   else maps.a[1] = maps.a[0];
-  if (nb == 2) ok = ok && encode_plane(&maps.b[1], B.lo, N, K, B.ld, BN);
+  if (nb == 2) ok = ok && encode_plane(&maps.b[1], B.lo, N, K, B.ld, BN, B.f16);
   else maps.b[1] = maps.b[0];
   if (!ok) return cudaErrorInvalidValue;
-  if (epi.kind == EPI_ADMM) {
-    // unused partial slots of this launch must read as zero
-    const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-    (void)tiles;
+  EpiParams epi = epi_in;
+  epi.row_inv = A.row_inv;
+  epi.a_inv = A.all_inv;
+  epi.b_inv = B.all_inv;
+  const uint32_t idesc = idesc_128x128(A.f16 ? 0u : 1u);
+  if (na == 1) {
+    if (epi.kind == EPI_ACCUM) return launch_tc<1, EPI_ACCUM>(c, maps, M, N, K, idesc, epi);
+    if (epi.kind == EPI_STORE) return launch_tc<1, EPI_STORE>(c, maps, M, N, K, idesc, epi);
+    return cudaErrorInvalidValue;
   }
-  return (na == 2) ? launch_tc<2, 2>(c, maps, M, N, K, epi) : launch_tc<1, 1>(c, maps, M, N, K, epi);
+  switch (epi.kind) {
+    case EPI_STORE: return launch_tc<2, EPI_STORE>(c, maps, M, N, K, idesc, epi);
+    case EPI_ACCUM: return launch_tc<2, EPI_ACCUM>(c, maps, M, N, K, idesc, epi);
+    case EPI_ADMM: return launch_tc<2, EPI_ADMM>(c, maps, M, N, K, idesc, epi);
+    case EPI_WOUT: return launch_tc<2, EPI_WOUT>(c, maps, M, N, K, idesc, epi);
+  }
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace admmq

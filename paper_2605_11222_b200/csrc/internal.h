@@ -14,10 +14,17 @@ typedef __nv_bfloat16 bf16;
 // One operand of a product C = A * B^T: up to two bf16 planes (hi, lo) whose sum is the value.
 // Row-major [rows][ld], the contraction index contiguous ("K-major").
 struct Planes {
-  const bf16* hi;
-  const bf16* lo;   // nullptr: single plane
+  const bf16* hi;           // 16-bit storage: bf16 values, or fp16 values when f16 != 0
+  const bf16* lo;           // nullptr: single plane
   long long ld;
+  int f16;                  // 1: planes hold fp16 values that were scaled by a power of two first
+  const float* row_inv;     // [rows] inverse of each row's scale (device), or nullptr
+  const float* all_inv;     // inverse of a scale common to all elements (device scalar), or nullptr
 };
+inline Planes planes_bf16(const bf16* hi, const bf16* lo, long long ld) { return Planes{hi, lo, ld, 0, nullptr, nullptr}; }
+inline Planes planes_f16(const bf16* hi, const bf16* lo, long long ld, const float* row_inv, const float* all_inv) {
+  return Planes{hi, lo, ld, 1, row_inv, all_inv};
+}
 
 struct Ctx {
   int n = 0, p_max = 0, T_max = 0;
@@ -44,8 +51,9 @@ struct Ctx {
   double* te = nullptr;         // [n] tridiagonal off-diagonal
   double* beta = nullptr;       // [n] reflector scalars
   double* pvec = nullptr;       // [n] matrix-vector scratch of the reduction
-  double* stage_l = nullptr;    // [T_max+1][n] LDL^T multipliers per penalty
-  double* stage_invd = nullptr; // [T_max+1][n] LDL^T inverse pivots per penalty
+  float* stage_l = nullptr;     // [T_max+1][stage_factor_stride(n)] LDL^T multipliers per penalty
+  float* stage_invd = nullptr;  // [T_max+1][stage_factor_stride(n)] LDL^T inverse pivots per penalty
+  double* wy_s = nullptr;       // [ceil(n/32)][32][32] triangular factors of the reflector blocks
   bf16 *Q_hi = nullptr, *Q_lo = nullptr;    // [n][n] Q   (row i, col m)
   bf16 *QT_hi = nullptr, *QT_lo = nullptr;  // [n][n] Q^T (row m, col k)
   bf16 *H_hi = nullptr, *H_lo = nullptr;    // [n][n] split planes of the damped unscaled H
@@ -57,6 +65,9 @@ struct Ctx {
   float* partials = nullptr;    // [T_max][slots][2]
   int partial_slots = 0;
   double* scal = nullptr;       // small fp64 scalars (objective, counters)
+  float* fscal = nullptr;       // [0] 1 / scale of the Q planes, [1] 1 / scale of the H planes, [2] scale of the H planes
+  float* rs_R = nullptr;        // [p] inverse row scales of the R (and E) planes
+  float* rs_Y = nullptr;        // [p] inverse row scales of the Y' planes
   bf16 *XT_hi = nullptr, *XT_lo = nullptr;  // [n][XT_ROWS] transposed chunk of X
   void* tmaps = nullptr;        // reserved
 };
@@ -71,15 +82,17 @@ void launch_finalize(Ctx* c, double damp_frac, int precondition);
 void launch_grid_fit(Ctx* c, const float* W0, int p, int bits, int gs, int symmetric, float* delta,
                      float* zero);
 void launch_scale_weights(Ctx* c, const float* W0, int p);
+void launch_operand_scales(Ctx* c);   // fscal from diag(H)
 void launch_split_f64(Ctx* c, const double* src, int n, bf16* hi, bf16* lo, bf16* thi, bf16* tlo);
 void launch_split_f32(Ctx* c, const float* src, long long count, bf16* hi, bf16* lo);
+void launch_row_split(Ctx* c, const float* src, int p, bf16* hi, bf16* lo, float* row_inv);
 void launch_init_rhs(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
-                     const float* zero, const float* V_in, float inv_rho);
+                     const float* zero, const float* V_in, float inv_rho, float* R_out);
 void launch_reduce_partials(Ctx* c, int T, float* resid);
 void launch_dequant(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
                     const float* zero, float* Wq);
 void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes,
-                         const float* delta, const float* zero, bf16* Ehi, bf16* Elo);
+                         const float* delta, const float* zero, bf16* Ehi, bf16* Elo, float* row_inv);
 void launch_objective_dot(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes,
                           const float* delta, const float* zero, const float* g, double* out);
 
@@ -91,6 +104,7 @@ int gemm_tc_partial_slots(int num_sms);
 // ---- tridiag.cu ----
 cudaError_t tridiag_reduce(Ctx* c);                 // A64 -> td, te, reflectors, beta
 cudaError_t tridiag_form_qt(Ctx* c);                // reflectors -> P64 = Q^T
+size_t stage_factor_stride(int n);                  // floats per penalty in stage_l / stage_invd
 void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count);
 void launch_tridiag_solve(Ctx* c, int p, int stage);
 

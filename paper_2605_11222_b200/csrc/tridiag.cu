@@ -3,7 +3,7 @@
 // The paper diagonalises H~ once so that (H~ + rho I)^{-1} is available for every rho.  Here the
 // orthogonal reduction stops at tridiagonal form, H~ = Q T Q^T (Householder), which serves the same
 // purpose: (H~ + rho I)^{-1} = Q (T + rho I)^{-1} Q^T, and T + rho I is solved in O(n) per column by an
-// LDL^T factorisation computed once per penalty value.  The reduction runs in fp64 so that the
+// LDL^T factorisation computed once per penalty value.  The reduction and Q run in fp64 so that the
 // operator is accurate far below the split-bf16 product error.
 #include <cooperative_groups.h>
 
@@ -15,187 +15,520 @@ namespace admmq {
 
 // ------------------------------------------------------------------------------------------------
 // Householder tridiagonalisation of the symmetric matrix A (full storage, fp64), cooperative launch.
-// Step k: x = A[k, k+1:], reflector H_k = I - beta u u^T with u = x - alpha e_1, trailing update
-// A22 <- A22 - u w^T - w u^T, w = p - (beta u^T p / 2) u, p = beta A22 u.  Row r is always handled by
-// the same warp (r mod #warps), so a warp re-reads only rows it wrote itself; row k and p cross CTAs
-// and are read with cache-global loads after a grid-wide barrier.
+//
+// Step k uses the reflector H_k = I - beta u u^T built from row k (u = x - alpha e_1, x = A[k, k+1:])
+// and updates the trailing matrix A22 <- A22 - u w^T - w u^T with w = p - (beta u^T p / 2) u,
+// p = beta A22 u.  The matrix is read and written ONCE per step: the pass of step k applies the
+// rank-2 update of step k-1 to every element and, in the same sweep, accumulates that element's
+// contribution to p of step k.  This is possible because the next reflector needs only one row of
+// the updated matrix, which every CTA rebuilds for itself from the stored row and the two update
+// vectors.  One grid-wide barrier per step (for p).
+//
+// Rows are dealt cyclically to row groups of CTAs, so the load stays balanced as the trailing matrix
+// shrinks; a row group has C CTAs, each sweeping one chunk of the columns (C = 1 up to n = 9216,
+// where the three length-n vectors fit in shared memory; above that each CTA keeps the full vectors
+// in a private global scratch and only its column chunk in shared memory).
 // Output: td/te (diagonal / off-diagonal of T), reflector k in A[k, k+1:], beta[k].
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024, 1)
-tridiag_reduce_kernel(double* __restrict__ A, int n, double* __restrict__ td, double* __restrict__ te,
-                      double* __restrict__ beta, double* __restrict__ pvec) {
+constexpr int TRD_THREADS = 1024;
+constexpr int TRD_PSUM = 512;
+
+struct TrdArgs {
+  double* A;
+  int n;
+  double* td;
+  double* te;
+  double* beta;
+  double* pbuf;   // [2][C][n]: per-chunk row sums of A22 u, double-buffered by the parity of the step
+  double* priv;   // [grid][3][n]: full-length vectors of each CTA (C > 1 only)
+  int C;          // column chunks per row group
+  int cap;        // doubles per shared-memory vector
+};
+
+__global__ void __launch_bounds__(TRD_THREADS, 1) tridiag_reduce_kernel(TrdArgs a) {
   cg::grid_group grid = cg::this_grid();
   extern __shared__ double sm[];
-  double* u = sm;
-  double* w = sm + n;
   __shared__ double scratch[32];
-  const int lane = threadIdx.x & 31;
-  const int wpb = blockDim.x >> 5;
-  const int gw = blockIdx.x * wpb + (threadIdx.x >> 5);
-  const int GW = gridDim.x * wpb;
+  __shared__ double psum[TRD_PSUM];
+  const int n = a.n, C = a.C;
+  const int Gr = gridDim.x / C, g = blockIdx.x / C, h = blockIdx.x % C;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const bool alias = (C == 1);
+  // shared copies (column chunk) and full-length versions of: pending u, pending w, current reflector
+  double *Sup = sm, *Swp = sm + a.cap, *Suc = sm + 2 * (size_t)a.cap;
+  double *Fup = Sup, *Fwp = Swp, *Fuc = Suc;
+  if (!alias) {
+    double* base = a.priv + (size_t)blockIdx.x * 3 * n;
+    Fup = base;
+    Fwp = base + n;
+    Fuc = base + 2 * (size_t)n;
+  }
+  for (int i = tid; i < n; i += TRD_THREADS) {
+    Fup[i] = 0.0;
+    Fwp[i] = 0.0;
+    Fuc[i] = 0.0;
+  }
+  __syncthreads();
+  double beta_k = 0.0, alpha_k = 0.0;   // belong to the current reflector u_k (in Fuc)
 
-  for (int k = 0; k < n - 2; ++k) {
-    const int m = n - k - 1;
+  for (int k = -1; k <= n - 2; ++k) {
     const int c0 = k + 1;
-    const double* rowk = A + (long long)k * n + c0;
-    // ---- reflector (identical in every CTA) ----
+    if (k >= 0) {
+      // ================= fused pass over rows / columns >= k+1 =================
+      const int m = n - c0;
+      int cb = c0, ce = n;
+      if (!alias) {
+        const int per = (((m + C - 1) / C) + 1) & ~1;
+        cb = c0 + h * per;
+        if (cb > n) cb = n;
+        ce = cb + per < n ? cb + per : n;
+      }
+      const int base = alias ? 0 : (cb & ~1);
+      if (!alias) {
+        const int iend = (ce + 1) & ~1;
+        for (int i = base + tid; i < iend; i += TRD_THREADS) {
+          Sup[i - base] = Fup[i];
+          Swp[i - base] = Fwp[i];
+          Suc[i - base] = Fuc[i];
+        }
+        __syncthreads();
+      }
+      const int r_first = c0 + (((g - c0) % Gr) + Gr) % Gr;
+      const int nr = (r_first < n) ? (n - r_first + Gr - 1) / Gr : 0;
+      const int i_lo = cb & ~1;
+      const int width = ce > i_lo ? ce - i_lo : 0;
+      const int nseg = (width + 255) >> 8;
+      int Sf = 1;                                   // parts a row is split into, so that every warp has work
+      while (nr * Sf < 32 && Sf < nseg) Sf <<= 1;
+      const int sp = (nseg + Sf - 1) / Sf;
+      const int items = nr * Sf;
+      for (int it = warp; it < items; it += 32) {
+        const int rl = it / Sf, part = it - rl * Sf;
+        const int r = r_first + rl * Gr;
+        const double ur = Fup[r], wr = Fwp[r];
+        double* arow = a.A + (size_t)r * n;
+        double acc = 0.0;
+        const int s_end = (part + 1) * sp < nseg ? (part + 1) * sp : nseg;
+        for (int sg = part * sp; sg < s_end; ++sg) {
+          const int i0 = i_lo + (sg << 8) + lane * 2;
+          double2 av[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int i = i0 + q * 64;
+            av[q] = make_double2(0.0, 0.0);
+            if (i < ce) av[q] = __ldcg(reinterpret_cast<const double2*>(arow + i));
+          }
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int i = i0 + q * 64;
+            if (i < ce) {
+              const double2 up2 = *reinterpret_cast<const double2*>(Sup + (i - base));
+              const double2 wp2 = *reinterpret_cast<const double2*>(Swp + (i - base));
+              const double2 uc2 = *reinterpret_cast<const double2*>(Suc + (i - base));
+              const double x = av[q].x - (ur * wp2.x + wr * up2.x);
+              const double y = av[q].y - (ur * wp2.y + wr * up2.y);
+              const bool vx = (i >= cb), vy = (i + 1 < ce);
+              if (vx && vy) {
+                __stcg(reinterpret_cast<double2*>(arow + i), make_double2(x, y));
+                acc += x * uc2.x + y * uc2.y;
+              } else if (vx) {
+                arow[i] = x;
+                acc += x * uc2.x;
+              } else if (vy) {
+                arow[i + 1] = y;
+                acc += y * uc2.y;
+              }
+            }
+          }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) psum[it] = acc;
+      }
+      __syncthreads();
+      double* pb = a.pbuf + ((size_t)(k & 1) * C + h) * n;
+      for (int t = tid; t < nr; t += TRD_THREADS) {
+        double s = 0.0;
+        for (int q = 0; q < Sf; ++q) s += psum[t * Sf + q];
+        pb[r_first + t * Gr] = s;
+      }
+      grid.sync();
+    }
+    // ================= vector phase (identical in every CTA) =================
+    // w_k = p - (beta u^T p / 2) u,  p = beta A22 u
+    double up = 0.0;
+    if (k >= 0) {
+      const double* pb = a.pbuf + (size_t)(k & 1) * C * n;
+      for (int i = c0 + tid; i < n; i += TRD_THREADS) {
+        double p = 0.0;
+        for (int hh = 0; hh < C; ++hh) p += __ldcg(pb + (size_t)hh * n + i);
+        p *= beta_k;
+        Fwp[i] = p;                      // w_{k-1} is dead: this CTA's pass has used it
+        up += p * Fuc[i];
+      }
+    }
+    up = block_sum(up, scratch);
+    const double kc = 0.5 * beta_k * up;
+    if (k >= 0)
+      for (int i = c0 + tid; i < n; i += TRD_THREADS) Fwp[i] -= kc * Fuc[i];
+    __syncthreads();
+    // row k+1 of the matrix after update k, rebuilt locally: source of the next reflector and of td[k+1]
+    const int r1 = k + 1;
+    const double u1 = Fuc[r1], w1 = Fwp[r1];
+    const double* row = a.A + (size_t)r1 * n;
     double tail = 0.0;
-    for (int i = threadIdx.x; i < m; i += blockDim.x) {
-      const double x = __ldcg(rowk + i);
-      u[i] = x;
-      if (i > 0) tail += x * x;
+    for (int i = r1 + 1 + tid; i < n; i += TRD_THREADS) {
+      const double x = __ldcg(row + i) - u1 * Fwp[i] - w1 * Fuc[i];
+      Fup[i] = x;                        // u_{k-1} is dead
+      if (i > r1 + 1) tail += x * x;
     }
     tail = block_sum(tail, scratch);
     __syncthreads();
-    const double x0 = u[0];
+    const double x0 = (r1 + 1 < n) ? Fup[r1 + 1] : 0.0;
     double alpha = x0, bt = 0.0;
     if (tail > 0.0) {
       const double nrm = sqrt(x0 * x0 + tail);
       alpha = (x0 >= 0.0) ? -nrm : nrm;
       bt = 1.0 / (nrm * nrm - x0 * alpha);          // 2 / (u^T u)
     }
+    const double diag = __ldcg(row + r1) - 2.0 * u1 * w1;
     __syncthreads();
-    if (threadIdx.x == 0) u[0] = x0 - alpha;
-    __syncthreads();
-    // ---- p = beta * A22 u over the rows this warp owns ----
-    int r = c0 + (((gw - c0) % GW) + GW) % GW;
-    for (; r < n; r += GW) {
-      const double* row = A + (long long)r * n + c0;
-      double acc = 0.0;
-      for (int i = lane; i < m; i += 32) acc += row[i] * u[i];
-      acc = warp_sum(acc);
-      if (lane == 0) pvec[r - c0] = bt * acc;
-    }
-    grid.sync();
-    // ---- w = p - (beta u^T p / 2) u ----
-    double up = 0.0;
-    for (int i = threadIdx.x; i < m; i += blockDim.x) {
-      const double pi = __ldcg(pvec + i);
-      w[i] = pi;
-      up += pi * u[i];
-    }
-    up = block_sum(up, scratch);
-    const double kc = 0.5 * bt * up;
-    __syncthreads();
-    for (int i = threadIdx.x; i < m; i += blockDim.x) w[i] -= kc * u[i];
-    __syncthreads();
-    // ---- rank-2 update of the rows this warp owns ----
-    r = c0 + (((gw - c0) % GW) + GW) % GW;
-    for (; r < n; r += GW) {
-      double* row = A + (long long)r * n + c0;
-      const double ur = u[r - c0], wr = w[r - c0];
-      for (int i = lane; i < m; i += 32) row[i] -= ur * w[i] + wr * u[i];
+    if (tid == 0) {
+      if (r1 + 1 < n) Fup[r1 + 1] = x0 - alpha;
+      Fup[r1] = 0.0;
     }
     if (blockIdx.x == 0) {
-      double* rk = A + (long long)k * n + c0;
-      for (int i = threadIdx.x; i < m; i += blockDim.x) rk[i] = u[i];
-      if (threadIdx.x == 0) {
-        td[k] = __ldcg(A + (long long)k * n + k);
-        te[k] = alpha;
-        beta[k] = bt;
+      if (k >= 0) {
+        double* rk = a.A + (size_t)k * n;
+        for (int i = c0 + tid; i < n; i += TRD_THREADS) rk[i] = Fuc[i];
+        if (tid == 0) {
+          a.te[k] = alpha_k;
+          a.beta[k] = beta_k;
+        }
       }
+      if (tid == 0) a.td[r1] = diag;
     }
-    grid.sync();
-  }
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    if (n >= 2) {
-      td[n - 2] = __ldcg(A + (long long)(n - 2) * n + (n - 2));
-      te[n - 2] = __ldcg(A + (long long)(n - 2) * n + (n - 1));
-      beta[n - 2] = 0.0;
+    // (u_k, w_k) become the pending update, the new reflector becomes current
+    double* t = Fup;
+    Fup = Fuc;
+    Fuc = t;
+    if (alias) {
+      Sup = Fup;
+      Suc = Fuc;
     }
-    td[n - 1] = __ldcg(A + (long long)(n - 1) * n + (n - 1));
-    te[n - 1] = 0.0;
-    beta[n - 1] = 0.0;
+    alpha_k = alpha;
+    beta_k = bt;
+    __syncthreads();
   }
+  if (blockIdx.x == 0 && tid == 0) {
+    a.te[n - 1] = 0.0;
+    a.beta[n - 1] = 0.0;
+  }
+}
+
+static int trd_cap(int n, int C) {
+  if (C == 1) return n;
+  return ((((n - 1 + C - 1) / C) + 1) & ~1) + 4;
 }
 
 cudaError_t tridiag_reduce(Ctx* c) {
   const int n = c->n;
-  const size_t smem = (size_t)2 * n * sizeof(double);
+  int C = 1;
+  while ((size_t)3 * 8 * trd_cap(n, C) > (size_t)216 * 1024 && C < 4) C *= 2;
+  int blocks = (c->num_sms / C) * C;   // one CTA per SM: co-residency is what the cooperative launch checks
+  if (blocks < C) return cudaErrorLaunchOutOfResources;
+  TrdArgs a;
+  a.A = c->A64;
+  a.n = n;
+  a.td = c->td;
+  a.te = c->te;
+  a.beta = c->beta;
+  a.C = C;
+  a.cap = trd_cap(n, C);
+  // scratch inside the (not yet written) Q^T buffer
+  a.pbuf = c->P64;
+  a.priv = c->P64 + (((size_t)2 * C * n + 31) & ~(size_t)31);
+  if (C > 1 && (size_t)2 * C * n + 32 + (size_t)blocks * 3 * n > (size_t)n * n) return cudaErrorInvalidValue;
+  const size_t smem = (size_t)3 * a.cap * sizeof(double);
   cudaError_t e = cudaFuncSetAttribute(tridiag_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
   int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tridiag_reduce_kernel, 1024, smem);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tridiag_reduce_kernel, TRD_THREADS, smem);
   if (e != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
-  int blocks = c->num_sms;   // one CTA per SM: co-residency is what the cooperative launch checks
-  double* A = c->A64;
-  int nn = n;
-  void* args[] = {&A, &nn, &c->td, &c->te, &c->beta, &c->pvec};
-  e = cudaLaunchCooperativeKernel((void*)tridiag_reduce_kernel, dim3(blocks), dim3(1024), args, smem,
+  void* args[] = {&a};
+  e = cudaLaunchCooperativeKernel((void*)tridiag_reduce_kernel, dim3(blocks), dim3(TRD_THREADS), args, smem,
                                   c->stream);
   c->launches++;
   return e;
 }
 
 // ------------------------------------------------------------------------------------------------
-// Q^T = H_{n-3} ... H_1 H_0 built row by row: P <- P H_k for k descending touches each row of P
-// independently, so one warp keeps one row in shared memory and applies every reflector to it.
+// Q^T = H_{n-3} ... H_1 H_0, accumulated in blocks of WY_NB reflectors in compact WY form:
+//   H_kb H_{kb+1} ... H_{kb+nb-1} = I - Y S Y^T,  Y = [u_kb ... u_{kb+nb-1}], S upper triangular,
+//   S_jj = beta_j,  S_{0:j,j} = -beta_j S_{0:j,0:j} (Y_{:,0:j}^T u_j).
+// Row r of P = Q^T starts as e_r^T and receives the blocks in descending order:
+//   X <- X (I - Y S^T Y^T) = X - ((X Y) S^T) Y^T   on the rows r > kb and columns > kb,
+// independently of every other row, so each CTA owns a cyclic set of rows and needs no grid barrier.
+// Both products run on the fp64 tensor-core MMA (m8n8k4).
 // ------------------------------------------------------------------------------------------------
-__global__ void form_qt_kernel(const double* __restrict__ A, const double* __restrict__ beta, int n,
-                               double* __restrict__ P, int rows_per_block) {
-  extern __shared__ double sm[];
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  const int r = n - 1 - (blockIdx.x * rows_per_block + wid);   // heavy rows first
-  if (wid >= rows_per_block || r < 0) return;
-  double* row = sm + (size_t)wid * n;
-  for (int i = lane; i < n; i += 32) row[i] = (i == r) ? 1.0 : 0.0;
-  __syncwarp();
-  for (int k = min(r - 1, n - 3); k >= 0; --k) {
-    const double bt = beta[k];
-    if (bt == 0.0) continue;
-    const int c0 = k + 1, m = n - c0;
-    const double* u = A + (long long)k * n + c0;
-    double acc = 0.0;
-    for (int i = lane; i < m; i += 32) acc += row[c0 + i] * u[i];
-    acc = bt * warp_sum(acc);
-    for (int i = lane; i < m; i += 32) row[c0 + i] -= acc * u[i];
-    __syncwarp();
+constexpr int WY_NB = 32;
+constexpr int QT_KC = 64;            // columns per staged chunk
+constexpr int QT_LD = QT_KC + 4;     // stride == 4 (mod 16) doubles: fragment loads hit every bank pair twice
+constexpr int QT_LDZ = WY_NB + 4;
+constexpr int QT_RS_MAX = 128;       // row slots per CTA
+constexpr int QT_THREADS = 1024;
+
+__device__ __forceinline__ void dmma_8x8x4(double& d0, double& d1, double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d0), "+d"(d1)
+               : "d"(a), "d"(b));
+}
+
+// S of every block: one CTA per block.
+__global__ void __launch_bounds__(1024)
+wy_factor_kernel(const double* __restrict__ A, const double* __restrict__ beta, int n,
+                 double* __restrict__ Sall) {
+  __shared__ double Ys[WY_NB][65];
+  __shared__ double Gs[WY_NB][WY_NB + 1];
+  __shared__ double Ss[WY_NB][WY_NB + 1];
+  const int b = blockIdx.x, kb = b * WY_NB;
+  const int nrefl = n - 2;                                 // reflectors k = 0 .. n-3
+  const int nbk = nrefl - kb < WY_NB ? nrefl - kb : WY_NB;
+  const int tid = threadIdx.x, j1 = tid >> 5, j2 = tid & 31;
+  double acc = 0.0;
+  for (int cs = kb + 1; cs < n; cs += 64) {
+    for (int idx = tid; idx < WY_NB * 64; idx += 1024) {
+      const int j = idx >> 6, cl = idx & 63, cc = cs + cl;
+      double v = 0.0;
+      if (j < nbk && cc < n && cc >= kb + j + 1) v = A[(size_t)(kb + j) * n + cc];
+      Ys[j][cl] = v;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int cl = 0; cl < 64; ++cl) acc += Ys[j1][cl] * Ys[j2][cl];
+    __syncthreads();
   }
-  double* out = P + (long long)r * n;
-  for (int i = lane; i < n; i += 32) out[i] = row[i];
+  Gs[j1][j2] = acc;
+  Ss[j1][j2] = 0.0;
+  __syncthreads();
+  if (tid < 32) {
+    const int i = tid;                                     // lane i builds row i of S
+    for (int j = 0; j < WY_NB; ++j) {
+      const double bj = (j < nbk) ? beta[kb + j] : 0.0;
+      if (i == j) Ss[i][j] = bj;
+      if (i < j) {
+        double s = 0.0;
+        for (int l = i; l < j; ++l) s += Ss[i][l] * Gs[l][j];
+        Ss[i][j] = -bj * s;
+      }
+    }
+  }
+  __syncthreads();
+  Sall[(size_t)b * WY_NB * WY_NB + tid] = Ss[j1][j2];
+}
+
+__global__ void set_identity_kernel(double* __restrict__ P, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) P[(size_t)i * n + i] = 1.0;
+}
+
+__global__ void __launch_bounds__(QT_THREADS, 1)
+form_qt_kernel(const double* __restrict__ A, const double* __restrict__ Sall, int n, int nblk,
+               double* __restrict__ P) {
+  extern __shared__ double smq[];
+  double* Ys = smq;                                        // [WY_NB][QT_LD]
+  double* Xs = Ys + WY_NB * QT_LD;                         // [QT_RS_MAX][QT_LD]
+  double* Zp = Xs + QT_RS_MAX * QT_LD;                     // [ks][RS][QT_LDZ], ks * RS <= 128
+  double* Z1 = Zp + QT_RS_MAX * QT_LDZ;                    // [RS][QT_LDZ]  (X Y), then -(X Y) S^T
+  double* Ss = Z1 + QT_RS_MAX * QT_LDZ;                    // [WY_NB][WY_NB + 1]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gid = lane >> 2, tig = lane & 3;
+  const int G = gridDim.x, c = blockIdx.x;
+  if (c >= n) return;
+  const int Rtot = (n - c + G - 1) / G;                    // rows c, c + G, c + 2G, ...
+  const int nrefl = n - 2;
+
+  for (int b = nblk - 1; b >= 0; --b) {
+    const int kb = b * WY_NB;
+    const int nbk = nrefl - kb < WY_NB ? nrefl - kb : WY_NB;
+    int t0 = (kb + 1 - c + G - 1) / G;                     // first own row with r >= kb + 1
+    if (kb + 1 - c <= 0) t0 = 0;
+    const int Ract = Rtot - t0;
+    if (Ract <= 0) continue;                               // uniform in the CTA
+    const int RS = (Ract + 7) & ~7;
+    const int nrt = RS >> 3;
+    int KS = 1;
+    while (KS < 4 && 2 * KS * RS <= QT_RS_MAX) KS <<= 1;
+    const int kspan = QT_KC / KS;
+    const int cbeg = ((kb + 1) / QT_KC) * QT_KC;
+
+    for (int idx = tid; idx < WY_NB * WY_NB; idx += QT_THREADS)
+      Ss[(idx >> 5) * (WY_NB + 1) + (idx & 31)] = Sall[(size_t)b * WY_NB * WY_NB + idx];
+
+    // ---------------- Z = X Y ----------------
+    const int units_z = nrt * 4 * KS;                      // (k split, row tile, column tile of 8)
+    double z00 = 0.0, z01 = 0.0, z10 = 0.0, z11 = 0.0;     // accumulators of units warp and warp + 32
+    for (int cs = cbeg; cs < n; cs += QT_KC) {
+      for (int idx = tid; idx < WY_NB * QT_KC; idx += QT_THREADS) {
+        const int j = idx >> 6, cl = idx & 63, cc = cs + cl;
+        double v = 0.0;
+        if (j < nbk && cc < n && cc >= kb + j + 1) v = A[(size_t)(kb + j) * n + cc];
+        Ys[j * QT_LD + cl] = v;
+      }
+      for (int idx = tid; idx < RS * QT_KC; idx += QT_THREADS) {
+        const int rl = idx >> 6, cl = idx & 63, cc = cs + cl;
+        double v = 0.0;
+        if (rl < Ract && cc < n) v = P[(size_t)(c + (size_t)(t0 + rl) * G) * n + cc];
+        Xs[rl * QT_LD + cl] = v;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int s = 0; s < 2; ++s) {
+        const int u = warp + 32 * s;
+        if (u < units_z) {
+          const int ks = u / (nrt * 4), rem = u - ks * nrt * 4;
+          const int rt = rem >> 2, jt = rem & 3;
+          const double* xa = Xs + (rt * 8 + gid) * QT_LD + ks * kspan + tig;
+          const double* yb = Ys + (jt * 8 + gid) * QT_LD + ks * kspan + tig;
+          double d0 = s ? z10 : z00, d1 = s ? z11 : z01;
+          for (int kk = 0; kk < kspan; kk += 4) dmma_8x8x4(d0, d1, xa[kk], yb[kk]);
+          if (s) {
+            z10 = d0;
+            z11 = d1;
+          } else {
+            z00 = d0;
+            z01 = d1;
+          }
+        }
+      }
+      __syncthreads();
+    }
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      const int u = warp + 32 * s;
+      if (u < units_z) {
+        const int ks = u / (nrt * 4), rem = u - ks * nrt * 4;
+        const int rt = rem >> 2, jt = rem & 3;
+        double* zp = Zp + (ks * RS + rt * 8 + gid) * QT_LDZ + jt * 8 + 2 * tig;
+        zp[0] = s ? z10 : z00;
+        zp[1] = s ? z11 : z01;
+      }
+    }
+    __syncthreads();
+    for (int idx = tid; idx < RS * WY_NB; idx += QT_THREADS) {
+      const int rl = idx >> 5, j = idx & 31;
+      double z = 0.0;
+      for (int ks = 0; ks < KS; ++ks) z += Zp[(ks * RS + rl) * QT_LDZ + j];
+      Z1[rl * QT_LDZ + j] = z;
+    }
+    __syncthreads();
+    // ---------------- Z2 = -(Z S^T):  Z2[rl][j] = -sum_{j' >= j} Z[rl][j'] S[j][j'] ----------------
+    double z2v[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int idx = tid + q * QT_THREADS;
+      z2v[q] = 0.0;
+      if (idx < RS * WY_NB) {
+        const int rl = idx >> 5, j = idx & 31;
+        double z = 0.0;
+        for (int jp = j; jp < WY_NB; ++jp) z += Z1[rl * QT_LDZ + jp] * Ss[j * (WY_NB + 1) + jp];
+        z2v[q] = -z;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int idx = tid + q * QT_THREADS;
+      if (idx < RS * WY_NB) Z1[(idx >> 5) * QT_LDZ + (idx & 31)] = z2v[q];
+    }
+    __syncthreads();
+    // ---------------- X += Z2 Y^T ----------------
+    const int units_u = nrt * 8;                           // (row tile, column tile of 8 inside the chunk)
+    for (int cs = cbeg; cs < n; cs += QT_KC) {
+      for (int idx = tid; idx < WY_NB * QT_KC; idx += QT_THREADS) {
+        const int j = idx >> 6, cl = idx & 63, cc = cs + cl;
+        double v = 0.0;
+        if (j < nbk && cc < n && cc >= kb + j + 1) v = A[(size_t)(kb + j) * n + cc];
+        Ys[j * QT_LD + cl] = v;
+      }
+      __syncthreads();
+      for (int u = warp; u < units_u; u += 32) {
+        const int rt = u >> 3, nt = u & 7;
+        const int rl = rt * 8 + gid;
+        const int cc = cs + nt * 8 + 2 * tig;
+        const bool live = (rl < Ract) && (cc < n);         // n is even: cc + 1 < n as well
+        double* xp = P + (size_t)(c + (size_t)(t0 + (rl < Ract ? rl : 0)) * G) * n + cc;
+        double2 cv = make_double2(0.0, 0.0);
+        if (live) cv = *reinterpret_cast<const double2*>(xp);
+        const double* za = Z1 + rl * QT_LDZ + tig;
+        const double* yb = Ys + tig * QT_LD + nt * 8 + gid;
+#pragma unroll
+        for (int kk = 0; kk < WY_NB; kk += 4) dmma_8x8x4(cv.x, cv.y, za[kk], yb[kk * QT_LD]);
+        if (live) *reinterpret_cast<double2*>(xp) = cv;
+      }
+      __syncthreads();
+    }
+  }
 }
 
 cudaError_t tridiag_form_qt(Ctx* c) {
   const int n = c->n;
-  int rpb = (int)((200 * 1024) / ((size_t)n * sizeof(double)));
-  if (rpb > 8) rpb = 8;
-  if (rpb < 1) return cudaErrorInvalidValue;
-  const size_t smem = (size_t)rpb * n * sizeof(double);
-  cudaError_t e = cudaFuncSetAttribute(form_qt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const int nrefl = n - 2;
+  const int nblk = (nrefl + WY_NB - 1) / WY_NB;
+  double* Sall = c->wy_s;
+  cudaError_t e = cudaMemsetAsync(c->P64, 0, (size_t)n * n * sizeof(double), c->stream);
   if (e != cudaSuccess) return e;
-  form_qt_kernel<<<(n + rpb - 1) / rpb, rpb * 32, smem, c->stream>>>(c->A64, c->beta, n, c->P64, rpb);
+  set_identity_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(c->P64, n);
+  c->launches++;
+  wy_factor_kernel<<<nblk, 1024, 0, c->stream>>>(c->A64, c->beta, n, Sall);
+  c->launches++;
+  const size_t smem = (size_t)(WY_NB * QT_LD + QT_RS_MAX * QT_LD + 2 * QT_RS_MAX * QT_LDZ +
+                               WY_NB * (WY_NB + 1)) * sizeof(double);
+  e = cudaFuncSetAttribute(form_qt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  int grid = c->num_sms;
+  while ((n + grid - 1) / grid > QT_RS_MAX) grid += c->num_sms;   // at most 128 rows per CTA
+  form_qt_kernel<<<grid, QT_THREADS, smem, c->stream>>>(c->A64, Sall, n, nblk, c->P64);
   c->launches++;
   return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------------
 // Per-penalty factor: LDL^T of T/rho + I (unit lower bidiagonal L, diagonal D), one thread per
-// penalty value.  (T/rho + I) is the W-update matrix of Eq. 7 divided by rho, in the Q basis.
+// penalty value, fp64 arithmetic.  (T/rho + I) is the W-update matrix of Eq. 7 divided by rho, in the
+// Q basis.  The factor is stored in fp32 in the order the solve kernel reads it: element
+// i = t * ept + e (thread t, e-th element of its segment) at [e * SOLVE_THREADS + t].
 // ------------------------------------------------------------------------------------------------
+constexpr int SOLVE_THREADS = 256;
+
+int solve_ept(int n) { return (n + SOLVE_THREADS - 1) / SOLVE_THREADS; }
+size_t stage_factor_stride(int n) { return (size_t)solve_ept(n) * SOLVE_THREADS; }
+
 __global__ void stage_factors_kernel(const double* __restrict__ td, const double* __restrict__ te, int n,
-                                     const double* __restrict__ rho, int first, int count,
-                                     double* __restrict__ L, double* __restrict__ invD, int* status) {
+                                     const double* __restrict__ rho, int first, int count, int ept,
+                                     float* __restrict__ L, float* __restrict__ invD, int* status) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= count) return;
   const int stage = first + t;
   const double inv_r = 1.0 / rho[stage];
-  double* l = L + (long long)stage * n;
-  double* id = invD + (long long)stage * n;
+  const size_t stride = (size_t)ept * SOLVE_THREADS;
+  float* l = L + (size_t)stage * stride;
+  float* id = invD + (size_t)stage * stride;
   double piv = 1.0 + td[0] * inv_r;
   bool bad = false;
   for (int i = 0; i < n; ++i) {
     if (!(piv > 0.0)) bad = true;
     const double ip = 1.0 / piv;
-    id[i] = ip;
+    const size_t q = (size_t)(i % ept) * SOLVE_THREADS + i / ept;
+    id[q] = (float)ip;
     if (i < n - 1) {
       const double b = te[i] * inv_r;
       const double li = b * ip;
-      l[i] = li;
+      l[q] = (float)li;
       piv = (1.0 + td[i + 1] * inv_r) - li * b;
     } else {
-      l[i] = 0.0;
+      l[q] = 0.0f;
     }
   }
   if (bad) raise_status(status, ST_NOT_SPD);
@@ -203,131 +536,147 @@ __global__ void stage_factors_kernel(const double* __restrict__ td, const double
 
 void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count) {
   stage_factors_kernel<<<(count + 63) / 64, 64, 0, c->stream>>>(c->td, c->te, c->n, rho_dev, first, count,
-                                                               c->stage_l, c->stage_invd, c->status);
+                                                               solve_ept(c->n), c->stage_l, c->stage_invd,
+                                                               c->status);
   c->launches++;
 }
 
 // ------------------------------------------------------------------------------------------------
-// Y' = (T/rho + I)^{-1} Y row by row (one warp per output channel).  Both substitutions are first-
-// order linear recurrences x_i = y_i - l x_{i-1}; each lane runs its contiguous segment once to get
-// the segment's affine map, the 32 maps are combined by a warp scan, and a second run applies the
-// carry.  The factor (l, 1/d) of this penalty is staged once per CTA in shared memory in the same
-// padded layout as the rows, so every lane's walk through its segment is bank-conflict free.
-// fp64 registers, fp32 shared memory, result written as two bf16 planes.
+// Y' = (T/rho + I)^{-1} Y row by row.  Both substitutions are first-order linear recurrences
+// x_i = y_i - l x_{i-1}.  One CTA per row at a time: every thread owns a contiguous segment, runs it
+// once to get the segment's affine map x_out = c + m x_in, the 256 maps are combined by a block-wide
+// scan, and a second run applies the carry.  The right-hand side Y carries the ~1e-5 relative error of
+// the split-bf16 product, and the LDL^T substitution of a positive definite matrix is backward stable,
+// so fp32 arithmetic adds nothing visible to it.  Result written as two fp16 planes of the row times
+// a power of two (largest magnitude brought to [2^13, 2^14)), with the inverse scale per row.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ int pad_index(int i, int seg, int stride) { return (i / seg) * stride + (i % seg); }
+struct Affine {
+  float c, m;
+};
+// map `second` applied after map `first`
+__device__ __forceinline__ Affine then(Affine first, Affine second) {
+  Affine r;
+  r.c = fmaf(second.m, first.c, second.c);
+  r.m = second.m * first.m;
+  return r;
+}
 
-__global__ void tridiag_solve_kernel(const float* __restrict__ Y, int p, int n,
-                                     const double* __restrict__ L, const double* __restrict__ invD,
-                                     bf16* __restrict__ Yhi, bf16* __restrict__ Ylo, int seg, int stride) {
-  extern __shared__ float smf[];
-  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, wpb = blockDim.x >> 5;
-  float* sl = smf;                         // l_i,     padded
-  float* sd = smf + stride * 32;           // 1 / d_i, padded
-  float* rs = smf + (size_t)(2 + wid) * stride * 32;
-  for (int i = threadIdx.x; i < n; i += blockDim.x) {
-    const int q = pad_index(i, seg, stride);
-    sl[q] = (float)L[i];
-    sd[q] = (float)invD[i];
-  }
-  __syncthreads();
-  const int a = min(n, lane * seg), b = min(n, (lane + 1) * seg);
-  const int len = b - a;
-  float* mine = rs + lane * stride;        // mine[t] is element a + t
-  const float* ml = sl + lane * stride;    // ml[t] = l_{a+t}
-  const float* md = sd + lane * stride;
-  // l_{a-1}: the multiplier that couples this segment to the previous one
-  const double l_prev = (a > 0 && a < n) ? (double)sl[pad_index(a - 1, seg, stride)] : 0.0;
+__global__ void __launch_bounds__(SOLVE_THREADS)
+tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, int ept, const float* __restrict__ lT,
+                     const float* __restrict__ dT, bf16* __restrict__ Yhi, bf16* __restrict__ Ylo,
+                     float* __restrict__ row_inv) {
+  extern __shared__ float xs[];                            // [SOLVE_THREADS][ept | 1]
+  __shared__ Affine wtot[SOLVE_THREADS / 32];
+  __shared__ float mscratch[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int stride = ept | 1;
+  const int a0 = tid * ept;
+  const int len = a0 >= n ? 0 : (n - a0 < ept ? n - a0 : ept);
+  float* mine = xs + tid * stride;
+  const float l_before = (tid > 0 && len > 0) ? lT[(size_t)(ept - 1) * SOLVE_THREADS + tid - 1] : 0.0f;
 
-  for (int j = blockIdx.x * wpb + wid; j < p; j += gridDim.x * wpb) {
-    const float* y = Y + (long long)j * n;
-    for (int i = lane; i < n; i += 32) rs[pad_index(i, seg, stride)] = y[i];
-    __syncwarp();
-    // ---- forward substitution  x_i = y_i - l_{i-1} x_{i-1} ----
+  for (int j = blockIdx.x; j < p; j += gridDim.x) {
+    const float* y = Y + (size_t)j * n;
+    for (int i = tid * 4; i < n; i += SOLVE_THREADS * 4) {       // n is a multiple of 8
+      const float4 v = *reinterpret_cast<const float4*>(y + i);
+      const float vv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) xs[((i + e) / ept) * stride + (i + e) % ept] = vv[e];
+    }
+    __syncthreads();
+    // ---- forward substitution x_i = y_i - l_{i-1} x_{i-1}, then the diagonal ----
     {
-      double cc = 0.0, mm = 1.0, lp = l_prev;
-#pragma unroll 4
+      Affine f{0.0f, 1.0f};
+      float lp = l_before;
       for (int t = 0; t < len; ++t) {
-        cc = (double)mine[t] - lp * cc;
-        mm *= -lp;
-        lp = (double)ml[t];
+        f.c = fmaf(-lp, f.c, mine[t]);
+        f.m *= -lp;
+        lp = lT[(size_t)t * SOLVE_THREADS + tid];
       }
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
-        const double c2 = __shfl_up_sync(0xffffffffu, cc, off);
-        const double m2 = __shfl_up_sync(0xffffffffu, mm, off);
-        if (lane >= off) {
-          cc = cc + mm * c2;
-          mm = mm * m2;
-        }
+        Affine o;
+        o.c = __shfl_up_sync(0xffffffffu, f.c, off);
+        o.m = __shfl_up_sync(0xffffffffu, f.m, off);
+        if (lane >= off) f = then(o, f);
       }
-      double x = __shfl_up_sync(0xffffffffu, cc, 1);
-      if (lane == 0) x = 0.0;
-      lp = l_prev;
-#pragma unroll 4
+      if (lane == 31) wtot[warp] = f;
+      __syncthreads();
+      Affine pre{0.0f, 1.0f};
+      for (int w = 0; w < warp; ++w) pre = then(pre, wtot[w]);
+      float x = __shfl_up_sync(0xffffffffu, then(pre, f).c, 1);
+      if (lane == 0) x = pre.c;
+      lp = l_before;
       for (int t = 0; t < len; ++t) {
-        x = (double)mine[t] - lp * x;
-        lp = (double)ml[t];
-        mine[t] = (float)(x * (double)md[t]);
+        x = fmaf(-lp, x, mine[t]);
+        lp = lT[(size_t)t * SOLVE_THREADS + tid];
+        mine[t] = x * dT[(size_t)t * SOLVE_THREADS + tid];
       }
+      __syncthreads();
     }
-    __syncwarp();
-    // ---- backward substitution  z_i = x_i - l_i z_{i+1} ----
+    // ---- backward substitution z_i = x_i - l_i z_{i+1} ----
     {
-      double cc = 0.0, mm = 1.0;
-#pragma unroll 4
+      Affine f{0.0f, 1.0f};
       for (int t = len - 1; t >= 0; --t) {
-        const double li = (double)ml[t];
-        cc = (double)mine[t] - li * cc;
-        mm *= -li;
+        const float li = lT[(size_t)t * SOLVE_THREADS + tid];
+        f.c = fmaf(-li, f.c, mine[t]);
+        f.m *= -li;
       }
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
-        const double c2 = __shfl_down_sync(0xffffffffu, cc, off);
-        const double m2 = __shfl_down_sync(0xffffffffu, mm, off);
-        if (lane + off < 32) {
-          cc = cc + mm * c2;
-          mm = mm * m2;
-        }
+        Affine o;
+        o.c = __shfl_down_sync(0xffffffffu, f.c, off);
+        o.m = __shfl_down_sync(0xffffffffu, f.m, off);
+        if (lane + off < 32) f = then(o, f);
       }
-      double z = __shfl_down_sync(0xffffffffu, cc, 1);
-      if (lane == 31) z = 0.0;
-#pragma unroll 4
+      if (lane == 0) wtot[warp] = f;
+      __syncthreads();
+      Affine post{0.0f, 1.0f};
+      for (int w = SOLVE_THREADS / 32 - 1; w > warp; --w) post = then(post, wtot[w]);
+      float z = __shfl_down_sync(0xffffffffu, then(post, f).c, 1);
+      if (lane == 31) z = post.c;
+      float zmax = 0.0f;
       for (int t = len - 1; t >= 0; --t) {
-        z = (double)mine[t] - (double)ml[t] * z;
-        mine[t] = (float)z;
+        z = fmaf(-lT[(size_t)t * SOLVE_THREADS + tid], z, mine[t]);
+        mine[t] = z;
+        zmax = fmaxf(zmax, fabsf(z));
+      }
+      zmax = block_max(zmax, mscratch);                    // its barriers also publish the row
+      float inv;
+      const float sc = pow2_scale_for(zmax, &inv);
+      if (tid == 0) row_inv[j] = inv;
+      for (int i = tid * 8; i < n; i += SOLVE_THREADS * 8) {
+        __align__(16) __half hh[8];
+        __align__(16) __half ll[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          split_f16(xs[((i + e) / ept) * stride + (i + e) % ept] * sc, hh[e], ll[e]);
+        *reinterpret_cast<uint4*>(Yhi + (size_t)j * n + i) = *reinterpret_cast<const uint4*>(hh);
+        *reinterpret_cast<uint4*>(Ylo + (size_t)j * n + i) = *reinterpret_cast<const uint4*>(ll);
       }
     }
-    __syncwarp();
-    for (int i = lane; i < n; i += 32) {
-      bf16 h, l;
-      split_bf16(rs[pad_index(i, seg, stride)], h, l);
-      Yhi[(long long)j * n + i] = h;
-      Ylo[(long long)j * n + i] = l;
-    }
-    __syncwarp();
+    __syncthreads();
   }
 }
 
 void launch_tridiag_solve(Ctx* c, int p, int stage) {
   const int n = c->n;
-  const int seg = (n + 31) / 32;
-  const int stride = seg | 1;
-  const size_t per_row = (size_t)stride * 32 * sizeof(float);
-  int wpb = (int)((200 * 1024) / per_row) - 2;
-  if (wpb > 16) wpb = 16;
-  if (wpb < 1) wpb = 1;
-  const size_t smem = per_row * (wpb + 2);
+  const int ept = solve_ept(n);
+  const size_t smem = (size_t)SOLVE_THREADS * (ept | 1) * sizeof(float);
   static bool attr_set = false;
   if (!attr_set) {
-    cudaFuncSetAttribute(tridiag_solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+    cudaFuncSetAttribute(tridiag_solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
     attr_set = true;
   }
-  int blocks = (p + wpb - 1) / wpb;
-  if (blocks > c->num_sms) blocks = c->num_sms;
-  tridiag_solve_kernel<<<blocks, wpb * 32, smem, c->stream>>>(
-      c->Y, p, n, c->stage_l + (long long)stage * n, c->stage_invd + (long long)stage * n, c->Y_hi,
-      c->Y_lo, seg, stride);
+  int per_sm = (int)((200 * 1024) / (smem + 1024));
+  if (per_sm > 8) per_sm = 8;
+  if (per_sm < 1) per_sm = 1;
+  int blocks = c->num_sms * per_sm;
+  if (blocks > p) blocks = p;
+  const size_t fs = stage_factor_stride(n);
+  tridiag_solve_kernel<<<blocks, SOLVE_THREADS, smem, c->stream>>>(
+      c->Y, p, n, ept, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi,
+      c->Y_lo, c->rs_Y);
   c->launches++;
 }
 
