@@ -76,6 +76,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
   return true;
 }
+// The same wait for a whole warp: lane 0 polls, the others sleep at the shuffle, so that the 16 worker
+// warps do not all hammer one barrier word.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               int* status) {
+  int ok = 1;
+  if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status) ? 1 : 0;
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x,
                                             int y) {
   asm volatile(
@@ -137,103 +145,99 @@ struct TcMaps {
   CUtensorMap b[2];
 };
 
-// ------------------------------------------------------------------ epilogue on 4 columns of one row
-// `a` holds the 4 products (already unscaled).  Everything is indexed statically so that the running
-// sums stay in registers; chunks of 4 keep the worker threads under their register budget.
-struct AdmmIn {
-  float4 w, v, s;
-  uint32_t codes;
-};
-__device__ __forceinline__ AdmmIn admm_load4(const EpiParams& P, long long o, int col) {
-  AdmmIn in;
-  in.w = *reinterpret_cast<const float4*>(P.Whs + o);
-  in.v = *reinterpret_cast<const float4*>(P.V + o);
-  in.s = *reinterpret_cast<const float4*>(P.s + col);
-  in.codes = 0u;
-  if (!P.first_iter) in.codes = *reinterpret_cast<const uint32_t*>(P.codes + o);
-  return in;
-}
-__device__ __forceinline__ void admm_apply4(const EpiParams& P, long long o, const AdmmIn& in,
-                                            const float (&a)[4], float dl, float z0, float& r2, float& s2) {
-  const float wh[4] = {in.w.x, in.w.y, in.w.z, in.w.w};
-  const float vv[4] = {in.v.x, in.v.y, in.v.z, in.v.w};
-  const float ss[4] = {in.s.x, in.s.y, in.s.z, in.s.w};
-  float vn[4], rn[4];
-  uint32_t cn = 0u;
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const int code_old = (int)((in.codes >> (8 * e)) & 0xffu);
-    AdmmElem r = admm_elem(a[e], wh[e], vv[e], code_old, ss[e], dl, z0, P);
-    vn[e] = r.v_new;
-    cn |= (uint32_t)r.code << (8 * e);
-    rn[e] = r.r_next;
-    r2 += r.dr2;
-    s2 += r.ds2;
-  }
-  *reinterpret_cast<float4*>(P.V + o) = make_float4(vn[0], vn[1], vn[2], vn[3]);
-  *reinterpret_cast<uint32_t*>(P.codes + o) = cn;
-  *reinterpret_cast<float4*>(P.Rnext + o) = make_float4(rn[0], rn[1], rn[2], rn[3]);
-}
+// ------------------------------------------------------------------ epilogue
+// A worker warp holds a 32-row x 64-column block of products, one row per lane.  Global accesses in
+// that ownership would touch 32 different lines per instruction, 16 bytes each, and choke the
+// load/store queue next to the draining warps.  So the block goes through a small per-warp staging
+// buffer in pieces of 8 columns: each lane writes its 8 values, then takes 4 consecutive values of
+// another row (lane / 2 + 16 i, columns 4 (lane & 1) ...), so that every global instruction covers 16
+// rows x 32 bytes in whole sectors.
+constexpr int PIECE_COLS = 8;
+constexpr int STAGE_FLOATS = 32 * PIECE_COLS;            // per worker warp
 
-// The 64 columns [col0, col0 + 64) of output row `row`, products in `sums`.
+// Four consecutive elements (row, col .. col + 3) of the output, products in `acc` (unscaled values).
 template <int EPI>
-__device__ __forceinline__ void epilogue_row64(const EpiParams& P, int row, int col0, int M, int N,
-                                               const float (&sums)[COLS_PER_THREAD], float& r2, float& s2) {
-  if (row >= M || col0 >= N) return;
-  const float sc = epi_row_factor(P, row);
-  const bool full = (col0 + COLS_PER_THREAD <= N);
+__device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, int N, const float4 acc,
+                                          float& r2, float& s2) {
+  const float a[4] = {acc.x, acc.y, acc.z, acc.w};
   if (EPI == EPI_ADMM) {
-    const long long base = (long long)row * N + col0;
-    if (full && (P.group_size & 3) == 0) {
-      // one (Delta, z0) per 4 columns; inputs of chunk c + 1 are requested before chunk c is computed
-      AdmmIn cur = admm_load4(P, base, col0);
-      const bool one_group = (P.group_size % COLS_PER_THREAD) == 0;   // then (Delta, z0) is fixed here
-      long long gi = (long long)row * P.n_groups + col0 / P.group_size;
-      float dl = P.delta[gi], z0 = P.zero[gi];
+    const long long o = (long long)row * N + col;
+    const float4 w = *reinterpret_cast<const float4*>(P.Whs + o);
+    const float4 v = *reinterpret_cast<const float4*>(P.V + o);
+    const float4 s = *reinterpret_cast<const float4*>(P.s + col);
+    uint32_t codes = 0u;
+    if (!P.first_iter) codes = *reinterpret_cast<const uint32_t*>(P.codes + o);
+    const float wh[4] = {w.x, w.y, w.z, w.w};
+    const float vv[4] = {v.x, v.y, v.z, v.w};
+    const float ss[4] = {s.x, s.y, s.z, s.w};
+    const bool one_group = (P.group_size & 3) == 0;        // then the 4 columns share (Delta, z0)
+    long long gi = (long long)row * P.n_groups + col / P.group_size;
+    float dl = P.delta[gi], z0 = P.zero[gi];
+    float vn[4], rn[4];
+    uint32_t cn = 0u;
 #pragma unroll
-      for (int c = 0; c < COLS_PER_THREAD / 4; ++c) {
-        AdmmIn nxt = cur;
-        if (c + 1 < COLS_PER_THREAD / 4) nxt = admm_load4(P, base + (c + 1) * 4, col0 + (c + 1) * 4);
-        if (!one_group) {
-          gi = (long long)row * P.n_groups + (col0 + c * 4) / P.group_size;
-          dl = P.delta[gi];
-          z0 = P.zero[gi];
-        }
-        float a[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) a[e] = sums[c * 4 + e] * sc;
-        admm_apply4(P, base + c * 4, cur, a, dl, z0, r2, s2);
-        cur = nxt;
+    for (int e = 0; e < 4; ++e) {
+      if (!one_group && e > 0) {
+        gi = (long long)row * P.n_groups + (col + e) / P.group_size;
+        dl = P.delta[gi];
+        z0 = P.zero[gi];
       }
+      const int code_old = (int)((codes >> (8 * e)) & 0xffu);
+      AdmmElem r = admm_elem(a[e], wh[e], vv[e], code_old, ss[e], dl, z0, P);
+      vn[e] = r.v_new;
+      cn |= (uint32_t)r.code << (8 * e);
+      rn[e] = r.r_next;
+      r2 += r.dr2;
+      s2 += r.ds2;
+    }
+    *reinterpret_cast<float4*>(P.V + o) = make_float4(vn[0], vn[1], vn[2], vn[3]);
+    *reinterpret_cast<uint32_t*>(P.codes + o) = cn;
+    *reinterpret_cast<float4*>(P.Rnext + o) = make_float4(rn[0], rn[1], rn[2], rn[3]);
+    return;
+  }
+  float* cp = P.C + (long long)row * P.ldc + col;
+  float o[4] = {a[0], a[1], a[2], a[3]};
+  if (EPI == EPI_WOUT) {
+    const float4 c = *reinterpret_cast<const float4*>(P.Whs + (long long)row * N + col);
+    o[0] += c.x; o[1] += c.y; o[2] += c.z; o[3] += c.w;
+  }
+  if (EPI == EPI_ACCUM) {
+    if (P.lower_only && col + 3 > row) {                   // the tile straddles the diagonal
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (col + e <= row) cp[e] += o[e];
       return;
     }
-#pragma unroll
-    for (int e = 0; e < COLS_PER_THREAD; ++e)
-      if (col0 + e < N) epi_scalar(P, row, col0 + e, N, sums[e], r2, s2);
-    return;
+    const float4 c = *reinterpret_cast<const float4*>(cp);
+    o[0] += c.x; o[1] += c.y; o[2] += c.z; o[3] += c.w;
   }
-  // STORE / ACCUM / WOUT
-  float* crow = P.C + (long long)row * P.ldc + col0;
-  const bool vec_ok = full && ((P.ldc & 3) == 0) &&
-                      (EPI != EPI_ACCUM || !P.lower_only || col0 + COLS_PER_THREAD - 1 <= row);
-  if (vec_ok) {
+  *reinterpret_cast<float4*>(cp) = make_float4(o[0], o[1], o[2], o[3]);
+}
+
+// The block rows [row0, row0 + 32) x columns [col0, col0 + 64) held by one warp.  All sizes on this path
+// keep N and the leading dimensions multiples of 4, so a group of 4 columns is inside or outside.
+template <int EPI>
+__device__ __forceinline__ void epilogue_block(const EpiParams& P, int row0, int col0, int M, int N,
+                                               const float (&sums)[COLS_PER_THREAD], float* stage, int lane,
+                                               float& r2, float& s2) {
+  const float sc = (row0 + lane < M) ? epi_row_factor(P, row0 + lane) : 0.0f;
 #pragma unroll
-    for (int q = 0; q < COLS_PER_THREAD / 4; ++q) {
-      float4 o = make_float4(sums[4 * q] * sc, sums[4 * q + 1] * sc, sums[4 * q + 2] * sc, sums[4 * q + 3] * sc);
-      if (EPI == EPI_ACCUM) {
-        const float4 c = *reinterpret_cast<const float4*>(crow + 4 * q);
-        o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
-      } else if (EPI == EPI_WOUT) {
-        const float4 c = *reinterpret_cast<const float4*>(P.Whs + (long long)row * N + col0 + 4 * q);
-        o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
-      }
-      *reinterpret_cast<float4*>(crow + 4 * q) = o;
+  for (int pc = 0; pc < COLS_PER_THREAD / PIECE_COLS; ++pc) {
+    float* mine = stage + lane * PIECE_COLS;
+    *reinterpret_cast<float4*>(mine) = make_float4(sums[pc * 8] * sc, sums[pc * 8 + 1] * sc,
+                                                   sums[pc * 8 + 2] * sc, sums[pc * 8 + 3] * sc);
+    *reinterpret_cast<float4*>(mine + 4) = make_float4(sums[pc * 8 + 4] * sc, sums[pc * 8 + 5] * sc,
+                                                       sums[pc * 8 + 6] * sc, sums[pc * 8 + 7] * sc);
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int r = (lane >> 1) + 16 * i, c4 = (lane & 1) * 4;
+      const float4 acc = *reinterpret_cast<const float4*>(stage + r * PIECE_COLS + c4);
+      const int row = row0 + r, col = col0 + pc * PIECE_COLS + c4;
+      if (row < M && col < N) epi_elem4<EPI>(P, row, col, N, acc, r2, s2);
     }
-    return;
+    __syncwarp();
   }
-#pragma unroll
-  for (int e = 0; e < COLS_PER_THREAD; ++e)
-    if (col0 + e < N) epi_scalar(P, row, col0 + e, N, sums[e], r2, s2);
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -251,6 +255,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ float red[2 * GROUP_WARPS * 2];
+  __shared__ __align__(16) float stage_all[2 * GROUP_WARPS * STAGE_FLOATS];
 
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -393,7 +398,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
       // A parity wait cannot tell a phase from the one two completions later, so a group starts
       // watching the partial barriers only once the other group has drained the tile before this one.
       if (it > 0) {
-        ok = mbar_wait(drained0 + 8 * (1 - gsel), (uint32_t)((it - 1) >> 1) & 1u, abort_flag, status);
+        ok = mbar_wait_warp(drained0 + 8 * (1 - gsel), (uint32_t)((it - 1) >> 1) & 1u, abort_flag, status);
         if (!ok) break;
       }
       float sums[COLS_PER_THREAD];
@@ -401,7 +406,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
       for (int e = 0; e < COLS_PER_THREAD; ++e) sums[e] = 0.f;
       for (int f = 0; f < num_flush; ++f) {
         const int pb = (int)(g % NPART);
-        ok = mbar_wait(pfull0 + 8 * pb, (g / NPART) & 1u, abort_flag, status);
+        ok = mbar_wait_warp(pfull0 + 8 * pb, (g / NPART) & 1u, abort_flag, status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t taddr = tmem_base + (uint32_t)pb * BN + (uint32_t)(half * COLS_PER_THREAD) +
@@ -422,8 +427,8 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
       }
       if (!ok) break;
       if (lane == 0) mbar_arrive(drained0 + 8 * gsel);
-      const int row = tm * BM + q * 32 + lane;
-      epilogue_row64<EPI>(epi, row, tn * BN + half * COLS_PER_THREAD, M, N, sums, r2, s2);
+      epilogue_block<EPI>(epi, tm * BM + q * 32, tn * BN + half * COLS_PER_THREAD, M, N, sums,
+                          stage_all + (warp - 2) * STAGE_FLOATS, lane, r2, s2);
       ++it;
     }
     if (EPI == EPI_ADMM) {
