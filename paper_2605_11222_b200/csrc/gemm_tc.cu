@@ -140,6 +140,19 @@ __host__ __device__ constexpr uint32_t idesc_128x128(uint32_t fmt) {
   return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
+// Tile order.  Consecutive tiles (the ones resident at the same time) form bands of RASTER_M tile rows
+// walked column by column, so that one wave of CTAs touches about 12 x 12 tiles: ~12 row blocks of A and
+// ~12 row blocks of B stay in L2 instead of a whole operand being streamed from HBM by every wave.
+constexpr int RASTER_M = 12;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
+  const int band = tile / (RASTER_M * tiles_n);
+  const int first = band * RASTER_M;
+  const int rows = tiles_m - first < RASTER_M ? tiles_m - first : RASTER_M;
+  const int in_band = tile - band * RASTER_M * tiles_n;
+  tn = in_band / rows;
+  tm = first + in_band - tn * rows;
+}
+
 struct TcMaps {
   CUtensorMap a[2];
   CUtensorMap b[2];
@@ -304,7 +317,8 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int tm = tile / tiles_n, tn = tile % tiles_n;
+        int tm, tn;
+        tile_coords(tile, tiles_m, tiles_n, tm, tn);
         if (lower && tn * BN > tm * BM + BM - 1) continue;
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag, status);
@@ -332,7 +346,8 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
       uint32_t g = 0;                        // flush counter, shared sequence with the workers
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int tm = tile / tiles_n, tn = tile % tiles_n;
+        int tm, tn;
+        tile_coords(tile, tiles_m, tiles_n, tm, tn);
         if (lower && tn * BN > tm * BM + BM - 1) continue;
         uint32_t d_tmem = 0, accumulate = 0;
         int pb = 0;
@@ -388,7 +403,8 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
     int it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-      const int tm = tile / tiles_n, tn = tile % tiles_n;
+      int tm, tn;
+        tile_coords(tile, tiles_m, tiles_n, tm, tn);
       if (lower && tn * BN > tm * BM + BM - 1) continue;
       if ((it & 1) != gsel) {                              // the other group's tile
         g += (uint32_t)num_flush;

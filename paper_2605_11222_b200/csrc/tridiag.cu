@@ -502,7 +502,8 @@ cudaError_t tridiag_form_qt(Ctx* c) {
 // ------------------------------------------------------------------------------------------------
 constexpr int SOLVE_THREADS = 256;
 
-int solve_ept(int n) { return (n + SOLVE_THREADS - 1) / SOLVE_THREADS; }
+// elements per thread of the solve kernel: n / 256 rounded up to a multiple of 8 (16-byte plane stores)
+int solve_ept(int n) { return (((n + SOLVE_THREADS - 1) / SOLVE_THREADS) + 7) & ~7; }
 size_t stage_factor_stride(int n) { return (size_t)solve_ept(n) * SOLVE_THREADS; }
 
 __global__ void stage_factors_kernel(const double* __restrict__ td, const double* __restrict__ te, int n,
@@ -543,12 +544,12 @@ void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count) {
 
 // ------------------------------------------------------------------------------------------------
 // Y' = (T/rho + I)^{-1} Y row by row.  Both substitutions are first-order linear recurrences
-// x_i = y_i - l x_{i-1}.  One CTA per row at a time: every thread owns a contiguous segment, runs it
-// once to get the segment's affine map x_out = c + m x_in, the 256 maps are combined by a block-wide
-// scan, and a second run applies the carry.  The right-hand side Y carries the ~1e-5 relative error of
-// the split-bf16 product, and the LDL^T substitution of a positive definite matrix is backward stable,
-// so fp32 arithmetic adds nothing visible to it.  Result written as two fp16 planes of the row times
-// a power of two (largest magnitude brought to [2^13, 2^14)), with the inverse scale per row.
+// x_i = y_i - l x_{i-1}.  One CTA per row at a time: every thread owns a contiguous segment of EPT
+// elements in registers, runs it once to get the segment's affine map x_out = c + m x_in, the 256 maps
+// are combined by a block-wide scan, and a second run applies the carry.  The LDL^T substitution of a
+// positive definite matrix is backward stable, so fp32 arithmetic keeps the result at the accuracy of
+// the fp32 right-hand side.  Result written as two fp16 planes of the row times a power of two
+// (largest magnitude brought to [2^13, 2^14)), with the inverse scale per row.
 // ------------------------------------------------------------------------------------------------
 struct Affine {
   float c, m;
@@ -561,38 +562,50 @@ __device__ __forceinline__ Affine then(Affine first, Affine second) {
   return r;
 }
 
+template <int EPT>
 __global__ void __launch_bounds__(SOLVE_THREADS)
-tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, int ept, const float* __restrict__ lT,
+tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, const float* __restrict__ lT,
                      const float* __restrict__ dT, bf16* __restrict__ Yhi, bf16* __restrict__ Ylo,
                      float* __restrict__ row_inv) {
-  extern __shared__ float xs[];                            // [SOLVE_THREADS][ept | 1]
   __shared__ Affine wtot[SOLVE_THREADS / 32];
   __shared__ float mscratch[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int stride = ept | 1;
-  const int a0 = tid * ept;
-  const int len = a0 >= n ? 0 : (n - a0 < ept ? n - a0 : ept);
-  float* mine = xs + tid * stride;
-  const float l_before = (tid > 0 && len > 0) ? lT[(size_t)(ept - 1) * SOLVE_THREADS + tid - 1] : 0.0f;
+  const int a0 = tid * EPT;
+  const int len = a0 >= n ? 0 : (n - a0 < EPT ? n - a0 : EPT);      // a multiple of 8
+  const float l_before = (tid > 0 && len > 0) ? lT[(size_t)(EPT - 1) * SOLVE_THREADS + tid - 1] : 0.0f;
 
-  for (int j = blockIdx.x; j < p; j += gridDim.x) {
-    const float* y = Y + (size_t)j * n;
-    for (int i = tid * 4; i < n; i += SOLVE_THREADS * 4) {       // n is a multiple of 8
-      const float4 v = *reinterpret_cast<const float4*>(y + i);
-      const float vv[4] = {v.x, v.y, v.z, v.w};
+  constexpr bool PREFETCH = (EPT <= 24);                   // next row's segment requested a row ahead
+  float xn[PREFETCH ? EPT : 4];
+  auto load_row = [&](int j, float* dst) {
+    const float* y = Y + (size_t)j * n + a0;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) xs[((i + e) / ept) * stride + (i + e) % ept] = vv[e];
+    for (int e = 0; e < EPT; e += 4) {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (e < len) v = *reinterpret_cast<const float4*>(y + e);
+      dst[e] = v.x; dst[e + 1] = v.y; dst[e + 2] = v.z; dst[e + 3] = v.w;
     }
-    __syncthreads();
+  };
+  if (PREFETCH && (int)blockIdx.x < p) load_row(blockIdx.x, xn);
+  for (int j = blockIdx.x; j < p; j += gridDim.x) {
+    float x[EPT];
+    if (PREFETCH) {
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) x[e] = xn[e];
+      if (j + (int)gridDim.x < p) load_row(j + gridDim.x, xn);
+    } else {
+      load_row(j, x);
+    }
     // ---- forward substitution x_i = y_i - l_{i-1} x_{i-1}, then the diagonal ----
     {
       Affine f{0.0f, 1.0f};
       float lp = l_before;
-      for (int t = 0; t < len; ++t) {
-        f.c = fmaf(-lp, f.c, mine[t]);
-        f.m *= -lp;
-        lp = lT[(size_t)t * SOLVE_THREADS + tid];
-      }
+#pragma unroll
+      for (int t = 0; t < EPT; ++t)
+        if (t < len) {
+          f.c = fmaf(-lp, f.c, x[t]);
+          f.m *= -lp;
+          lp = lT[(size_t)t * SOLVE_THREADS + tid];
+        }
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
         Affine o;
@@ -604,24 +617,29 @@ tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, int ept, const f
       __syncthreads();
       Affine pre{0.0f, 1.0f};
       for (int w = 0; w < warp; ++w) pre = then(pre, wtot[w]);
-      float x = __shfl_up_sync(0xffffffffu, then(pre, f).c, 1);
-      if (lane == 0) x = pre.c;
+      float xin = __shfl_up_sync(0xffffffffu, then(pre, f).c, 1);
+      if (lane == 0) xin = pre.c;
       lp = l_before;
-      for (int t = 0; t < len; ++t) {
-        x = fmaf(-lp, x, mine[t]);
-        lp = lT[(size_t)t * SOLVE_THREADS + tid];
-        mine[t] = x * dT[(size_t)t * SOLVE_THREADS + tid];
-      }
+#pragma unroll
+      for (int t = 0; t < EPT; ++t)
+        if (t < len) {
+          xin = fmaf(-lp, xin, x[t]);
+          lp = lT[(size_t)t * SOLVE_THREADS + tid];
+          x[t] = xin * dT[(size_t)t * SOLVE_THREADS + tid];
+        }
       __syncthreads();
     }
     // ---- backward substitution z_i = x_i - l_i z_{i+1} ----
+    float zmax = 0.0f;
     {
       Affine f{0.0f, 1.0f};
-      for (int t = len - 1; t >= 0; --t) {
-        const float li = lT[(size_t)t * SOLVE_THREADS + tid];
-        f.c = fmaf(-li, f.c, mine[t]);
-        f.m *= -li;
-      }
+#pragma unroll
+      for (int t = EPT - 1; t >= 0; --t)
+        if (t < len) {
+          const float li = lT[(size_t)t * SOLVE_THREADS + tid];
+          f.c = fmaf(-li, f.c, x[t]);
+          f.m *= -li;
+        }
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
         Affine o;
@@ -635,48 +653,52 @@ tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, int ept, const f
       for (int w = SOLVE_THREADS / 32 - 1; w > warp; --w) post = then(post, wtot[w]);
       float z = __shfl_down_sync(0xffffffffu, then(post, f).c, 1);
       if (lane == 31) z = post.c;
-      float zmax = 0.0f;
-      for (int t = len - 1; t >= 0; --t) {
-        z = fmaf(-lT[(size_t)t * SOLVE_THREADS + tid], z, mine[t]);
-        mine[t] = z;
-        zmax = fmaxf(zmax, fabsf(z));
-      }
-      zmax = block_max(zmax, mscratch);                    // its barriers also publish the row
-      float inv;
-      const float sc = pow2_scale_for(zmax, &inv);
-      if (tid == 0) row_inv[j] = inv;
-      for (int i = tid * 8; i < n; i += SOLVE_THREADS * 8) {
+#pragma unroll
+      for (int t = EPT - 1; t >= 0; --t)
+        if (t < len) {
+          z = fmaf(-lT[(size_t)t * SOLVE_THREADS + tid], z, x[t]);
+          x[t] = z;
+          zmax = fmaxf(zmax, fabsf(z));
+        }
+    }
+    zmax = block_max(zmax, mscratch);                      // its barriers also separate the rows' use of wtot
+    float inv;
+    const float sc = pow2_scale_for(zmax, &inv);
+    if (tid == 0) row_inv[j] = inv;
+#pragma unroll
+    for (int e = 0; e < EPT; e += 8) {
+      if (e < len) {
         __align__(16) __half hh[8];
         __align__(16) __half ll[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
-          split_f16(xs[((i + e) / ept) * stride + (i + e) % ept] * sc, hh[e], ll[e]);
-        *reinterpret_cast<uint4*>(Yhi + (size_t)j * n + i) = *reinterpret_cast<const uint4*>(hh);
-        *reinterpret_cast<uint4*>(Ylo + (size_t)j * n + i) = *reinterpret_cast<const uint4*>(ll);
+        for (int k = 0; k < 8; ++k) split_f16(x[e + k] * sc, hh[k], ll[k]);
+        *reinterpret_cast<uint4*>(Yhi + (size_t)j * n + a0 + e) = *reinterpret_cast<const uint4*>(hh);
+        *reinterpret_cast<uint4*>(Ylo + (size_t)j * n + a0 + e) = *reinterpret_cast<const uint4*>(ll);
       }
     }
-    __syncthreads();
   }
 }
 
+template <int EPT>
+static void launch_solve_t(Ctx* c, int p, int stage, int blocks) {
+  const size_t fs = stage_factor_stride(c->n);
+  tridiag_solve_kernel<EPT><<<blocks, SOLVE_THREADS, 0, c->stream>>>(
+      c->Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi, c->Y_lo,
+      c->rs_Y);
+}
+
 void launch_tridiag_solve(Ctx* c, int p, int stage) {
-  const int n = c->n;
-  const int ept = solve_ept(n);
-  const size_t smem = (size_t)SOLVE_THREADS * (ept | 1) * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(tridiag_solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-    attr_set = true;
-  }
-  int per_sm = (int)((200 * 1024) / (smem + 1024));
-  if (per_sm > 8) per_sm = 8;
-  if (per_sm < 1) per_sm = 1;
-  int blocks = c->num_sms * per_sm;
+  int blocks = c->num_sms * 8;
   if (blocks > p) blocks = p;
-  const size_t fs = stage_factor_stride(n);
-  tridiag_solve_kernel<<<blocks, SOLVE_THREADS, smem, c->stream>>>(
-      c->Y, p, n, ept, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi,
-      c->Y_lo, c->rs_Y);
+  switch (solve_ept(c->n)) {
+    case 8: launch_solve_t<8>(c, p, stage, blocks); break;
+    case 16: launch_solve_t<16>(c, p, stage, blocks); break;
+    case 24: launch_solve_t<24>(c, p, stage, blocks); break;
+    case 32: launch_solve_t<32>(c, p, stage, blocks); break;
+    case 40: launch_solve_t<40>(c, p, stage, blocks); break;
+    case 48: launch_solve_t<48>(c, p, stage, blocks); break;
+    default: launch_solve_t<56>(c, p, stage, blocks); break;     // n <= 14336
+  }
   c->launches++;
 }
 
