@@ -567,12 +567,20 @@ __global__ void __launch_bounds__(SOLVE_THREADS)
 tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, const float* __restrict__ lT,
                      const float* __restrict__ dT, bf16* __restrict__ Yhi, bf16* __restrict__ Ylo,
                      float* __restrict__ row_inv) {
+  extern __shared__ float fac[];                           // this penalty's factor: l then 1/d, [e][thread]
   __shared__ Affine wtot[SOLVE_THREADS / 32];
   __shared__ float mscratch[32];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float* sl = fac;
+  float* sd = fac + EPT * SOLVE_THREADS;
+  for (int i = tid; i < EPT * SOLVE_THREADS; i += SOLVE_THREADS) {
+    sl[i] = lT[i];
+    sd[i] = dT[i];
+  }
+  __syncthreads();
   const int a0 = tid * EPT;
   const int len = a0 >= n ? 0 : (n - a0 < EPT ? n - a0 : EPT);      // a multiple of 8
-  const float l_before = (tid > 0 && len > 0) ? lT[(size_t)(EPT - 1) * SOLVE_THREADS + tid - 1] : 0.0f;
+  const float l_before = (tid > 0 && len > 0) ? sl[(EPT - 1) * SOLVE_THREADS + tid - 1] : 0.0f;
 
   constexpr bool PREFETCH = (EPT <= 24);                   // next row's segment requested a row ahead
   float xn[PREFETCH ? EPT : 4];
@@ -604,7 +612,7 @@ tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, const float* __r
         if (t < len) {
           f.c = fmaf(-lp, f.c, x[t]);
           f.m *= -lp;
-          lp = lT[(size_t)t * SOLVE_THREADS + tid];
+          lp = sl[t * SOLVE_THREADS + tid];
         }
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
@@ -624,8 +632,8 @@ tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, const float* __r
       for (int t = 0; t < EPT; ++t)
         if (t < len) {
           xin = fmaf(-lp, xin, x[t]);
-          lp = lT[(size_t)t * SOLVE_THREADS + tid];
-          x[t] = xin * dT[(size_t)t * SOLVE_THREADS + tid];
+          lp = sl[t * SOLVE_THREADS + tid];
+          x[t] = xin * sd[t * SOLVE_THREADS + tid];
         }
       __syncthreads();
     }
@@ -636,7 +644,7 @@ tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, const float* __r
 #pragma unroll
       for (int t = EPT - 1; t >= 0; --t)
         if (t < len) {
-          const float li = lT[(size_t)t * SOLVE_THREADS + tid];
+          const float li = sl[t * SOLVE_THREADS + tid];
           f.c = fmaf(-li, f.c, x[t]);
           f.m *= -li;
         }
@@ -656,7 +664,7 @@ tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, const float* __r
 #pragma unroll
       for (int t = EPT - 1; t >= 0; --t)
         if (t < len) {
-          z = fmaf(-lT[(size_t)t * SOLVE_THREADS + tid], z, x[t]);
+          z = fmaf(-sl[t * SOLVE_THREADS + tid], z, x[t]);
           x[t] = z;
           zmax = fmaxf(zmax, fabsf(z));
         }
@@ -682,13 +690,19 @@ tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, const float* __r
 template <int EPT>
 static void launch_solve_t(Ctx* c, int p, int stage, int blocks) {
   const size_t fs = stage_factor_stride(c->n);
-  tridiag_solve_kernel<EPT><<<blocks, SOLVE_THREADS, 0, c->stream>>>(
+  const size_t smem = (size_t)2 * EPT * SOLVE_THREADS * sizeof(float);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(tridiag_solve_kernel<EPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    attr_set = true;
+  }
+  tridiag_solve_kernel<EPT><<<blocks, SOLVE_THREADS, smem, c->stream>>>(
       c->Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi, c->Y_lo,
       c->rs_Y);
 }
 
 void launch_tridiag_solve(Ctx* c, int p, int stage) {
-  int blocks = c->num_sms * 8;
+  int blocks = c->num_sms * 3;                             // resident CTAs; each loads the factor once
   if (blocks > p) blocks = p;
   switch (solve_ept(c->n)) {
     case 8: launch_solve_t<8>(c, p, stage, blocks); break;
