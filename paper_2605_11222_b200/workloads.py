@@ -167,6 +167,23 @@ def config5(n_blocks: int = 36, n_tokens: int = 131072):
     return out
 
 
+def named_workload(name: str) -> LayerSpec:
+    """One layer of the benchmark configurations by name: cfg1, cfg2, cfg3_<gate|up|down>,
+    cfg4_<k|v|o>, cfg5_<q|k|v|o|gate|up|down> (block 0 of the 36-block stack)."""
+    if name == "cfg1":
+        return config1()
+    if name == "cfg2":
+        return config2()
+    table = {}
+    for s in config3() + config4():
+        table[s.name.replace("_proj", "")] = s
+    for s in config5(n_blocks=1):
+        table[s.name.replace("_b0", "")] = s
+    if name not in table:
+        raise KeyError(f"unknown workload {name!r}; known: cfg1, cfg2, {', '.join(sorted(table))}")
+    return table[name]
+
+
 def small_case(d_in=512, d_out=384, n_tokens=6144, **kw) -> LayerSpec:
     """Mid-size parity case: several tiles and a ragged tail, seconds on the CPU checker."""
     base = dict(x_dtype="bf16", bits=3, group_size=128, T=40, rho0=0.1, gamma=1.25, seed=77,
