@@ -1,7 +1,7 @@
 // Greedy single-entry local search (Sec. 3.5; Eq. 11 with the second perturbation zero).
 // One CTA per output channel: its gradient g = H (w_q - w_hat), its codes and diag(H) stay in shared
-// memory; every step scans the 2 n candidate moves, a block-wide argmin picks the best one, and the
-// gradient takes the rank-1 correction g += d H[:, i] (row i of the symmetric H, contiguous).
+// memory (the diagonal as Delta_i^2 H_ii, the quadratic term of a move); every step scans the 2 n
+// candidate moves, a block-wide argmin picks the best one, and the gradient takes the rank-1 correction g += d H[:, i] (row i of the symmetric H, contiguous).
 #include "internal.h"
 
 namespace admmq {
@@ -16,7 +16,7 @@ __device__ __forceinline__ Cand better(Cand a, Cand b) {
   return a;
 }
 
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(512)
 local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag, int n, int p, int gs,
                     int kmax, long long max_moves, float tau, const float* __restrict__ W0,
                     unsigned char* __restrict__ codes, const float* __restrict__ delta,
@@ -24,17 +24,21 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
                     long long* __restrict__ moves_out, int* __restrict__ capped_out) {
   extern __shared__ float smf[];
   float* g = smf;                  // [n]
-  float* hd = smf + n;             // [n]
-  unsigned char* kc = (unsigned char*)(smf + 2 * n);   // [n]
-  __shared__ Cand wbest[8];
+  float* quad = smf + n;           // [n]  Delta_i^2 H_ii, the quadratic term of a move of entry i
+  float* sdl = smf + 2 * n;        // [n / gs]  this channel's Delta per group
+  unsigned char* kc = (unsigned char*)(smf + 2 * n + n / gs);   // [n]
+  __shared__ Cand wbest[16];
   __shared__ Cand chosen;
   const int j = blockIdx.x;
   if (j >= p) return;
   const int ng = n / gs;
   const float* dl = delta + (long long)j * ng;
+  const int shift = (gs & (gs - 1)) == 0 ? __ffs(gs) - 1 : -1;   // group of entry i: i >> shift, or i / gs
+  for (int i = threadIdx.x; i < ng; i += blockDim.x) sdl[i] = dl[i];
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const float d = dl[i / gs];
     g[i] = g_glob[(long long)j * n + i];
-    hd[i] = hdiag[i];
+    quad[i] = d * d * hdiag[i];
     kc[i] = codes[(long long)j * n + i];
   }
   __syncthreads();
@@ -45,13 +49,21 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
     Cand best;
     best.cost = INFINITY;
     best.idx = 0x7fffffff;
+    // a thread meets its candidates in increasing index order, so a strict "<" keeps the earliest
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
-      const float d = dl[i / gs];
-      const float quad = d * d * hd[i];
+      const float d = sdl[shift >= 0 ? (i >> shift) : (i / gs)];
+      const float q = quad[i];
       const float lin = 2.0f * d * g[i];
       const int k = kc[i];
-      if (k < kmax) best = better(best, Cand{lin + quad, 2 * i});
-      if (k > 0) best = better(best, Cand{-lin + quad, 2 * i + 1});
+      const float cp = lin + q, cm = q - lin;
+      if (k < kmax && cp < best.cost) {
+        best.cost = cp;
+        best.idx = 2 * i;
+      }
+      if (k > 0 && cm < best.cost) {
+        best.cost = cm;
+        best.idx = 2 * i + 1;
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -67,8 +79,7 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
       for (int w = 1; w < nw; ++w) b = better(b, wbest[w]);
       if (b.idx != 0x7fffffff) {
         const int i = b.idx >> 1;
-        const float d = dl[i / gs];
-        if (!(b.cost < -tau * hd[i] * d * d)) b.idx = -1;   // no improving move: stop
+        if (!(b.cost < -tau * quad[i])) b.idx = -1;         // no improving move: stop
       } else {
         b.idx = -1;
       }
@@ -106,11 +117,12 @@ cudaError_t launch_local_search(Ctx* c, const float* W0, int p, int bits, int gs
                                 float tau, unsigned char* codes, const float* delta, const float* zero,
                                 float* Wq, float* g, long long* d_moves, int* d_capped) {
   const int n = c->n;
-  const size_t smem = (size_t)n * 9 + 16;
+  const size_t smem = (size_t)n * 9 + (size_t)(n / gs) * 4 + 16;
+  const int threads = n >= 8192 ? 512 : 256;               // long rows: more warps per channel
   cudaError_t e = cudaFuncSetAttribute(local_search_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  local_search_kernel<<<p, 256, smem, c->stream>>>(c->H, c->hdiag, n, p, gs, (1 << bits) - 1, max_moves,
+  local_search_kernel<<<p, threads, smem, c->stream>>>(c->H, c->hdiag, n, p, gs, (1 << bits) - 1, max_moves,
                                                    tau, W0, codes, delta, zero, Wq, g, d_moves, d_capped);
   c->launches++;
   return cudaGetLastError();
