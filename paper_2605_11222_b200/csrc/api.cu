@@ -71,6 +71,7 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   c.pvec = cv.take<double>(n);
   c.stage_l = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
   c.stage_invd = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
+  c.trd_ws = cv.take<double>(tridiag_blocked_scratch_doubles(n));
   c.wy_s = cv.take<double>((size_t)((n + 31) / 32) * 1024);
   c.Q_hi = cv.take<bf16>(nn);
   c.Q_lo = cv.take<bf16>(nn);

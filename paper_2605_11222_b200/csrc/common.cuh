@@ -67,6 +67,14 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;
 }
 
+// D (8x8, fp64) += A (8x4) B (4x8) on the fp64 tensor-core MMA.  Lane l holds A[l / 4][l % 4],
+// B[l % 4][l / 4] and D[l / 4][2 (l % 4) .. + 1].
+__device__ __forceinline__ void dmma_8x8x4(double& d0, double& d1, double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d0), "+d"(d1)
+               : "d"(a), "d"(b));
+}
+
 // Sum over the block, result in every thread.  `scratch` holds >= 32 elements.
 template <typename T>
 __device__ __forceinline__ T block_sum(T v, T* scratch) {

@@ -53,6 +53,7 @@ struct Ctx {
   double* pvec = nullptr;       // [n] matrix-vector scratch of the reduction
   float* stage_l = nullptr;     // [T_max+1][stage_factor_stride(n)] LDL^T multipliers per penalty
   float* stage_invd = nullptr;  // [T_max+1][stage_factor_stride(n)] LDL^T inverse pivots per penalty
+  double* trd_ws = nullptr;     // scratch of the blocked reduction: 66 n + 67 * 256 doubles
   double* wy_s = nullptr;       // [ceil(n/32)][32][32] triangular factors of the reflector blocks
   bf16 *Q_hi = nullptr, *Q_lo = nullptr;    // [n][n] Q   (row i, col m)
   bf16 *QT_hi = nullptr, *QT_lo = nullptr;  // [n][n] Q^T (row m, col k)
@@ -103,6 +104,8 @@ int gemm_tc_partial_slots(int num_sms);
 
 // ---- tridiag.cu ----
 cudaError_t tridiag_reduce(Ctx* c);                 // A64 -> td, te, reflectors, beta
+cudaError_t tridiag_reduce_blocked(Ctx* c);         // the same result, panels of 32 columns
+size_t tridiag_blocked_scratch_doubles(int n);
 cudaError_t tridiag_form_qt(Ctx* c);                // reflectors -> P64 = Q^T
 size_t stage_factor_stride(int n);                  // floats per penalty in stage_l / stage_invd
 void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count);

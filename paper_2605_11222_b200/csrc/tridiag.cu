@@ -31,6 +31,7 @@ namespace admmq {
 // Output: td/te (diagonal / off-diagonal of T), reflector k in A[k, k+1:], beta[k].
 // ------------------------------------------------------------------------------------------------
 constexpr int TRD_THREADS = 1024;
+constexpr int TRD_BLOCKED_FROM = 6144;
 constexpr int TRD_PSUM = 512;
 
 struct TrdArgs {
@@ -232,6 +233,12 @@ static int trd_cap(int n, int C) {
 
 cudaError_t tridiag_reduce(Ctx* c) {
   const int n = c->n;
+  // The blocked kernel halves the traffic per column but pays a second grid barrier and more serial
+  // work per column; measured, it wins from about n = 6000 (n = 4096: 100 ms vs 84 ms; n = 12288: 1.4 s vs 2.0 s).
+  if (n >= TRD_BLOCKED_FROM) {
+    const cudaError_t eb = tridiag_reduce_blocked(c);
+    if (eb != cudaErrorInvalidConfiguration) return eb;    // too large for its shared memory: fall through
+  }
   int C = 1;
   while ((size_t)3 * 8 * trd_cap(n, C) > (size_t)216 * 1024 && C < 4) C *= 2;
   int blocks = (c->num_sms / C) * C;   // one CTA per SM: co-residency is what the cooperative launch checks
@@ -279,11 +286,6 @@ constexpr int QT_LDZ = WY_NB + 4;
 constexpr int QT_RS_MAX = 128;       // row slots per CTA
 constexpr int QT_THREADS = 1024;
 
-__device__ __forceinline__ void dmma_8x8x4(double& d0, double& d1, double a, double b) {
-  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
-               : "+d"(d0), "+d"(d1)
-               : "d"(a), "d"(b));
-}
 
 // S of every block: one CTA per block.
 __global__ void __launch_bounds__(1024)
