@@ -6,19 +6,26 @@
 // Accumulation.  The tensor core adds into its fp32 accumulator with truncation, so a long chain of
 // accumulating MMAs drifts toward zero (measured ~3e-5 relative after the 768 steps of K = 4096).
 // The chain is therefore kept short: one flush = 12 MMA steps (one 64-wide K block with two planes,
-// three with one plane) goes into one of four 128-column accumulators in tensor memory, and the
+// three with one plane) goes into one of two 256-column accumulators in tensor memory, and the
 // worker warps add each finished partial into fp32 registers with round-to-nearest adds.
 //
-// One persistent CTA per SM, 576 threads, output tiles of 128 x 128:
+// Tiles.  An MMA reads its operands from shared memory at (M + N) * 32 bytes per 16-deep step, and
+// the next stage is written into the same memory meanwhile; at 128 x 128 that traffic alone caps the
+// tensor pipe near 60 %.  Output tiles are therefore 128 x 256 (one MMA of N = 256).  The tiles that
+// would form a last, partly filled wave are cut into 128 x 128 halves, so that the wave costs half a
+// tile time instead of a whole one.
+//
+// One persistent CTA per SM, 576 threads:
 //   warp 0       TMA producer: cp.async.bulk.tensor loads of 128B-swizzled K-major tiles into a ring
 //                of shared-memory stages, completion counted by mbarriers;
-//   warp 1       MMA issuer: one elected thread issues tcgen05.mma (M = 128, N = 128, K = 16 per
+//   warp 1       MMA issuer: one elected thread issues tcgen05.mma (M = 128, N = 256 or 128, K = 16 per
 //                instruction) and tcgen05.commit, which releases stages and publishes partials;
-//   warps 2-9    worker group 0, warps 10-17 worker group 1.  The groups take alternate tiles.  A
-//                group drains the partials of its tile (tcgen05.ld, lane = output row; the two
-//                warps of a lane quarter split the 128 columns) and then runs the epilogue from its
-//                registers -- for the ADMM iteration the projection, dual update, residual sums and
-//                the next right-hand side -- while the other group drains the next tile.
+//   warps 2-17   workers: warp w owns tensor-memory lanes 32 (w mod 4) .. +31 (output rows) and 64 of
+//                the 256 columns.  They drain every partial (tcgen05.ld) into 64 register sums per
+//                thread and, when the tile is complete, run the epilogue from those registers -- for the
+//                ADMM iteration the projection, dual update, residual sums and the next right-hand
+//                side -- through a per-warp staging buffer that makes the global accesses coalesced.
+//                The issuer runs up to two flushes into the next tile meanwhile.
 // Every wait is bounded: on expiry the kernel records ADMMQ_ERR_TIMEOUT, stops issuing work, lets
 // copies in flight land, frees tensor memory and returns.
 #include <cuda.h>
@@ -27,11 +34,12 @@
 
 namespace admmq {
 
-constexpr int BM = 128, BN = 128, BK = 64;
-constexpr int NPART = 4;                 // partial accumulators in tensor memory (4 x 128 columns)
-constexpr int GROUP_WARPS = 8;
-constexpr int TC_THREADS = 32 * (2 + 2 * GROUP_WARPS);
-constexpr int COLS_PER_THREAD = BN / 2;  // 64
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int BN_BOX = 128;              // rows of B per TMA box (a tile takes two, a half tile one)
+constexpr int NPART = 2;                 // partial accumulators in tensor memory (2 x 256 columns)
+constexpr int WORKER_WARPS = 16;
+constexpr int TC_THREADS = 32 * (2 + WORKER_WARPS);
+constexpr int COLS_PER_THREAD = BN / 4;  // 64
 constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // about a second
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -135,9 +143,9 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t smem_addr) {
   return d;
 }
 // Instruction descriptor: fp32 accumulate, A and B of the same 16-bit type (format 1 = bf16, 0 = fp16),
-// both K-major, N = 128, M = 128.
-__host__ __device__ constexpr uint32_t idesc_128x128(uint32_t fmt) {
-  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// both K-major, M = 128, N columns.
+__host__ __device__ constexpr uint32_t idesc_m128(uint32_t fmt, uint32_t n_cols) {
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((n_cols >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
 // Tile order.  Consecutive tiles (the ones resident at the same time) form bands of RASTER_M tile rows
@@ -151,6 +159,41 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
   const int in_band = tile - band * RASTER_M * tiles_n;
   tn = in_band / rows;
   tm = first + in_band - tn * rows;
+}
+
+// Work units of the persistent loop: whole 128 x 256 tiles, except that the tiles of a last wave that
+// would fill at most half of the CTAs are cut into two 128 x 128 units.
+struct Schedule {
+  int tiles_m, tiles_n, full_units, num_units;
+};
+__device__ __forceinline__ Schedule make_schedule(int M, int N, int ctas) {
+  Schedule s;
+  s.tiles_m = (M + BM - 1) / BM;
+  s.tiles_n = (N + BN - 1) / BN;
+  const int tiles = s.tiles_m * s.tiles_n;
+  const int waves = tiles / ctas, rem = tiles - waves * ctas;
+  const bool split = rem > 0 && 2 * rem <= ctas;
+  s.full_units = split ? waves * ctas : tiles;
+  s.num_units = split ? waves * ctas + 2 * rem : tiles;
+  return s;
+}
+struct Unit {
+  int tm, col0, ncols;   // first column and width (256 or 128)
+};
+__device__ __forceinline__ Unit unit_of(const Schedule& s, int u) {
+  Unit x;
+  int tile = u, off = 0;
+  x.ncols = BN;
+  if (u >= s.full_units) {
+    const int h = u - s.full_units;
+    tile = s.full_units + (h >> 1);
+    off = (h & 1) * BN_BOX;
+    x.ncols = BN_BOX;
+  }
+  int tn;
+  tile_coords(tile, s.tiles_m, s.tiles_n, x.tm, tn);
+  x.col0 = tn * BN + off;
+  return x;
 }
 
 struct TcMaps {
@@ -227,6 +270,28 @@ __device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, 
   *reinterpret_cast<float4*>(cp) = make_float4(o[0], o[1], o[2], o[3]);
 }
 
+// Asks L2 for the lines the epilogue of (row, [col0, col0 + 64)) will read, a few flushes ahead.
+template <int EPI>
+__device__ __forceinline__ void epilogue_prefetch(const EpiParams& P, int row, int col0, int M, int N) {
+  if (row >= M || col0 + COLS_PER_THREAD > N) return;
+  if (EPI == EPI_ADMM) {
+    const long long o = (long long)row * N + col0;
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(P.Whs + o));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(P.Whs + o + 32));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(P.V + o));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(P.V + o + 32));
+    if (!P.first_iter) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.codes + o));
+  } else if (EPI == EPI_ACCUM) {
+    const float* c = P.C + (long long)row * P.ldc + col0;
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(c));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(c + 32));
+  } else if (EPI == EPI_WOUT) {
+    const float* c = P.Whs + (long long)row * N + col0;
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(c));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(c + 32));
+  }
+}
+
 // The block rows [row0, row0 + 32) x columns [col0, col0 + 64) held by one warp.  All sizes on this path
 // keep N and the leading dimensions multiples of 4, so a group of 4 columns is inside or outside.
 template <int EPI>
@@ -257,18 +322,18 @@ __device__ __forceinline__ void epilogue_block(const EpiParams& P, int row0, int
 // NP: planes per operand (1 or 2).  EPI: epilogue kind (compile-time copy of epi.kind).
 template <int NP, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_t idesc, EpiParams epi,
+gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_t fmt, EpiParams epi,
                int* status) {
-  constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+  constexpr int A_BYTES = BM * BK * 2, BOX_BYTES = BN_BOX * BK * 2, B_BYTES = 2 * BOX_BYTES;
   constexpr int STAGE_BYTES = NP * (A_BYTES + B_BYTES);
-  constexpr int STAGES = (NP == 1) ? 6 : 3;
+  constexpr int STAGES = (NP == 1) ? 4 : 2;
   constexpr int KB_PER_FLUSH = (NP == 1) ? 3 : 1;        // 12 accumulating MMA steps per flush either way
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 2 * NPART + 2];
+  __shared__ __align__(8) uint64_t bars[2 * STAGES + 2 * NPART];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
-  __shared__ float red[2 * GROUP_WARPS * 2];
-  __shared__ __align__(16) float stage_all[2 * GROUP_WARPS * STAGE_FLOATS];
+  __shared__ float red[WORKER_WARPS * 2];
+  __shared__ __align__(16) float stage_all[WORKER_WARPS * STAGE_FLOATS];
 
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -278,7 +343,6 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
   const uint32_t empty0 = smem_u32(&bars[STAGES]);
   const uint32_t pfull0 = smem_u32(&bars[2 * STAGES]);
   const uint32_t pempty0 = smem_u32(&bars[2 * STAGES + NPART]);
-  const uint32_t drained0 = smem_u32(&bars[2 * STAGES + 2 * NPART]);   // [group]: that group has drained a tile
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
@@ -288,9 +352,8 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
     }
     for (int a = 0; a < NPART; ++a) {
       mbar_init(pfull0 + 8 * a, 1);
-      mbar_init(pempty0 + 8 * a, GROUP_WARPS);
+      mbar_init(pempty0 + 8 * a, WORKER_WARPS);
     }
-    for (int a = 0; a < 2; ++a) mbar_init(drained0 + 8 * a, GROUP_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -304,8 +367,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
-  const int tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
-  const int num_tiles = tiles_m * tiles_n;
+  const Schedule sched = make_schedule(M, N, gridDim.x);
   const int num_kb = (K + BK - 1) / BK;
   const int num_flush = (num_kb + KB_PER_FLUSH - 1) / KB_PER_FLUSH;
   const bool lower = (EPI == EPI_ACCUM) && epi.lower_only;
@@ -316,21 +378,23 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        int tm, tn;
-        tile_coords(tile, tiles_m, tiles_n, tm, tn);
-        if (lower && tn * BN > tm * BM + BM - 1) continue;
+      for (int u = blockIdx.x; u < sched.num_units && ok; u += gridDim.x) {
+        const Unit un = unit_of(sched, u);
+        if (lower && un.col0 > un.tm * BM + BM - 1) continue;
+        const int boxes = un.ncols / BN_BOX;
         for (int kb = 0; kb < num_kb; ++kb) {
           ok = mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag, status);
           if (!ok) break;
           const uint32_t sbase = tiles_base + stage * STAGE_BYTES;
           const uint32_t fb = full0 + 8 * stage;
-          mbar_expect_tx(fb, STAGE_BYTES);
+          mbar_expect_tx(fb, NP * (A_BYTES + boxes * BOX_BYTES));
 #pragma unroll
-          for (int pl = 0; pl < NP; ++pl) tma_load_2d(sbase + pl * A_BYTES, &maps.a[pl], fb, kb * BK, tm * BM);
+          for (int pl = 0; pl < NP; ++pl) tma_load_2d(sbase + pl * A_BYTES, &maps.a[pl], fb, kb * BK, un.tm * BM);
 #pragma unroll
           for (int pl = 0; pl < NP; ++pl)
-            tma_load_2d(sbase + NP * A_BYTES + pl * B_BYTES, &maps.b[pl], fb, kb * BK, tn * BN);
+            for (int bx = 0; bx < boxes; ++bx)
+              tma_load_2d(sbase + NP * A_BYTES + pl * B_BYTES + bx * BOX_BYTES, &maps.b[pl], fb, kb * BK,
+                          un.col0 + bx * BN_BOX);
           if (++stage == STAGES) {
             stage = 0;
             phase ^= 1u;
@@ -345,10 +409,10 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
       uint32_t phase = 0;
       uint32_t g = 0;                        // flush counter, shared sequence with the workers
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        int tm, tn;
-        tile_coords(tile, tiles_m, tiles_n, tm, tn);
-        if (lower && tn * BN > tm * BM + BM - 1) continue;
+      for (int u = blockIdx.x; u < sched.num_units && ok; u += gridDim.x) {
+        const Unit un = unit_of(sched, u);
+        if (lower && un.col0 > un.tm * BM + BM - 1) continue;
+        const uint32_t idesc = idesc_m128(fmt, (uint32_t)un.ncols);
         uint32_t d_tmem = 0, accumulate = 0;
         int pb = 0;
         for (int kb = 0; kb < num_kb; ++kb) {
@@ -393,59 +457,51 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
       }
     }
   } else {
-    // ===================== worker groups =====================
-    const int gsel = (warp - 2) / GROUP_WARPS;             // 0 or 1
-    const int wi = (warp - 2) % GROUP_WARPS;
+    // ===================== workers =====================
     const int q = warp & 3;                                // tensor-memory lane quarter this warp may read
-    const int half = wi >> 2;                              // which 64 of the 128 columns
+    const int cq = (warp - 2) >> 2;                        // which 64 of the 256 columns
     float r2 = 0.f, s2 = 0.f;
     uint32_t g = 0;
-    int it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-      int tm, tn;
-        tile_coords(tile, tiles_m, tiles_n, tm, tn);
-      if (lower && tn * BN > tm * BM + BM - 1) continue;
-      if ((it & 1) != gsel) {                              // the other group's tile
-        g += (uint32_t)num_flush;
-        ++it;
-        continue;
-      }
-      // A parity wait cannot tell a phase from the one two completions later, so a group starts
-      // watching the partial barriers only once the other group has drained the tile before this one.
-      if (it > 0) {
-        ok = mbar_wait_warp(drained0 + 8 * (1 - gsel), (uint32_t)((it - 1) >> 1) & 1u, abort_flag, status);
-        if (!ok) break;
-      }
+    for (int u = blockIdx.x; u < sched.num_units && ok; u += gridDim.x) {
+      const Unit un = unit_of(sched, u);
+      if (lower && un.col0 > un.tm * BM + BM - 1) continue;
+      const bool mine = cq * COLS_PER_THREAD < un.ncols;   // a half unit has columns for cq = 0, 1 only
+      const int row0 = un.tm * BM + q * 32, col0 = un.col0 + cq * COLS_PER_THREAD;
+      const int pf_at = num_flush > 6 ? num_flush - 6 : 0;
       float sums[COLS_PER_THREAD];
 #pragma unroll
       for (int e = 0; e < COLS_PER_THREAD; ++e) sums[e] = 0.f;
       for (int f = 0; f < num_flush; ++f) {
+        if (f == pf_at && mine) epilogue_prefetch<EPI>(epi, row0 + lane, col0, M, N);
         const int pb = (int)(g % NPART);
         ok = mbar_wait_warp(pfull0 + 8 * pb, (g / NPART) & 1u, abort_flag, status);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t taddr = tmem_base + (uint32_t)pb * BN + (uint32_t)(half * COLS_PER_THREAD) +
-                               ((uint32_t)(q * 32) << 16);
-        uint32_t v[32];
-        tc_ld32_issue(taddr, v);
-        tc_ld_wait();
+        if (mine) {
+          const uint32_t taddr = tmem_base + (uint32_t)pb * BN + (uint32_t)(cq * COLS_PER_THREAD) +
+                                 ((uint32_t)(q * 32) << 16);
+          uint32_t v[32];
+          tc_ld32_issue(taddr, v);
+          tc_ld_wait();
 #pragma unroll
-        for (int e = 0; e < 32; ++e) sums[e] += __uint_as_float(v[e]);
-        tc_ld32_issue(taddr + 32, v);
-        tc_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(pempty0 + 8 * pb);      // the partial is in registers: buffer free
+          for (int e = 0; e < 32; ++e) sums[e] += __uint_as_float(v[e]);
+          tc_ld32_issue(taddr + 32, v);
+          tc_ld_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(pempty0 + 8 * pb);    // the partial is in registers: buffer free
 #pragma unroll
-        for (int e = 0; e < 32; ++e) sums[32 + e] += __uint_as_float(v[e]);
+          for (int e = 0; e < 32; ++e) sums[32 + e] += __uint_as_float(v[e]);
+        } else {
+          tc_fence_before();
+          if (lane == 0) mbar_arrive(pempty0 + 8 * pb);
+        }
         ++g;
       }
       if (!ok) break;
-      if (lane == 0) mbar_arrive(drained0 + 8 * gsel);
-      epilogue_block<EPI>(epi, tm * BM + q * 32, tn * BN + half * COLS_PER_THREAD, M, N, sums,
-                          stage_all + (warp - 2) * STAGE_FLOATS, lane, r2, s2);
-      ++it;
+      if (mine)
+        epilogue_block<EPI>(epi, row0, col0, M, N, sums, stage_all + (warp - 2) * STAGE_FLOATS, lane, r2, s2);
     }
     if (EPI == EPI_ADMM) {
       r2 = warp_sum(r2);
@@ -466,7 +522,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
   }
   if (EPI == EPI_ADMM && threadIdx.x == 0) {
     float a = 0.f, b = 0.f;                  // fixed order over the worker warps
-    for (int w = 0; w < 2 * GROUP_WARPS; ++w) {
+    for (int w = 0; w < WORKER_WARPS; ++w) {
       a += red[2 * w];
       b += red[2 * w + 1];
     }
@@ -516,10 +572,10 @@ static bool encode_plane(CUtensorMap* map, const bf16* ptr, long long rows, long
 int gemm_tc_partial_slots(int num_sms) { return num_sms; }
 
 template <int NP, int EPI>
-static cudaError_t launch_tc(Ctx* c, const TcMaps& maps, int M, int N, int K, uint32_t idesc,
+static cudaError_t launch_tc(Ctx* c, const TcMaps& maps, int M, int N, int K, uint32_t fmt,
                              const EpiParams& epi) {
   constexpr int STAGE_BYTES = NP * (BM * BK * 2 + BN * BK * 2);
-  constexpr int STAGES = (NP == 1) ? 6 : 3;
+  constexpr int STAGES = (NP == 1) ? 4 : 2;
   const size_t smem = (size_t)STAGES * STAGE_BYTES + 1024;
   static bool attr_set = false;
   if (!attr_set) {
@@ -530,7 +586,7 @@ static cudaError_t launch_tc(Ctx* c, const TcMaps& maps, int M, int N, int K, ui
   }
   const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = tiles < c->num_sms ? tiles : c->num_sms;
-  gemm_tc_kernel<NP, EPI><<<grid, TC_THREADS, smem, c->stream>>>(maps, M, N, K, idesc, epi, c->status);
+  gemm_tc_kernel<NP, EPI><<<grid, TC_THREADS, smem, c->stream>>>(maps, M, N, K, fmt, epi, c->status);
   c->launches++;
   return cudaGetLastError();
 }
@@ -541,17 +597,17 @@ cudaError_t gemm_tc(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiPa
   if ((A.ld & 7) || (B.ld & 7)) return cudaErrorInvalidValue;
   TcMaps maps;
   bool ok = encode_plane(&maps.a[0], A.hi, M, K, A.ld, BM, A.f16) &&
-            encode_plane(&maps.b[0], B.hi, N, K, B.ld, BN, B.f16);
+            encode_plane(&maps.b[0], B.hi, N, K, B.ld, BN_BOX, B.f16);
   if (na == 2) ok = ok && encode_plane(&maps.a[1], A.lo, M, K, A.ld, BM, A.f16);
   else maps.a[1] = maps.a[0];
-  if (nb == 2) ok = ok && encode_plane(&maps.b[1], B.lo, N, K, B.ld, BN, B.f16);
+  if (nb == 2) ok = ok && encode_plane(&maps.b[1], B.lo, N, K, B.ld, BN_BOX, B.f16);
   else maps.b[1] = maps.b[0];
   if (!ok) return cudaErrorInvalidValue;
   EpiParams epi = epi_in;
   epi.row_inv = A.row_inv;
   epi.a_inv = A.all_inv;
   epi.b_inv = B.all_inv;
-  const uint32_t idesc = idesc_128x128(A.f16 ? 0u : 1u);
+  const uint32_t idesc = A.f16 ? 0u : 1u;                  // operand format: 0 = fp16, 1 = bf16
   if (na == 1) {
     if (epi.kind == EPI_ACCUM) return launch_tc<1, EPI_ACCUM>(c, maps, M, N, K, idesc, epi);
     if (epi.kind == EPI_STORE) return launch_tc<1, EPI_STORE>(c, maps, M, N, K, idesc, epi);
