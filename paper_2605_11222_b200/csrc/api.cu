@@ -62,6 +62,7 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   c.H_raw = cv.take<float>(nn);
   c.H = cv.take<float>(nn);
   c.s = cv.take<float>(n);
+  c.inv_s = cv.take<float>(n);
   c.hdiag = cv.take<float>(n);
   c.A64 = cv.take<double>(nn);
   c.P64 = cv.take<double>(nn);
@@ -394,6 +395,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.V = c->V;
   e.codes = d_codes;
   e.s = c->s;
+  e.inv_s = c->inv_s;
   e.delta = d_scale;
   e.zero = d_zero;
   e.group_size = gs;

@@ -72,8 +72,8 @@ __global__ void diag_sum_kernel(const float* __restrict__ Hraw, int n, double in
 
 __global__ void finalize_diag_kernel(const float* __restrict__ Hraw, int n, double inv_N,
                                      double damp_frac, int precondition, const double* __restrict__ dsum,
-                                     float* __restrict__ hdiag, float* __restrict__ s, double* s64,
-                                     int* status) {
+                                     float* __restrict__ hdiag, float* __restrict__ s,
+                                     float* __restrict__ inv_s, double* s64, int* status) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const double lam = damp_frac * dsum[0] / n;
@@ -82,12 +82,14 @@ __global__ void finalize_diag_kernel(const float* __restrict__ Hraw, int n, doub
   if (!(hii > 0.f) || !isfinite(hii)) {
     raise_status(status, isfinite(hii) ? ST_NOT_SPD : ST_NONFINITE);
     s[i] = 1.f;
+    inv_s[i] = 1.f;
     s64[i] = 1.0;
     return;
   }
   const double sv = precondition ? sqrt((double)hii) : 1.0;
   s64[i] = sv;
   s[i] = (float)sv;
+  inv_s[i] = (float)(1.0 / sv);
 }
 
 __global__ void finalize_full_kernel(const float* __restrict__ Hraw, int n, double inv_N,
@@ -112,7 +114,7 @@ void launch_finalize(Ctx* c, double damp_frac, int precondition) {
   LAUNCH(c);
   finalize_diag_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(c->H_raw, n, inv_N, damp_frac,
                                                               precondition, c->scal, c->hdiag, c->s,
-                                                              s64, c->status);
+                                                              c->inv_s, s64, c->status);
   LAUNCH(c);
   dim3 grid((n + 255) / 256, n);
   finalize_full_kernel<<<grid, 256, 0, c->stream>>>(c->H_raw, n, inv_N, c->hdiag, s64, c->H, c->A64,

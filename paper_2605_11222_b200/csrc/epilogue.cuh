@@ -23,6 +23,7 @@ struct EpiParams {
   float* V;                 // dual V (in/out)
   unsigned char* codes;     // codes of D (in: D^(t), out: D^(t+1))
   const float* s;           // [n] s_i = sqrt(H_ii)
+  const float* inv_s;       // [n] 1 / s_i
   const float* delta;       // [p][n_groups]
   const float* zero;        // [p][n_groups]
   int group_size, n_groups;
@@ -52,13 +53,16 @@ struct AdmmElem {
   unsigned char code;
   float v_new, r_next, dr2, ds2;
 };
-__device__ __forceinline__ AdmmElem admm_elem(float z, float wh, float v, int code_old, float s,
-                                              float dl, float z0, const EpiParams& P) {
+// The two divisions of the projection are taken as products with 1 / s_i and 1 / Delta (each correctly
+// rounded): the epilogue runs on the critical path of every tile, and a full-precision division costs as
+// much as the rest of the element.
+__device__ __forceinline__ AdmmElem admm_elem(float z, float wh, float v, int code_old, float s, float inv_s,
+                                              float dl, float inv_dl, float z0, const EpiParams& P) {
   AdmmElem o;
   const float w = wh + z;                                  // W^(t+1)
-  const float wt = w + v * P.inv_rho;                      // target W~ = W + V/rho          (Eq. 8)
-  const float y = wt / s;                                  // unscaled coordinate Sigma W~
-  float k = rintf((y - z0) / dl);                          // nearest level, ties to even    (Eq. 10)
+  const float wt = fmaf(v, P.inv_rho, w);                  // target W~ = W + V/rho          (Eq. 8)
+  const float y = wt * inv_s;                              // unscaled coordinate Sigma W~
+  float k = rintf((y - z0) * inv_dl);                      // nearest level, ties to even    (Eq. 10)
   k = fminf(fmaxf(k, 0.0f), (float)P.kmax);
   const float d_new = s * (z0 + dl * k);                   // D^(t+1), scaled coordinates
   const float d_old = P.first_iter ? wh : s * (z0 + dl * (float)code_old);
@@ -88,7 +92,7 @@ __device__ __forceinline__ void epi_scalar(const EpiParams& P, int row, int col,
     const float dl = P.delta[(long long)row * P.n_groups + g];
     const float z0 = P.zero[(long long)row * P.n_groups + g];
     AdmmElem e = admm_elem(acc, P.Whs[idx], P.V[idx], P.first_iter ? 0 : (int)P.codes[idx], P.s[col],
-                           dl, z0, P);
+                           P.inv_s[col], dl, __frcp_rn(dl), z0, P);
     P.codes[idx] = e.code;
     P.V[idx] = e.v_new;
     P.Rnext[idx] = e.r_next;

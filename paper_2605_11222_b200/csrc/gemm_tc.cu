@@ -221,14 +221,17 @@ __device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, 
     const float4 w = *reinterpret_cast<const float4*>(P.Whs + o);
     const float4 v = *reinterpret_cast<const float4*>(P.V + o);
     const float4 s = *reinterpret_cast<const float4*>(P.s + col);
+    const float4 is = *reinterpret_cast<const float4*>(P.inv_s + col);
     uint32_t codes = 0u;
     if (!P.first_iter) codes = *reinterpret_cast<const uint32_t*>(P.codes + o);
     const float wh[4] = {w.x, w.y, w.z, w.w};
     const float vv[4] = {v.x, v.y, v.z, v.w};
     const float ss[4] = {s.x, s.y, s.z, s.w};
+    const float si[4] = {is.x, is.y, is.z, is.w};
     const bool one_group = (P.group_size & 3) == 0;        // then the 4 columns share (Delta, z0)
     long long gi = (long long)row * P.n_groups + col / P.group_size;
     float dl = P.delta[gi], z0 = P.zero[gi];
+    float inv_dl = __frcp_rn(dl);
     float vn[4], rn[4];
     uint32_t cn = 0u;
 #pragma unroll
@@ -237,9 +240,10 @@ __device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, 
         gi = (long long)row * P.n_groups + (col + e) / P.group_size;
         dl = P.delta[gi];
         z0 = P.zero[gi];
+        inv_dl = __frcp_rn(dl);
       }
       const int code_old = (int)((codes >> (8 * e)) & 0xffu);
-      AdmmElem r = admm_elem(a[e], wh[e], vv[e], code_old, ss[e], dl, z0, P);
+      AdmmElem r = admm_elem(a[e], wh[e], vv[e], code_old, ss[e], si[e], dl, inv_dl, z0, P);
       vn[e] = r.v_new;
       cn |= (uint32_t)r.code << (8 * e);
       rn[e] = r.r_next;

@@ -44,6 +44,7 @@ struct Ctx {
   float* H_raw = nullptr;       // [n][n] fp32 accumulator of X^T X (lower triangle valid until finalize)
   float* H = nullptr;           // [n][n] fp32 damped, unscaled
   float* s = nullptr;           // [n]
+  float* inv_s = nullptr;       // [n] 1 / s_i
   float* hdiag = nullptr;       // [n] diag of damped H
   double* A64 = nullptr;        // [n][n] fp64 working copy of H~, reflectors afterwards
   double* P64 = nullptr;        // [n][n] fp64 Q^T
