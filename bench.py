@@ -166,6 +166,60 @@ def run_reference(args, spec, wl):
 
 
 # ---------------------------------------------------------------------------------------------------
+def run_stack(args, wl):
+    """Config 5: every linear layer of the first B decoder blocks, each quantized once from its own seeded
+    calibration set (generated on the device, generation timed separately)."""
+    from paper_2605_11222_b200 import binding as B
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    layers = wl.config5(n_blocks=args.stack_blocks)
+    if args.tokens > 0:
+        import dataclasses
+        layers = [dataclasses.replace(l, n_tokens=args.tokens) for l in layers]
+    T = layers[0].T
+    solvers = {}
+    for n in sorted({l.d_in for l in layers}):
+        solvers[n] = B.Solver(n, max(l.d_out for l in layers if l.d_in == n), T_max=T, device=dev)
+    per_shape, gen_s, solve_ms, moves = {}, 0.0, 0.0, 0
+    torch.cuda.synchronize(dev)
+    t_wall = time.perf_counter()
+    for spec in layers:
+        sol = solvers[spec.d_in]
+        t0 = time.perf_counter()
+        W = wl.gen_weight(spec, dev)
+        Xs = [wl.gen_x_chunk(spec, c, dev) for c in range(spec.n_chunks)]
+        torch.cuda.synchronize(dev)
+        gen_s += time.perf_counter() - t0
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        sol.hessian_reset()
+        for x in Xs:
+            sol.hessian_accumulate(x)
+        sol.factor(rho=spec.rho())
+        codes, scale, zero, _ = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, report=False)
+        rep, st = sol.local_search(W, spec.bits, spec.group_size, codes, scale, zero, report=True)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1)
+        solve_ms += ms
+        moves += rep.moves
+        key = f"{spec.d_in}x{spec.d_out}"
+        a = per_shape.setdefault(key, [0, 0.0])
+        a[0] += 1
+        a[1] += ms
+        del Xs, W
+    wall = time.perf_counter() - t_wall
+    print(json.dumps({
+        "metric": "admmq_stack_solve_time", "value": solve_ms / 1e3, "unit": "s", "n_gpus": 1,
+        "higher_is_better": False, "data": "synthetic", "dtype": "f16x2-split (fp32 accumulate)",
+        "config": {"workload": f"cfg5 first {args.stack_blocks} of 36 blocks", "layers": len(layers),
+                   "n_tokens": layers[0].n_tokens, "T": T, "bits": layers[0].bits, "group_size": layers[0].group_size},
+        "wall_s_with_generation": wall, "generation_s": gen_s, "local_search_moves": moves,
+        "per_shape": {k: {"layers": v[0], "s_per_layer": v[1] / v[0] / 1e3} for k, v in per_shape.items()}}))
+    return 0
+
+
+# ---------------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -176,6 +230,9 @@ def main():
     ap.add_argument("--workload", default="cfg2", help="cfg1 | cfg2 | cfg3_gate | cfg3_up | cfg3_down | "
                     "cfg4_k | cfg4_v | cfg4_o | cfg5_<q|k|v|o|gate|up|down>  (default: the metric's own, cfg2)")
     ap.add_argument("--iters", type=int, default=0, help="ADMM iterations T (0: the workload's own, 300)")
+    ap.add_argument("--stack-blocks", type=int, default=0,
+                    help="instead of one layer: quantize the first B decoder blocks of config 5 (7 layers each, "
+                         "36 = the whole stack), every layer once, and report the wall time")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -195,6 +252,8 @@ def main():
 
     if args.impl == "reference":
         return run_reference(args, spec, wl)
+    if args.stack_blocks > 0:
+        return run_stack(args, wl)
 
     from paper_2605_11222_b200 import binding as B, sharding
     import torch.distributed as dist
