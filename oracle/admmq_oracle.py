@@ -302,6 +302,96 @@ def local_search(H: np.ndarray, W_hat: np.ndarray, codes: np.ndarray, delta: np.
 
 
 # --------------------------------------------------------------------------
+# Pair-swap local search (Sec. 3.5 "Algorithm"; Eq. 11 in full)
+# --------------------------------------------------------------------------
+@dataclasses.dataclass
+class PairSwapResult:
+    codes: np.ndarray
+    Wq: np.ndarray
+    g: np.ndarray            # maintained gradient H (W_q - W_hat), [p, n]
+    chosen: list             # per round: index of the applied pair in that round's batch, or -1
+    totals: list             # per round: total loss change of the applied pair (0 if none)
+    moves: int               # (pair, column) moves applied
+
+
+PAIR_SIGNS = ((1.0, 1.0), (1.0, -1.0), (-1.0, 1.0), (-1.0, -1.0))
+
+
+def pair_move_costs(g1, g2, h11, h22, h12, d1, d2):
+    """Eq. 11 for the four sign combinations, with g = H (W_q - W_hat) = -G:
+      c = 2 a d1 g1 + d1^2 H11 + 2 b d2 g2 + d2^2 H22 + 2 a b d1 d2 H12,  (a, b) in PAIR_SIGNS.
+    Arrays broadcast; returns an array with a leading axis of length 4."""
+    out = []
+    for a, b in PAIR_SIGNS:
+        out.append(2.0 * a * d1 * g1 + d1 * d1 * h11 + 2.0 * b * d2 * g2 + d2 * d2 * h22
+                   + 2.0 * a * b * d1 * d2 * h12)
+    return np.stack(out)
+
+
+def pair_swap(H: np.ndarray, W_hat: np.ndarray, codes: np.ndarray, delta: np.ndarray, z0: np.ndarray,
+              bits: int, pairs: np.ndarray, tau: float = 1e-6) -> PairSwapResult:
+    """The paper's pair-swap refinement.  `pairs` is [rounds, batch, 2]: the row pairs sampled for every
+    round (the random draws are an input).  Each round: for every candidate pair (i1, i2), i1 != i2, and
+    every output column independently, the best of the four sign combinations that keep both codes in
+    [0, 2^b - 1] is found by Eq. 11; a column takes part only if that cost is below
+    -tau (d1^2 H11 + d2^2 H22); the pair's total is the sum of the participating columns' costs.  The pair
+    with the smallest total is applied in all participating columns (ties: first in the batch; nothing is
+    applied when no total is negative) and the gradient takes the rank-2 correction
+    g_j += d1 H[:, i1] + d2 H[:, i2].  H is the unscaled damped Hessian.
+    Readings: one pair applied per round (the paper's step (iv)); a column may decline; sign combinations
+    are tried in the order (+,+), (+,-), (-,+), (-,-) and the first minimum wins."""
+    H = np.asarray(H, dtype=F64)
+    W_hat = np.asarray(W_hat, dtype=F64)
+    p, n = codes.shape
+    kmax = (1 << bits) - 1
+    dl = _expand(delta, n)
+    k = codes.astype(np.int64).copy()
+    Wq = dequantize(codes, delta, z0)
+    g = (Wq - W_hat) @ H
+    chosen, totals, moves = [], [], 0
+
+    def evaluate(i1, i2):
+        d1, d2 = dl[:, i1], dl[:, i2]
+        c = pair_move_costs(g[:, i1], g[:, i2], H[i1, i1], H[i2, i2], H[i1, i2], d1, d2)   # [4, p]
+        for q, (a, b) in enumerate(PAIR_SIGNS):
+            ok = (k[:, i1] + a >= 0) & (k[:, i1] + a <= kmax) & (k[:, i2] + b >= 0) & (k[:, i2] + b <= kmax)
+            c[q] = np.where(ok, c[q], np.inf)
+        q_best = np.argmin(c, axis=0)
+        c_best = c[q_best, np.arange(p)]
+        take = c_best < -tau * (d1 * d1 * H[i1, i1] + d2 * d2 * H[i2, i2])
+        return q_best, c_best, take
+
+    for batch in np.asarray(pairs):
+        best_t, best_b = 0.0, -1
+        for b_idx, (i1, i2) in enumerate(batch):
+            i1, i2 = int(i1), int(i2)
+            if i1 == i2:
+                continue
+            _, c_best, take = evaluate(i1, i2)
+            t = float(np.sum(np.where(take, c_best, 0.0)))
+            if t < best_t:
+                best_t, best_b = t, b_idx
+        chosen.append(best_b)
+        totals.append(best_t)
+        if best_b < 0:
+            continue
+        i1, i2 = int(batch[best_b][0]), int(batch[best_b][1])
+        q_best, _, take = evaluate(i1, i2)
+        sa = np.array([s[0] for s in PAIR_SIGNS])[q_best]
+        sb = np.array([s[1] for s in PAIR_SIGNS])[q_best]
+        cols = np.nonzero(take)[0]
+        da = sa[cols] * dl[cols, i1]
+        db = sb[cols] * dl[cols, i2]
+        k[cols, i1] += sa[cols].astype(np.int64)
+        k[cols, i2] += sb[cols].astype(np.int64)
+        Wq[cols, i1] += da
+        Wq[cols, i2] += db
+        g[cols] += da[:, None] * H[i1, :][None, :] + db[:, None] * H[i2, :][None, :]
+        moves += int(cols.size)
+    return PairSwapResult(k.astype(np.uint8), Wq, g, chosen, totals, moves)
+
+
+# --------------------------------------------------------------------------
 # Whole layer: Algorithm 1
 # --------------------------------------------------------------------------
 @dataclasses.dataclass

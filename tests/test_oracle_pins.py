@@ -348,3 +348,95 @@ def test_local_search_respects_move_cap_and_bounds():
     full = O.local_search(H, W, codes, delta, z0, 2)
     assert full.codes.max() <= 3 and not full.capped.any()
     assert O.objective(H, W, full.Wq) < O.objective(H, W, O.dequantize(codes, delta, z0))
+
+
+# ------------------------------------------------------------------ pair-swap local search (Sec. 3.5, Eq. 11 in full)
+def _pair_case(seed, n=10, p=6, bits=2):
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((40, n))
+    X[:, 1] = 0.9 * X[:, 0] + 0.1 * X[:, 1]              # correlated channels: cross terms matter
+    H = O.hessian_finalize(X.T @ X, 40)
+    W = 0.02 * rng.standard_normal((p, n))
+    delta, z0 = O.grid_fit(W, bits, 0, False)
+    codes = O.project(W, np.ones(n), delta, z0, bits)[0]
+    return H, W, delta, z0, codes
+
+
+def test_pair_cost_closed_form_equals_recomputed_loss():
+    """Eq. 11: the closed-form change of eps^T H eps for every sign combination."""
+    H, W, delta, z0, codes = _pair_case(3)
+    Wq = O.dequantize(codes, delta, z0)
+    g = (Wq - W) @ H
+    j, i1, i2 = 2, 0, 1
+    d = delta[j, 0]
+    c = O.pair_move_costs(g[j, i1], g[j, i2], H[i1, i1], H[i2, i2], H[i1, i2], d, d)
+    e0 = Wq[j] - W[j]
+    for q, (a, b) in enumerate(O.PAIR_SIGNS):
+        e1 = e0.copy()
+        e1[i1] += a * d
+        e1[i2] += b * d
+        assert abs((e1 @ H @ e1 - e0 @ H @ e0) - c[q]) <= 1e-12 * abs(e0 @ H @ e0)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_pair_swap_brute_force_choice_and_invariants(seed):
+    """One round over ALL row pairs: the applied pair and every column's sign combination are the best ones
+    by direct evaluation of the loss; codes stay in range; the maintained gradient stays exact."""
+    bits = 2
+    H, W, delta, z0, codes0 = _pair_case(seed, bits=bits)
+    p, n = codes0.shape
+    codes = O.local_search(H, W, codes0, delta, z0, bits).codes          # start from a 1-move optimum
+    pairs = np.array([[(a, b) for a in range(n) for b in range(a + 1, n)]])
+    res = O.pair_swap(H, W, codes, delta, z0, bits, pairs)
+    # brute force: total improvement of every pair, every column choosing freely among the 4 combos or none
+    Wq = O.dequantize(codes, delta, z0)
+    base = np.einsum("jn,nm,jm->j", Wq - W, H, Wq - W)
+    best_total, best_pair = 0.0, -1
+    for b, (i1, i2) in enumerate(pairs[0]):
+        tot = 0.0
+        for j in range(p):
+            best = 0.0
+            for a, s2 in O.PAIR_SIGNS:
+                k1, k2 = codes[j, i1] + a, codes[j, i2] + s2
+                if 0 <= k1 <= 3 and 0 <= k2 <= 3:
+                    e = Wq[j] - W[j]
+                    e = e.copy()
+                    e[i1] += a * delta[j, 0]
+                    e[i2] += s2 * delta[j, 0]
+                    best = min(best, e @ H @ e - base[j])
+            tot += best
+        if tot < best_total - 1e-15:
+            best_total, best_pair = tot, b
+    assert res.chosen[0] == best_pair
+    if best_pair >= 0:
+        assert abs(res.totals[0] - best_total) <= 1e-9 * abs(best_total)
+        assert abs((O.objective(H, W, res.Wq) - base.sum()) - best_total) <= 1e-9 * abs(base.sum())
+        i1, i2 = pairs[0][best_pair]
+        changed = np.nonzero((res.codes != codes).any(axis=1))[0]
+        assert res.moves == changed.size
+        assert set(np.nonzero((res.codes != codes).any(axis=0))[0]) <= {i1, i2}
+    assert res.codes.max() <= 3
+    assert np.allclose(res.g, (res.Wq - W) @ H, rtol=0, atol=1e-12 * np.abs(res.g).max())
+    assert np.allclose(res.Wq, O.dequantize(res.codes, delta, z0), rtol=0, atol=1e-15)
+
+
+def test_pair_swap_monotone_and_diagonal_hessian_declines():
+    bits = 3
+    H, W, delta, z0, codes0 = _pair_case(5, n=16, p=12, bits=bits)
+    codes = O.local_search(H, W, codes0, delta, z0, bits).codes
+    rng = np.random.default_rng(1)
+    pairs = rng.integers(0, 16, size=(5, 40, 2))
+    res = O.pair_swap(H, W, codes, delta, z0, bits, pairs)
+    errs = [O.objective(H, W, O.dequantize(codes, delta, z0))]
+    c = codes
+    for r in range(5):                                            # round by round: never increases
+        c = O.pair_swap(H, W, c, delta, z0, bits, pairs[r:r + 1]).codes
+        errs.append(O.objective(H, W, O.dequantize(c, delta, z0)))
+    assert all(b <= a * (1 + 1e-12) for a, b in zip(errs, errs[1:]))
+    assert np.array_equal(c, res.codes)
+    assert all(t <= 0 for t in res.totals)
+    # separable problem: the 1-move optimum is the nearest grid point and no pair move can improve it
+    Hd = np.diag(np.diag(H))
+    cd = O.local_search(Hd, W, codes0, delta, z0, bits).codes
+    rd = O.pair_swap(Hd, W, cd, delta, z0, bits, pairs)
+    assert rd.moves == 0 and rd.chosen == [-1] * 5 and np.array_equal(rd.codes, cd)
