@@ -171,6 +171,32 @@ admmq_status admmq_local_search(admmq_ctx* ctx, const float* d_W0, int d_out, co
                                 unsigned char* d_codes, const float* d_scale, const float* d_zero,
                                 float* d_Wq, admmq_report* h_report);
 
+/* ---- Pair-swap refinement (Sec. 3.5 "Algorithm"; Eq. 11 with both perturbations). --------------------
+ * cfg->d_pairs: DEVICE array [rounds][batch][2] of row indices in [0, d_in): the candidate row pairs of
+ * every round, drawn by the caller (entries with equal or out-of-range indices are ignored).  Per round,
+ * with g = H (W_q - W_hat): for a pair (i1, i2) every output channel finds the best of the four sign
+ * combinations d1 = +-Delta, d2 = +-Delta that keep both codes in range,
+ *   c = 2 d1 g_i1 + d1^2 H_i1i1 + 2 d2 g_i2 + d2^2 H_i2i2 + 2 d1 d2 H_i1i2
+ * (order (+,+), (+,-), (-,+), (-,-), first minimum), and takes part if
+ * c < -accept_tol (d1^2 H_i1i1 + d2^2 H_i2i2).  The pair with the smallest sum of c over the channels that
+ * take part (first in the batch on ties; none if no sum is negative) is applied in those channels, then
+ * g += d1 H[:, i1] + d2 H[:, i2].  One pair per round, as the paper's step (iv); the paper runs at most 5
+ * rounds.  Codes (and d_Wq if non-NULL) are updated in place.  Usually called after admmq_local_search.
+ * Report: err_before / err_after as for local search, moves = (pair, channel) moves applied, iters_run =
+ * rounds in which a pair was applied. */
+typedef struct {
+  size_t struct_size;           /* sizeof(admmq_pairswap_cfg) */
+  int bits;
+  int group_size;
+  int rounds;                   /* >= 0 */
+  int batch;                    /* candidate pairs per round, 0..65536 */
+  const int* d_pairs;           /* device, [rounds][batch][2] */
+  double accept_tol;            /* relative threshold tau, 1e-6 by default */
+} admmq_pairswap_cfg;
+admmq_status admmq_pair_swap(admmq_ctx* ctx, const float* d_W0, int d_out, const admmq_pairswap_cfg* cfg,
+                             unsigned char* d_codes, const float* d_scale, const float* d_zero,
+                             float* d_Wq, admmq_report* h_report);
+
 /* Tr(E^T H E) with E = (z0 + Delta k) - W_hat and the unscaled damped H (Eq. 2 without the 1/2, as in
  * Sec. 3.5).  Synchronises; the value is written to *h_err (host). */
 admmq_status admmq_objective(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,

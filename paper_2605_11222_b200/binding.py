@@ -27,7 +27,7 @@ EXPORTS = [
     "admmq_hessian_accumulate", "admmq_hessian_set", "admmq_factor", "admmq_quantize_layer",
     "admmq_w_update", "admmq_local_search", "admmq_objective", "admmq_get_hessian",
     "admmq_launch_count", "admmq_set_timing", "admmq_reset_timing", "admmq_get_timing",
-    "admmq_objective_static", "admmq_get_factor",
+    "admmq_objective_static", "admmq_get_factor", "admmq_pair_swap",
 ]
 T_HESSIAN_PRODUCT, T_TRANSPOSE, T_FACTOR, T_WUPDATE_PRODUCT1, T_TRIDIAG_SOLVE, T_WUPDATE_PRODUCT2, \
     T_GRADIENT_PRODUCT, T_LOCAL_SEARCH, T_ROW_SPLIT = range(9)
@@ -49,6 +49,11 @@ class QuantCfg(C.Structure):
 class LsCfg(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("bits", C.c_int), ("group_size", C.c_int),
                 ("max_moves_per_col", C.c_longlong), ("accept_tol", C.c_double)]
+
+
+class PairSwapCfg(C.Structure):
+    _fields_ = [("struct_size", C.c_size_t), ("bits", C.c_int), ("group_size", C.c_int), ("rounds", C.c_int),
+                ("batch", C.c_int), ("d_pairs", C.c_void_p), ("accept_tol", C.c_double)]
 
 
 class Report(C.Structure):
@@ -94,6 +99,7 @@ def load_library(path: Optional[str] = None):
     lib.admmq_w_update.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, cd, vp]
     lib.admmq_local_search.argtypes = [vp, vp, ci, C.POINTER(LsCfg), vp, vp, vp, vp, C.POINTER(Report)]
     lib.admmq_objective.argtypes = [vp, vp, ci, ci, vp, vp, vp, C.POINTER(cd)]
+    lib.admmq_pair_swap.argtypes = [vp, vp, ci, C.POINTER(PairSwapCfg), vp, vp, vp, vp, C.POINTER(Report)]
     lib.admmq_get_hessian.argtypes = [vp, vp, vp]
     lib.admmq_get_factor.argtypes = [vp, vp, vp, vp]
     lib.admmq_set_timing.argtypes = [vp, ci]
@@ -230,6 +236,18 @@ class Solver:
         st = self.lib.admmq_local_search(self.h, _ptr(W0), W0.shape[0], C.byref(cfg), _ptr(codes),
                                          _ptr(scale), _ptr(zero), _ptr(Wq), C.byref(rep) if report else None)
         _check(st, "admmq_local_search", allow=(OK, WARN_MOVE_CAP))
+        return (rep if report else None), st
+
+    def pair_swap(self, W0, bits, group_size, codes, scale, zero, pairs, Wq=None, accept_tol: float = 1e-6,
+                  report: bool = True):
+        """pairs: int32 device tensor [rounds, batch, 2] of candidate row pairs (the caller's random draws)."""
+        assert pairs.dtype == torch.int32 and pairs.dim() == 3 and pairs.shape[2] == 2
+        cfg = PairSwapCfg(C.sizeof(PairSwapCfg), bits, group_size, pairs.shape[0], pairs.shape[1],
+                          pairs.data_ptr() if pairs.numel() else None, accept_tol)
+        rep = Report()
+        st = self.lib.admmq_pair_swap(self.h, _ptr(W0), W0.shape[0], C.byref(cfg), _ptr(codes), _ptr(scale),
+                                      _ptr(zero), _ptr(Wq), C.byref(rep) if report else None)
+        _check(st, "admmq_pair_swap")
         return (rep if report else None), st
 
     def objective(self, W0, group_size, codes, scale, zero) -> float:

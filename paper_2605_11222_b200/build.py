@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libadmmq.so")
-SOURCES = ["api.cu", "elem.cu", "gemm_simt.cu", "gemm_tc.cu", "tridiag.cu", "tridiag_blocked.cu", "local_search.cu",
+SOURCES = ["api.cu", "elem.cu", "gemm_simt.cu", "gemm_tc.cu", "tridiag.cu", "tridiag_blocked.cu", "local_search.cu", "pair_swap.cu",
            "objective_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]

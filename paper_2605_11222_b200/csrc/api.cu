@@ -72,6 +72,9 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   c.pvec = cv.take<double>(n);
   c.stage_l = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
   c.stage_invd = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
+  c.ps_totals = cv.take<double>(PAIR_BATCH_MAX);
+  c.ps_chosen = cv.take<int>(16);
+  c.ps_d = cv.take<float>((size_t)2 * p);
   c.trd_ws = cv.take<double>(tridiag_blocked_scratch_doubles(n));
   c.wy_s = cv.take<double>((size_t)((n + 31) / 32) * 1024);
   c.Q_hi = cv.take<bf16>(nn);
@@ -509,6 +512,54 @@ admmq_status admmq_local_search(admmq_ctx* ctx, const float* d_W0, int d_out, co
   h_report->moves = moves;
   h_report->capped_columns = capped;
   if (st == ADMMQ_OK && capped > 0) st = ADMMQ_WARN_MOVE_CAP;
+  return st;
+}
+
+admmq_status admmq_pair_swap(admmq_ctx* ctx, const float* d_W0, int d_out, const admmq_pairswap_cfg* cfg,
+                             unsigned char* d_codes, const float* d_scale, const float* d_zero, float* d_Wq,
+                             admmq_report* h_report) {
+  if (!cfg || cfg->struct_size != sizeof(admmq_pairswap_cfg)) return ADMMQ_ERR_INVALID_ARG;
+  admmq_status st = check_layer_args(ctx, d_W0, d_out, cfg->bits, cfg->group_size, d_codes, d_scale, d_zero);
+  if (st != ADMMQ_OK) return st;
+  if (d_Wq && !aligned16(d_Wq)) return ADMMQ_ERR_INVALID_ARG;
+  if (cfg->rounds < 0 || cfg->batch < 0 || !(cfg->accept_tol >= 0.0)) return ADMMQ_ERR_INVALID_ARG;
+  if (cfg->batch > PAIR_BATCH_MAX) return ADMMQ_ERR_SHAPE;
+  if (cfg->rounds > 0 && cfg->batch > 0 && (!cfg->d_pairs || !aligned16(cfg->d_pairs))) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  const int n = c->n, p = d_out, gs = group_of(n, cfg->group_size);
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  if (h_report) {
+    if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return ADMMQ_ERR_CUDA;
+    cudaEventRecord(ev0, c->stream);
+  }
+  if (gradient(ctx, d_W0, p, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  if (h_report) launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 1);
+  launch_zero(c, ctx->d_moves, 64);
+  launch_zero(c, ctx->d_capped, 64);
+  for (int r = 0; r < cfg->rounds && cfg->batch > 0; ++r)
+    if (launch_pair_round(c, p, cfg->bits, gs, (float)cfg->accept_tol, d_codes, d_scale, d_zero, d_Wq, c->Y,
+                          cfg->d_pairs + (size_t)r * cfg->batch * 2, cfg->batch, ctx->d_moves,
+                          ctx->d_capped) != cudaSuccess)
+      return ADMMQ_ERR_CUDA;
+  if (!h_report) return ADMMQ_OK;
+  cudaEventRecord(ev1, c->stream);
+  memset(h_report, 0, sizeof(*h_report));
+  if (gradient(ctx, d_W0, p, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 2);
+  st = read_status(ctx);
+  double errs[2] = {0, 0};
+  long long moves = 0;
+  int rounds_applied = 0;
+  cudaMemcpy(errs, c->scal + 1, 2 * sizeof(double), cudaMemcpyDeviceToHost);
+  cudaMemcpy(&moves, ctx->d_moves, sizeof(long long), cudaMemcpyDeviceToHost);
+  cudaMemcpy(&rounds_applied, ctx->d_capped, sizeof(int), cudaMemcpyDeviceToHost);
+  cudaEventElapsedTime(&h_report->ms, ev0, ev1);
+  cudaEventDestroy(ev0);
+  cudaEventDestroy(ev1);
+  h_report->err_before = errs[0];
+  h_report->err_after = errs[1];
+  h_report->moves = moves;
+  h_report->iters_run = rounds_applied;
   return st;
 }
 

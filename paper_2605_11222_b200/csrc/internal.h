@@ -54,6 +54,9 @@ struct Ctx {
   double* pvec = nullptr;       // [n] matrix-vector scratch of the reduction
   float* stage_l = nullptr;     // [T_max+1][stage_factor_stride(n)] LDL^T multipliers per penalty
   float* stage_invd = nullptr;  // [T_max+1][stage_factor_stride(n)] LDL^T inverse pivots per penalty
+  double* ps_totals = nullptr;  // [PAIR_BATCH_MAX] totals of the candidate pairs of a pair-swap round
+  int* ps_chosen = nullptr;     // [1] index of the applied pair, -1: none
+  float* ps_d = nullptr;        // [2][p] applied perturbations of the two rows
   double* trd_ws = nullptr;     // scratch of the blocked reduction: 66 n + 67 * 256 doubles
   double* wy_s = nullptr;       // [ceil(n/32)][32][32] triangular factors of the reflector blocks
   bf16 *Q_hi = nullptr, *Q_lo = nullptr;    // [n][n] Q   (row i, col m)
@@ -117,5 +120,11 @@ cudaError_t launch_local_search(Ctx* c, const float* W0, int p, int bits, int gs
                                 float tau, unsigned char* codes, const float* delta,
                                 const float* zero, float* Wq, float* g, long long* d_moves,
                                 int* d_capped);
+
+// ---- pair_swap.cu ----
+constexpr int PAIR_BATCH_MAX = 65536;
+cudaError_t launch_pair_round(Ctx* c, int p, int bits, int gs, float tau, unsigned char* codes,
+                              const float* delta, const float* zero, float* Wq, float* g, const int* pairs,
+                              int batch, long long* d_moves, int* d_rounds);
 
 }  // namespace admmq

@@ -357,3 +357,42 @@ def test_error_paths():
     sol2.hessian_set(torch.eye(n, device=DEV))
     sol2.factor(rho=[0.1], damp_frac=0.0)
     assert sol2.last_device_status() == B.OK
+
+
+# ------------------------------------------------------------------ pair-swap refinement (Sec. 3.5, Eq. 11 in full)
+@pytest.mark.parametrize("kw", [dict(d_in=512, d_out=96, n_tokens=4096, bits=3),
+                                dict(d_in=264, d_out=70, n_tokens=3000, bits=2, group_size=0, symmetric=True)])
+def test_pair_swap_parity(kw):
+    spec = wl.small_case(**kw)
+    g = _solve_gpu(spec)                                         # ADMM + single-entry local search on the GPU
+    H, Wn, _ = _solve_oracle(spec)
+    codes = g["codes_final"].clone()
+    c0 = codes.cpu().numpy()
+    delta, z0 = O.grid_fit(Wn, spec.bits, spec.group_size, spec.symmetric)
+    rng = np.random.default_rng(9)
+    pairs = rng.integers(0, spec.d_in, size=(5, 512, 2)).astype(np.int32)
+    pairs[0, 0] = (7, 7)                                         # not a pair: ignored on both sides
+    ref = O.pair_swap(H, Wn, c0, delta, z0, spec.bits, pairs)
+    Wq = g["Wq_final"].clone()
+    rep, st = g["sol"].pair_swap(g["W"], spec.bits, spec.group_size, codes, g["scale"], g["zero"],
+                                 to_dev(pairs, torch.int32, DEV), Wq=Wq)
+    assert st == B.OK and g["sol"].last_device_status() == B.OK
+    cg = codes.cpu().numpy()
+    e0 = O.objective(H, Wn, O.dequantize(c0, delta, z0))
+    e_g = O.objective(H, Wn, O.dequantize(cg, delta, z0))
+    e_o = O.objective(H, Wn, ref.Wq)
+    assert e_g <= e0 * (1 + 1e-9)                                # never worse than the start
+    assert abs(e_g - e_o) <= ERR_TOL * e_o
+    assert abs(rep.err_after - e_g) <= ERR_TOL * e_g and abs(rep.err_before - e0) <= ERR_TOL * e0
+    assert (cg == ref.codes).mean() >= CODE_AGREEMENT
+    # only the rows of candidate pairs can have moved, by one level
+    assert np.abs(cg.astype(int) - c0.astype(int)).max() <= 5
+    moved_rows = set(np.nonzero((cg != c0).any(axis=0))[0])
+    assert moved_rows <= set(pairs.reshape(-1).tolist())
+    assert rep.iters_run == sum(1 for b in ref.chosen if b >= 0) or abs(e_g - e_o) <= 1e-6 * e_o
+    assert np.allclose(Wq.cpu().numpy(), O.dequantize(cg, delta, z0), rtol=1e-6, atol=3e-8)
+    # no rounds, no batch: a no-op
+    c2 = codes.clone()
+    rep2, _ = g["sol"].pair_swap(g["W"], spec.bits, spec.group_size, c2, g["scale"], g["zero"],
+                                 torch.zeros(0, 0, 2, dtype=torch.int32, device=DEV))
+    assert torch.equal(c2, codes) and rep2.moves == 0
