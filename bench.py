@@ -321,6 +321,14 @@ def main():
     timing = sol.get_timing()
     sol.set_timing(False)
 
+    # ---- the paper's pair-swap refinement after the timed path (a widened row: measured, not part of `value`) ----
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(spec.seed + 17)
+    pairs = torch.randint(0, n, (5, 4096, 2), generator=gen, dtype=torch.int32).to(dev)
+    ps_rep, _ = sol.pair_swap(W, spec.bits, spec.group_size, codes, scale, zero, pairs)
+    pair_swap = {"rounds": 5, "pairs_per_round": 4096, "ms": ps_rep.ms, "rounds_applied": ps_rep.iters_run,
+                 "moves": ps_rep.moves, "err_before": ps_rep.err_before, "err_after": ps_rep.err_after}
+
     # ---- end to end through the public API: host (pinned) inputs, results read back ----
     e2e = None
     if not args.no_e2e:
@@ -418,7 +426,7 @@ def main():
         "w_update_useful_tflops": 4.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
         "w_update_executed_tflops": 12.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
         "err_before_local_search": rep.err_before, "err_after_local_search": rep.err_after,
-        "local_search_moves": rep.moves,
+        "local_search_moves": rep.moves, "pair_swap_after_local_search": pair_swap,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "cpu_baseline": cpu_baseline, "breakdown": breakdown,
     }
