@@ -29,7 +29,7 @@ tests/test_oracle_pins.py):
 from __future__ import annotations
 
 import dataclasses
-from typing import Callable, Optional
+from typing import Sequence, Callable, Optional
 
 import numpy as np
 import scipy.linalg
@@ -177,17 +177,27 @@ class AdmmResult:
     s: np.ndarray            # [n]  sqrt(diag H)
     V: np.ndarray            # [p, n] final dual
     W: np.ndarray            # [p, n] final continuous iterate (scaled)
+    refreshed_at: int = -1   # iteration of the accepted grid refresh, -1: none
 
 
 def admm(H: np.ndarray, W_hat: np.ndarray, bits: int, group_size: int, symmetric: bool,
          rho: np.ndarray, precond: bool = True, use_cholesky: bool = False,
          grid: Optional[tuple] = None,
-         probe: Optional[Callable[[int, dict], None]] = None) -> AdmmResult:
-    """Algorithm 1 lines 1-11 with a fixed grid (no grid refresh).
+         probe: Optional[Callable[[int, dict], None]] = None,
+         refresh_at: Sequence[int] = ()) -> AdmmResult:
+    """Algorithm 1 lines 1-11.
 
     H is the damped, unscaled Hessian; W_hat is [p, n].  `rho` is the array of
     penalties, one per iteration.  `probe(t, state)` is called each iteration
     with the state BEFORE the W-update (D, V, rho) and the W it produces.
+
+    Grid refresh (Sec. 3.3 "Grid refresh", App. B): at the iterations listed in `refresh_at`, until one
+    attempt is accepted, the grid (Delta, z0) is refitted by the initial fitting routine on the unscaled
+    projection target Sigma W~ = (W + V/rho) / s, the same target is projected again, and the new grid is
+    kept iff || D_new - W~ ||_F^2 <= || D_old - W~ ||_F^2 (whole matrix, scaled coordinates).  The dual
+    update then uses D_new, which is the paper's V <- V + rho (D_old - D_new) applied after Eq. 9.
+    Readings: when the refresh is attempted is the caller's choice; the fit uses the projected point W~
+    (the paper says "the current continuous weights"); at most one refresh is accepted.
     """
     W_hat = np.asarray(W_hat, dtype=F64)
     p, n = W_hat.shape
@@ -204,6 +214,8 @@ def admm(H: np.ndarray, W_hat: np.ndarray, bits: int, group_size: int, symmetric
     changed = np.zeros(T, dtype=np.int64)
     codes = None
     W = Ws
+    refresh_set = set(int(x) for x in refresh_at)
+    refreshed_at = -1
     for t in range(T):
         rt = float(rho[t])
         if use_cholesky:
@@ -214,6 +226,12 @@ def admm(H: np.ndarray, W_hat: np.ndarray, bits: int, group_size: int, symmetric
             probe(t, dict(D=D, V=V, rho=rt, W=W, codes=codes))
         W_tilde = W + V / rt
         k_new, D_new = project(W_tilde, s, delta, z0, bits)    # line 7
+        if refreshed_at < 0 and t in refresh_set:
+            d2, z2 = grid_fit(W_tilde / s[None, :], bits, group_size, symmetric)
+            k2, D2 = project(W_tilde, s, d2, z2, bits)
+            if np.sum((D2 - W_tilde) ** 2) <= np.sum((D_new - W_tilde) ** 2):
+                delta, z0, k_new, D_new = d2, z2, k2, D2
+                refreshed_at = t
         r[t] = np.linalg.norm(W - D_new)
         sres[t] = np.linalg.norm(D_new - D)
         if codes is not None:
@@ -222,7 +240,7 @@ def admm(H: np.ndarray, W_hat: np.ndarray, bits: int, group_size: int, symmetric
         D = D_new
         codes = k_new
     Wq = dequantize(codes, delta, z0)                          # line 11
-    return AdmmResult(codes, delta, z0, Wq, r, sres, changed, s, V, W)
+    return AdmmResult(codes, delta, z0, Wq, r, sres, changed, s, V, W, refreshed_at)
 
 
 # --------------------------------------------------------------------------

@@ -440,3 +440,85 @@ def test_pair_swap_monotone_and_diagonal_hessian_declines():
     cd = O.local_search(Hd, W, codes0, delta, z0, bits).codes
     rd = O.pair_swap(Hd, W, cd, delta, z0, bits, pairs)
     assert rd.moves == 0 and rd.chosen == [-1] * 5 and np.array_equal(rd.codes, cd)
+
+
+# ------------------------------------------------------------------ grid refresh (Sec. 3.3 "Grid refresh", App. B)
+def _refresh_case(seed=4, n=48, p=10, bits=3, gs=16):
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((200, n))
+    X[:, :3] *= 8.0
+    H = O.hessian_finalize(X.T @ X, 200)
+    W = 0.02 * rng.standard_normal((p, n))
+    rho = O.rho_schedule(40, 0.05, 1.25)
+    return H, W, bits, gs, rho
+
+
+def test_grid_refresh_at_first_iteration_changes_nothing():
+    """W^1 = W_hat and V^0 = 0, so the refit sees the dense weights: same grid, accepted with equality."""
+    H, W, bits, gs, rho = _refresh_case()
+    a = O.admm(H, W, bits, gs, False, rho)
+    b = O.admm(H, W, bits, gs, False, rho, refresh_at=[0])
+    assert b.refreshed_at == 0
+    assert np.allclose(a.delta, b.delta, rtol=1e-12) and np.allclose(a.z0, b.z0, rtol=1e-12, atol=1e-18)
+    assert np.array_equal(a.codes, b.codes)
+
+
+def test_grid_refresh_acceptance_dual_consistency_and_single_acceptance():
+    H, W, bits, gs, rho = _refresh_case()
+    snaps = {}
+    O.admm(H, W, bits, gs, False, rho, probe=lambda t, st: snaps.setdefault(t, {k: (v.copy() if hasattr(v, "copy") else v) for k, v in st.items()}))
+    res = O.admm(H, W, bits, gs, False, rho, refresh_at=range(3, 40))
+    t = res.refreshed_at
+    assert t >= 3                                                   # some attempt is accepted on this problem
+    # up to the accepted attempt the run is the fixed-grid run: rebuild that iteration by hand
+    st = snaps[t]
+    s, Ht, Ws = O.precondition(H, W)
+    Wt = st["W"] + st["V"] / st["rho"]
+    d_old, z_old = O.grid_fit(W, bits, gs, False)
+    k_old, D_old = O.project(Wt, s, d_old, z_old, bits)
+    k_new, D_new = O.project(Wt, s, res.delta, res.z0, bits)
+    assert np.sum((D_new - Wt) ** 2) <= np.sum((D_old - Wt) ** 2)   # the acceptance criterion held
+    y = Wt / s[None, :]
+    d_fit, z_fit = O.grid_fit(y, bits, gs, False)
+    assert np.allclose(d_fit, res.delta, rtol=1e-12) and np.allclose(z_fit, res.z0, rtol=1e-12, atol=1e-18)
+    lo = z_fit.repeat(gs, axis=1)
+    hi = lo + 7 * d_fit.repeat(gs, axis=1)
+    assert (y >= lo - 1e-15).all() and (y <= hi + 1e-12).all()      # the new grid spans the target
+    # dual consistency: Eq. 9 with D_old, then V += rho (D_old - D_new), equals the update with D_new
+    V_two_step = st["V"] + st["rho"] * (st["W"] - D_old) + st["rho"] * (D_old - D_new)
+    snaps2 = {}
+    O.admm(H, W, bits, gs, False, rho, refresh_at=[t],
+           probe=lambda tt, s2: snaps2.setdefault(tt, {k: (v.copy() if hasattr(v, "copy") else v) for k, v in s2.items()}))
+    assert np.allclose(snaps2[t + 1]["V"], V_two_step, rtol=0, atol=1e-12 * np.abs(V_two_step).max())
+    assert np.array_equal(snaps2[t + 1]["codes"], k_new)
+    # feasibility on the final grid, exactly one accepted refresh
+    assert res.codes.max() <= 7
+    assert np.allclose(res.Wq, O.dequantize(res.codes, res.delta, res.z0))
+    again = O.admm(H, W, bits, gs, False, rho, refresh_at=[t])
+    assert np.array_equal(again.codes, res.codes) and again.refreshed_at == t
+
+
+@pytest.mark.parametrize("seed", [4, 5])
+def test_grid_refresh_first_accepted_attempt_and_declined_ones(seed):
+    """Attempts at every iteration from 1 on: each attempt before the accepted one fails Eq. (refresh
+    criterion) when rebuilt by hand from the fixed-grid run, the accepted one passes it; without attempts the
+    run is the fixed-grid run."""
+    H, W, bits, gs, rho = _refresh_case(seed=seed)
+    snaps = {}
+    base = O.admm(H, W, bits, gs, False, rho,
+                  probe=lambda t, st: snaps.setdefault(t, {k: (v.copy() if hasattr(v, "copy") else v) for k, v in st.items()}))
+    res = O.admm(H, W, bits, gs, False, rho, refresh_at=range(1, 40))
+    t_acc = res.refreshed_at
+    assert t_acc > 1                                                # these seeds decline at least one attempt
+    s, _, _ = O.precondition(H, W)
+    d_old, z_old = O.grid_fit(W, bits, gs, False)
+    for t in range(1, t_acc + 1):
+        st = snaps[t]
+        Wt = st["W"] + st["V"] / st["rho"]
+        _, D_old = O.project(Wt, s, d_old, z_old, bits)
+        d2, z2 = O.grid_fit(Wt / s[None, :], bits, gs, False)
+        _, D2 = O.project(Wt, s, d2, z2, bits)
+        accepted = np.sum((D2 - Wt) ** 2) <= np.sum((D_old - Wt) ** 2)
+        assert accepted == (t == t_acc), t
+    never = O.admm(H, W, bits, gs, False, rho, refresh_at=[])
+    assert np.array_equal(never.codes, base.codes) and never.refreshed_at == -1
