@@ -125,6 +125,11 @@ admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg);
  * The grid is the min-max grid of the unscaled weights (Sec. 3.4): asymmetric lo = min, hi = max;
  * symmetric hi = max|w|, lo = -hi; Delta = (hi - lo)/(2^bits - 1), z0 = lo; Delta = 1 for a constant
  * group.  Rounding is to nearest, ties to even, then clamped to the grid's range.
+ * Grid refresh: at the listed iterations, until one attempt is accepted, (Delta, z0) are refitted by the same
+ * rule on the unscaled projection target (W + V/rho)/s, the target is projected on both grids, and the new grid
+ * replaces the old one (in d_scale / d_zero) iff ||D_new - W~||_F^2 <= ||D_old - W~||_F^2 over the whole matrix;
+ * the dual update then uses D_new.  Needs a group size >= 2.  At such an iteration W^(t+1) makes one trip through
+ * memory (the epilogue is not fused).
  * h_report NULL: nothing is synchronised.  Non-NULL: the call synchronises, fills the report and
  * returns the device status. */
 typedef struct {
@@ -133,6 +138,8 @@ typedef struct {
   int group_size;       /* along d_in; 0 or d_in: one group per output channel */
   int symmetric;        /* 0 asymmetric, 1 symmetric */
   int use_caller_grid;  /* 1: d_scale / d_zero are inputs */
+  int n_refresh;        /* grid refresh (Sec. 3.3, App. B): number of iterations at which it is attempted, 0: never */
+  const int* h_refresh_iters; /* HOST array [n_refresh] of iteration indices t in [0, T) */
 } admmq_quant_cfg;
 typedef struct {
   double err_before;    /* Tr(E^T H E), E = W_q - W_hat, at entry (local search) / of the ADMM result */
@@ -141,6 +148,7 @@ typedef struct {
   int iters_run;        /* ADMM iterations run */
   int capped_columns;   /* columns that hit max_moves_per_col */
   float ms;             /* device time of the call, CUDA events */
+  int refreshed_iter;   /* quantize_layer: iteration of the accepted grid refresh, -1: none */
 } admmq_report;
 admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out,
                                   const admmq_quant_cfg* cfg, unsigned char* d_codes, float* d_scale,

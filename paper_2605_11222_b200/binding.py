@@ -43,7 +43,8 @@ class FactorCfg(C.Structure):
 
 class QuantCfg(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("bits", C.c_int), ("group_size", C.c_int),
-                ("symmetric", C.c_int), ("use_caller_grid", C.c_int)]
+                ("symmetric", C.c_int), ("use_caller_grid", C.c_int), ("n_refresh", C.c_int),
+                ("h_refresh_iters", C.POINTER(C.c_int))]
 
 
 class LsCfg(C.Structure):
@@ -58,7 +59,8 @@ class PairSwapCfg(C.Structure):
 
 class Report(C.Structure):
     _fields_ = [("err_before", C.c_double), ("err_after", C.c_double), ("moves", C.c_longlong),
-                ("iters_run", C.c_int), ("capped_columns", C.c_int), ("ms", C.c_float)]
+                ("iters_run", C.c_int), ("capped_columns", C.c_int), ("ms", C.c_float),
+                ("refreshed_iter", C.c_int)]
 
 
 class AdmmqError(RuntimeError):
@@ -208,14 +210,16 @@ class Solver:
 
     def quantize_layer(self, W0: torch.Tensor, bits: int, group_size: int = 0, symmetric: bool = False,
                        codes=None, scale=None, zero=None, Wq=None, resid=None, use_caller_grid=False,
-                       report: bool = True):
+                       report: bool = True, refresh_at: Sequence[int] = ()):
         p, n = W0.shape
         gs = n if group_size in (0, n) else group_size
         dev = W0.device
         codes = codes if codes is not None else torch.empty(p, n, dtype=torch.uint8, device=dev)
         scale = scale if scale is not None else torch.empty(p, n // gs, dtype=torch.float32, device=dev)
         zero = zero if zero is not None else torch.empty(p, n // gs, dtype=torch.float32, device=dev)
-        cfg = QuantCfg(C.sizeof(QuantCfg), bits, group_size, int(symmetric), int(use_caller_grid))
+        iters = (C.c_int * max(1, len(refresh_at)))(*[int(t) for t in refresh_at])
+        cfg = QuantCfg(C.sizeof(QuantCfg), bits, group_size, int(symmetric), int(use_caller_grid),
+                       len(refresh_at), C.cast(iters, C.POINTER(C.c_int)) if len(refresh_at) else None)
         rep = Report()
         st = self.lib.admmq_quantize_layer(self.h, _ptr(W0), p, C.byref(cfg), _ptr(codes), _ptr(scale),
                                            _ptr(zero), _ptr(Wq), _ptr(resid),

@@ -382,6 +382,8 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   admmq_status st = check_layer_args(ctx, d_W0, d_out, cfg->bits, cfg->group_size, d_codes, d_scale, d_zero);
   if (st != ADMMQ_OK) return st;
   if ((d_Wq && !aligned16(d_Wq)) || (d_resid && !aligned16(d_resid))) return ADMMQ_ERR_INVALID_ARG;
+  if (cfg->n_refresh < 0 || (cfg->n_refresh > 0 && !cfg->h_refresh_iters)) return ADMMQ_ERR_INVALID_ARG;
+  if (cfg->n_refresh > 0 && group_of(ctx->c.n, cfg->group_size) < 2) return ADMMQ_ERR_UNSUPPORTED;
   Ctx* c = &ctx->c;
   const int n = c->n, p = d_out, gs = group_of(n, cfg->group_size), T = c->T;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -392,6 +394,8 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   if (!cfg->use_caller_grid) launch_grid_fit(c, d_W0, p, cfg->bits, gs, cfg->symmetric, d_scale, d_zero);
   launch_scale_weights(c, d_W0, p);                        // W_hat', V = 0, R = 0 (Algorithm 1 l.2, l.4)
   launch_zero(c, c->partials, (size_t)T * c->partial_slots * 2 * sizeof(float));
+  int* refresh_flags = c->ps_chosen + 4;                   // [0] this attempt accepted, [1] 1 + accepted iteration
+  launch_zero(c, c->ps_chosen, 64);
   EpiParams e{};
   e.kind = EPI_ADMM;
   e.Whs = c->Whs;
@@ -413,7 +417,19 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     e.inv_rho = (float)(1.0 / rho);
     e.inv_rho_next = (float)(1.0 / rho_next);
     e.partials = c->partials + (size_t)t * c->partial_slots * 2;
-    if (w_update_products(ctx, p, t, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
+    bool refresh = false;
+    for (int q = 0; q < cfg->n_refresh; ++q) refresh = refresh || (cfg->h_refresh_iters[q] == t);
+    if (refresh) {
+      // grid refresh attempt: W^(t+1) is stored by the plain epilogue, then evaluated on both grids
+      EpiParams w = e;
+      w.kind = EPI_WOUT;
+      w.C = c->Y;
+      w.ldc = n;
+      if (w_update_products(ctx, p, t, w) != cudaSuccess) return ADMMQ_ERR_CUDA;
+      launch_grid_refresh(c, e, p, cfg->bits, cfg->symmetric, t, d_scale, d_zero, refresh_flags);
+    } else if (w_update_products(ctx, p, t, e) != cudaSuccess) {
+      return ADMMQ_ERR_CUDA;
+    }
     if (t + 1 < T) {
       Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
       launch_row_split(c, c->Y, p, c->R_hi, c->R_lo, c->rs_R);
@@ -433,9 +449,12 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   cudaEventElapsedTime(&h_report->ms, ev0, ev1);
   cudaEventDestroy(ev0);
   cudaEventDestroy(ev1);
+  int flags[2] = {0, 0};
+  cudaMemcpy(flags, refresh_flags, sizeof(flags), cudaMemcpyDeviceToHost);
   h_report->err_before = err;
   h_report->err_after = err;
   h_report->iters_run = T;
+  h_report->refreshed_iter = flags[1] - 1;
   return st;
 }
 

@@ -428,6 +428,147 @@ void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned 
   LAUNCH(c);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Grid refresh (Sec. 3.3 "Grid refresh", App. B) at one iteration, from the stored W^(t+1):
+//   eval:   per (channel, group) refit (Delta', z0') on the unscaled target (W + V/rho)/s by the initial
+//           fitting rule, project the target on the old and on the new grid, sum both squared distances;
+//   decide: new grid kept iff its sum <= the old one (Eq. of App. B) and no refresh was accepted before;
+//   apply:  the ADMM element update (projection, dual, residual sums, next right-hand side) with the grid
+//           that was kept.  Same arithmetic as the fused epilogue.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+refresh_eval_kernel(const float* __restrict__ Wc, const float* __restrict__ V, const float* __restrict__ s,
+                    const float* __restrict__ inv_s, int p, int n, int gs, int kmax, int symmetric,
+                    float inv_rho, const float* __restrict__ delta, const float* __restrict__ zero,
+                    float* __restrict__ cand_delta, float* __restrict__ cand_zero, double* __restrict__ partial) {
+  __shared__ double scratch[32];
+  const int ng = n / gs, lane = threadIdx.x & 31;
+  const long long groups = (long long)p * ng;
+  double e_old = 0.0, e_new = 0.0;
+  for (long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; gw < groups;
+       gw += ((long long)gridDim.x * blockDim.x) >> 5) {
+    const int j = (int)(gw / ng), gq = (int)(gw % ng);
+    const size_t base = (size_t)j * n + (size_t)gq * gs;
+    float lo = INFINITY, hi = -INFINITY;
+    for (int i = lane; i < gs; i += 32) {
+      const float y = fmaf(V[base + i], inv_rho, Wc[base + i]) * inv_s[gq * gs + i];
+      lo = fminf(lo, y);
+      hi = fmaxf(hi, y);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+    }
+    if (symmetric) {
+      hi = fmaxf(fabsf(lo), fabsf(hi));
+      lo = -hi;
+    }
+    float dn = (hi - lo) / (float)kmax;
+    if (hi - lo == 0.f) dn = 1.f;
+    const float zn = lo;
+    if (lane == 0) {
+      cand_delta[gw] = dn;
+      cand_zero[gw] = zn;
+    }
+    const float d0 = delta[gw], z0 = zero[gw];
+    const float id0 = __frcp_rn(d0), idn = __frcp_rn(dn);
+    float a = 0.f, b = 0.f;
+    for (int i = lane; i < gs; i += 32) {
+      const float sv = s[gq * gs + i];
+      const float wt = fmaf(V[base + i], inv_rho, Wc[base + i]);
+      const float y = wt * inv_s[gq * gs + i];
+      const float k0 = fminf(fmaxf(rintf((y - z0) * id0), 0.f), (float)kmax);
+      const float kn = fminf(fmaxf(rintf((y - zn) * idn), 0.f), (float)kmax);
+      const float eo = sv * (z0 + d0 * k0) - wt, en = sv * (zn + dn * kn) - wt;
+      a = fmaf(eo, eo, a);
+      b = fmaf(en, en, b);
+    }
+    e_old += (double)warp_sum(a);
+    e_new += (double)warp_sum(b);
+  }
+  e_old = block_sum(e_old, scratch);       // every lane of a warp carries its warp's sums: divide by 32 below
+  e_new = block_sum(e_new, scratch);
+  if (threadIdx.x == 0) {
+    partial[2 * blockIdx.x] = e_old / 32.0;
+    partial[2 * blockIdx.x + 1] = e_new / 32.0;
+  }
+}
+
+// flags[0]: 1 if this attempt is accepted; flags[1]: 1 + iteration of the accepted refresh (0: none so far)
+__global__ void refresh_decide_kernel(const double* __restrict__ partial, int blocks, int iter, int* flags) {
+  __shared__ double scratch[32];
+  double a = 0.0, b = 0.0;
+  for (int i = threadIdx.x; i < blocks; i += blockDim.x) {
+    a += partial[2 * i];
+    b += partial[2 * i + 1];
+  }
+  a = block_sum(a, scratch);
+  b = block_sum(b, scratch);
+  if (threadIdx.x == 0) {
+    const int ok = (flags[1] == 0 && b <= a) ? 1 : 0;
+    flags[0] = ok;
+    if (ok) flags[1] = iter + 1;
+  }
+}
+
+__global__ void refresh_commit_kernel(long long groups, const int* __restrict__ flags,
+                                      const float* __restrict__ cand_delta, const float* __restrict__ cand_zero,
+                                      float* __restrict__ delta, float* __restrict__ zero) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= groups || !flags[0]) return;
+  delta[i] = cand_delta[i];
+  zero[i] = cand_zero[i];
+}
+
+// The ADMM element update from a stored W^(t+1) (in P.Rnext, overwritten by the next right-hand side).
+__global__ void __launch_bounds__(256) admm_elementwise_kernel(EpiParams P, long long total, int n) {
+  __shared__ float red[32];
+  float r2 = 0.f, s2 = 0.f;
+  for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int col = (int)(idx % n);
+    const long long row = idx / n;
+    const long long gi = row * P.n_groups + col / P.group_size;
+    const float dl = P.delta[gi], z0 = P.zero[gi];
+    const float wh = P.Whs[idx];
+    AdmmElem e = admm_elem(P.Rnext[idx] - wh, wh, P.V[idx], P.first_iter ? 0 : (int)P.codes[idx], P.s[col],
+                           P.inv_s[col], dl, __frcp_rn(dl), z0, P);
+    P.codes[idx] = e.code;
+    P.V[idx] = e.v_new;
+    P.Rnext[idx] = e.r_next;
+    r2 += e.dr2;
+    s2 += e.ds2;
+  }
+  r2 = block_sum(r2, red);
+  s2 = block_sum(s2, red);
+  if (threadIdx.x == 0) {
+    P.partials[2 * blockIdx.x + 0] = r2;
+    P.partials[2 * blockIdx.x + 1] = s2;
+  }
+}
+
+void launch_grid_refresh(Ctx* c, const EpiParams& P, int p, int bits, int symmetric, int iter, float* delta,
+                         float* zero, int* flags) {
+  const int n = c->n, gs = P.group_size, ng = n / gs;
+  const long long groups = (long long)p * ng;
+  float* cand_delta = reinterpret_cast<float*>(c->R_hi);      // the R planes are free between the products
+  float* cand_zero = reinterpret_cast<float*>(c->R_lo);       // and the row pass that rewrites them
+  long long want = (groups * 32 + 255) / 256;
+  const int blocks = (int)(want < 1184 ? want : 1184);
+  refresh_eval_kernel<<<blocks, 256, 0, c->stream>>>(P.Rnext, P.V, P.s, P.inv_s, p, n, gs, (1 << bits) - 1,
+                                                     symmetric, P.inv_rho, delta, zero, cand_delta, cand_zero,
+                                                     c->ps_totals);
+  refresh_decide_kernel<<<1, 256, 0, c->stream>>>(c->ps_totals, blocks, iter, flags);
+  refresh_commit_kernel<<<(unsigned)((groups + 255) / 256), 256, 0, c->stream>>>(groups, flags, cand_delta,
+                                                                                 cand_zero, delta, zero);
+  const long long total = (long long)p * n;
+  int eb = c->partial_slots < 1184 ? c->partial_slots : 1184;
+  if ((long long)eb * 256 > total) eb = (int)((total + 255) / 256);
+  admm_elementwise_kernel<<<eb, 256, 0, c->stream>>>(P, total, n);
+  c->launches += 4;
+}
+
 // sum_j eps_j . g_j  =  Tr(E^T H E)  when g = H E  (fp64 accumulation).
 __global__ void objective_dot_kernel(long long total, int n, int gs, int ng, const float* __restrict__ W0,
                                      const unsigned char* __restrict__ codes,

@@ -98,6 +98,8 @@ void launch_dequant(Ctx* c, int p, int gs, const unsigned char* codes, const flo
                     const float* zero, float* Wq);
 void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes,
                          const float* delta, const float* zero, bf16* Ehi, bf16* Elo, float* row_inv);
+void launch_grid_refresh(Ctx* c, const EpiParams& P, int p, int bits, int symmetric, int iter, float* delta,
+                         float* zero, int* flags);
 void launch_objective_dot(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes,
                           const float* delta, const float* zero, const float* g, double* out);
 

@@ -396,3 +396,48 @@ def test_pair_swap_parity(kw):
     rep2, _ = g["sol"].pair_swap(g["W"], spec.bits, spec.group_size, c2, g["scale"], g["zero"],
                                  torch.zeros(0, 0, 2, dtype=torch.int32, device=DEV))
     assert torch.equal(c2, codes) and rep2.moves == 0
+
+
+# ------------------------------------------------------------------ grid refresh (Sec. 3.3 "Grid refresh", App. B)
+@pytest.mark.parametrize("kw,attempts", [
+    (dict(d_in=512, d_out=384, n_tokens=6144), list(range(1, 40))),          # g128, asym: first accepted attempt
+    (dict(d_in=264, d_out=70, n_tokens=3000, bits=2, group_size=0, symmetric=True), [4]),
+    (dict(d_in=256, d_out=64, n_tokens=2048, group_size=64), [0]),            # at t = 0 the refit sees W_hat: no change
+])
+def test_grid_refresh_parity(kw, attempts):
+    spec = wl.small_case(**kw)
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(spec.d_in, spec.d_out, T_max=spec.T)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=spec.rho())
+    resid = torch.zeros(spec.T, 2, device=DEV)
+    codes, scale, zero, rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, resid=resid,
+                                                 refresh_at=attempts)
+    assert sol.last_device_status() == B.OK
+    H = oracle_hessian(spec, DEV)
+    Wn = np64(W)
+    ref = O.admm(H, Wn, spec.bits, spec.group_size, spec.symmetric, np.array(spec.rho()), refresh_at=attempts)
+    # The accepted attempt is a comparison of two sums over the whole matrix.  At t = 0 the target is W_hat
+    # itself, both grids coincide and the two sums are equal up to rounding: either answer is right there.
+    if attempts != [0]:
+        assert rep.refreshed_iter == ref.refreshed_at
+    assert np.allclose(scale.cpu().numpy(), ref.delta, rtol=2e-5, atol=0)
+    assert np.allclose(zero.cpu().numpy(), ref.z0, rtol=2e-5, atol=1e-7)
+    cg = codes.cpu().numpy()
+    assert cg.max() <= (1 << spec.bits) - 1
+    assert (cg == ref.codes).mean() >= CODE_AGREEMENT
+    e_g = O.objective(H, Wn, O.dequantize(cg, ref.delta, ref.z0))
+    e_o = O.objective(H, Wn, ref.Wq)
+    assert abs(e_g - e_o) <= ERR_TOL * e_o
+    assert abs(rep.err_before - e_g) <= 2 * ERR_TOL * e_g
+    r = resid.cpu().numpy()
+    assert np.abs(r[:, 0] - ref.r).max() <= 1e-3 * ref.r.max()
+    if attempts == [0]:
+        base = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric)[0]
+        assert (base == codes).float().mean().item() >= 0.9999
+    # a refresh needs groups of at least two entries
+    with pytest.raises(B.AdmmqError) as e:
+        sol.quantize_layer(W, spec.bits, 1, spec.symmetric, refresh_at=[3])
+    assert e.value.status == B.ERR_UNSUPPORTED
