@@ -329,6 +329,18 @@ def main():
     pair_swap = {"rounds": 5, "pairs_per_round": 4096, "ms": ps_rep.ms, "rounds_applied": ps_rep.iters_run,
                  "moves": ps_rep.moves, "err_before": ps_rep.err_before, "err_after": ps_rep.err_after}
 
+    # ---- a run with grid-refresh attempts at iterations 2..11 (another widened row: measured, not part of `value`) ----
+    attempts = list(range(2, min(12, T)))
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    _, _, _, gr_rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, codes=codes, scale=scale,
+                                         zero=zero, resid=resid, refresh_at=attempts)
+    t1.record()
+    torch.cuda.synchronize(dev)
+    grid_refresh = {"attempt_iters": attempts, "accepted_at": gr_rep.refreshed_iter,
+                    "quantize_layer_ms": gr_rep.ms, "err_admm": gr_rep.err_before}
+
     # ---- end to end through the public API: host (pinned) inputs, results read back ----
     e2e = None
     if not args.no_e2e:
@@ -426,7 +438,7 @@ def main():
         "w_update_useful_tflops": 4.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
         "w_update_executed_tflops": 12.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
         "err_before_local_search": rep.err_before, "err_after_local_search": rep.err_after,
-        "local_search_moves": rep.moves, "pair_swap_after_local_search": pair_swap,
+        "local_search_moves": rep.moves, "pair_swap_after_local_search": pair_swap, "admm_with_grid_refresh": grid_refresh,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "cpu_baseline": cpu_baseline, "breakdown": breakdown,
     }
