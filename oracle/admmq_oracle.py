@@ -106,6 +106,42 @@ def grid_fit(W_hat: np.ndarray, bits: int, group_size: int, symmetric: bool):
     return delta, lo.copy()
 
 
+def grid_fit_mse(W_hat: np.ndarray, bits: int, group_size: int, symmetric: bool, points: int = 100,
+                 min_ratio: float = 0.8):
+    """MSE search for the clipping ratio (Sec. 3.4 "Clipping Heuristics"; App. D: 100 grid points, maximum
+    shrink ratio 0.8).  Per (output channel, group): candidates r_i = 1 - (1 - min_ratio) i / (points - 1),
+    i = 0 .. points-1; the min-max range is shrunk to [r lo, r hi] (symmetric: +-r max|w|), Delta and z0
+    follow as in grid_fit, the group is rounded to that grid with clamping, and the candidate with the
+    smallest sum of squared rounding errors is kept (the largest ratio on ties).
+    Readings: the ratio scales both ends of the range towards zero; the candidates run from 1.0 down to
+    min_ratio inclusive; the error is the plain squared error of the unscaled weights."""
+    W = np.asarray(W_hat, dtype=F64)
+    p, n = W.shape
+    gs = n if group_size in (0, n) else group_size
+    Wg = W.reshape(p, n // gs, gs)
+    if symmetric:
+        hi0 = np.abs(Wg).max(axis=2)
+        lo0 = -hi0
+    else:
+        hi0 = Wg.max(axis=2)
+        lo0 = Wg.min(axis=2)
+    levels = (1 << bits) - 1
+    best_err = np.full(hi0.shape, np.inf)
+    best_delta = np.ones(hi0.shape)
+    best_z0 = lo0.copy()
+    for i in range(points):
+        r = 1.0 - (1.0 - min_ratio) * i / max(points - 1, 1)
+        lo, hi = r * lo0, r * hi0
+        delta = np.where(hi - lo == 0.0, 1.0, (hi - lo) / levels)
+        k = np.clip(np.rint((Wg - lo[..., None]) / delta[..., None]), 0, levels)
+        err = ((lo[..., None] + delta[..., None] * k - Wg) ** 2).sum(axis=2)
+        take = err < best_err
+        best_err = np.where(take, err, best_err)
+        best_delta = np.where(take, delta, best_delta)
+        best_z0 = np.where(take, lo, best_z0)
+    return best_delta, best_z0
+
+
 def _expand(g: np.ndarray, n: int) -> np.ndarray:
     """[p, n/gs] per-group values -> [p, n]."""
     return np.repeat(g, n // g.shape[1], axis=1)

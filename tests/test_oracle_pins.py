@@ -522,3 +522,40 @@ def test_grid_refresh_first_accepted_attempt_and_declined_ones(seed):
         assert accepted == (t == t_acc), t
     never = O.admm(H, W, bits, gs, False, rho, refresh_at=[])
     assert np.array_equal(never.codes, base.codes) and never.refreshed_at == -1
+
+
+# ------------------------------------------------------------------ MSE search for the clipping ratio (Sec. 3.4, App. D)
+def test_mse_clip_search_brute_force_and_limits():
+    rng = np.random.default_rng(21)
+    p, n, gs, bits = 6, 64, 16, 3
+    W = 0.02 * rng.standard_normal((p, n))
+    W[0, 3] = 0.2                                               # an outlier: clipping it pays
+    delta, z0 = O.grid_fit_mse(W, bits, gs, False)
+    d_mm, z_mm = O.grid_fit(W, bits, gs, False)
+    levels = 7
+    ratios = [1.0 - 0.2 * i / 99 for i in range(100)]
+
+    def group_err(w, lo, dl):
+        k = np.clip(np.rint((w - lo) / dl), 0, levels)
+        return float(((lo + dl * k - w) ** 2).sum())
+
+    for j in range(p):
+        for g in range(n // gs):
+            w = W[j, g * gs:(g + 1) * gs]
+            errs = [group_err(w, r * w.min(), (r * w.max() - r * w.min()) / levels) for r in ratios]
+            i_best = int(np.argmin(errs))                        # first minimum = largest ratio
+            r = ratios[i_best]
+            assert abs(z0[j, g] - r * w.min()) <= 1e-15
+            assert abs(delta[j, g] - r * (w.max() - w.min()) / levels) <= 1e-15
+            assert errs[i_best] <= group_err(w, z_mm[j, g], d_mm[j, g]) + 1e-18   # never worse than min-max
+    assert delta[0, 0] < d_mm[0, 0]                              # the outlier group is clipped
+    # one candidate = the min-max grid; a constant group keeps Delta = 1
+    d1, z1 = O.grid_fit_mse(W, bits, gs, False, points=1)
+    assert np.array_equal(d1, d_mm) and np.array_equal(z1, z_mm)
+    Wc = W.copy()
+    Wc[1, :gs] = 0.5
+    dc, zc = O.grid_fit_mse(Wc, bits, gs, False)
+    assert dc[1, 0] == 1.0
+    # symmetric: the grid stays symmetric around zero
+    ds, zs = O.grid_fit_mse(W, bits, gs, True)
+    assert np.allclose(zs, -0.5 * levels * ds)
