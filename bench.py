@@ -341,6 +341,14 @@ def main():
     grid_refresh = {"attempt_iters": attempts, "accepted_at": gr_rep.refreshed_iter,
                     "quantize_layer_ms": gr_rep.ms, "err_admm": gr_rep.err_before}
 
+    # ---- a run whose grid comes from the MSE search for the clipping ratio, 100 candidates down to 0.8
+    #      (another widened row: measured, not part of `value`), followed by the local search ----
+    _, _, _, cl_rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, codes=codes, scale=scale,
+                                         zero=zero, resid=resid, clip_points=100, clip_min_ratio=0.8)
+    cl_ls, _ = sol.local_search(W, spec.bits, spec.group_size, codes, scale, zero)
+    mse_clip = {"points": 100, "min_ratio": 0.8, "quantize_layer_ms": cl_rep.ms, "err_admm": cl_rep.err_before,
+                "err_after_local_search": cl_ls.err_after}
+
     # ---- end to end through the public API: host (pinned) inputs, results read back ----
     e2e = None
     if not args.no_e2e:
@@ -439,6 +447,7 @@ def main():
         "w_update_executed_tflops": 12.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
         "err_before_local_search": rep.err_before, "err_after_local_search": rep.err_after,
         "local_search_moves": rep.moves, "pair_swap_after_local_search": pair_swap, "admm_with_grid_refresh": grid_refresh,
+        "admm_with_mse_clip_search": mse_clip,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "cpu_baseline": cpu_baseline, "breakdown": breakdown,
     }

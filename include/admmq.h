@@ -140,6 +140,12 @@ typedef struct {
   int use_caller_grid;  /* 1: d_scale / d_zero are inputs */
   int n_refresh;        /* grid refresh (Sec. 3.3, App. B): number of iterations at which it is attempted, 0: never */
   const int* h_refresh_iters; /* HOST array [n_refresh] of iteration indices t in [0, T) */
+  int clip_points;      /* MSE search for the clipping ratio (Sec. 3.4 "Clipping Heuristics", App. D): number of
+                           candidate ratios, 0: plain min-max grid; the paper uses 100.  Ignored with a caller grid. */
+  double clip_min_ratio;/* smallest candidate ratio in (0, 1]; the paper uses 0.8.  Candidates are
+                           r_i = 1 - (1 - clip_min_ratio) i / (clip_points - 1); each scales both ends of the group's
+                           min-max range (symmetric: +-r max|w|), and the candidate with the smallest sum of squared
+                           rounding errors of the group is kept (the largest ratio on ties). */
 } admmq_quant_cfg;
 typedef struct {
   double err_before;    /* Tr(E^T H E), E = W_q - W_hat, at entry (local search) / of the ADMM result */

@@ -44,7 +44,8 @@ class FactorCfg(C.Structure):
 class QuantCfg(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("bits", C.c_int), ("group_size", C.c_int),
                 ("symmetric", C.c_int), ("use_caller_grid", C.c_int), ("n_refresh", C.c_int),
-                ("h_refresh_iters", C.POINTER(C.c_int))]
+                ("h_refresh_iters", C.POINTER(C.c_int)), ("clip_points", C.c_int),
+                ("clip_min_ratio", C.c_double)]
 
 
 class LsCfg(C.Structure):
@@ -210,7 +211,8 @@ class Solver:
 
     def quantize_layer(self, W0: torch.Tensor, bits: int, group_size: int = 0, symmetric: bool = False,
                        codes=None, scale=None, zero=None, Wq=None, resid=None, use_caller_grid=False,
-                       report: bool = True, refresh_at: Sequence[int] = ()):
+                       report: bool = True, refresh_at: Sequence[int] = (), clip_points: int = 0,
+                       clip_min_ratio: float = 0.8):
         p, n = W0.shape
         gs = n if group_size in (0, n) else group_size
         dev = W0.device
@@ -219,7 +221,8 @@ class Solver:
         zero = zero if zero is not None else torch.empty(p, n // gs, dtype=torch.float32, device=dev)
         iters = (C.c_int * max(1, len(refresh_at)))(*[int(t) for t in refresh_at])
         cfg = QuantCfg(C.sizeof(QuantCfg), bits, group_size, int(symmetric), int(use_caller_grid),
-                       len(refresh_at), C.cast(iters, C.POINTER(C.c_int)) if len(refresh_at) else None)
+                       len(refresh_at), C.cast(iters, C.POINTER(C.c_int)) if len(refresh_at) else None,
+                       int(clip_points), float(clip_min_ratio))
         rep = Report()
         st = self.lib.admmq_quantize_layer(self.h, _ptr(W0), p, C.byref(cfg), _ptr(codes), _ptr(scale),
                                            _ptr(zero), _ptr(Wq), _ptr(resid),

@@ -383,6 +383,8 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   if (st != ADMMQ_OK) return st;
   if ((d_Wq && !aligned16(d_Wq)) || (d_resid && !aligned16(d_resid))) return ADMMQ_ERR_INVALID_ARG;
   if (cfg->n_refresh < 0 || (cfg->n_refresh > 0 && !cfg->h_refresh_iters)) return ADMMQ_ERR_INVALID_ARG;
+  if (cfg->clip_points < 0 || cfg->clip_points > 4096) return ADMMQ_ERR_INVALID_ARG;
+  if (cfg->clip_points > 0 && !(cfg->clip_min_ratio > 0.0 && cfg->clip_min_ratio <= 1.0)) return ADMMQ_ERR_INVALID_ARG;
   if (cfg->n_refresh > 0 && group_of(ctx->c.n, cfg->group_size) < 2) return ADMMQ_ERR_UNSUPPORTED;
   Ctx* c = &ctx->c;
   const int n = c->n, p = d_out, gs = group_of(n, cfg->group_size), T = c->T;
@@ -391,7 +393,13 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return ADMMQ_ERR_CUDA;
     cudaEventRecord(ev0, c->stream);
   }
-  if (!cfg->use_caller_grid) launch_grid_fit(c, d_W0, p, cfg->bits, gs, cfg->symmetric, d_scale, d_zero);
+  if (!cfg->use_caller_grid) {
+    if (cfg->clip_points > 0)
+      launch_grid_fit_mse(c, d_W0, p, cfg->bits, gs, cfg->symmetric, cfg->clip_points, cfg->clip_min_ratio,
+                          d_scale, d_zero);
+    else
+      launch_grid_fit(c, d_W0, p, cfg->bits, gs, cfg->symmetric, d_scale, d_zero);
+  }
   launch_scale_weights(c, d_W0, p);                        // W_hat', V = 0, R = 0 (Algorithm 1 l.2, l.4)
   launch_zero(c, c->partials, (size_t)T * c->partial_slots * 2 * sizeof(float));
   int* refresh_flags = c->ps_chosen + 4;                   // [0] this attempt accepted, [1] 1 + accepted iteration

@@ -167,6 +167,102 @@ void launch_grid_fit(Ctx* c, const float* W0, int p, int bits, int gs, int symme
   LAUNCH(c);
 }
 
+// Grid fit with an MSE search for the clipping ratio (Sec. 3.4 "Clipping Heuristics"; App. D: 100 grid
+// points, maximum shrink ratio 0.8): candidates r_i = 1 - (1 - min_ratio) i / (points - 1) scale both ends
+// of the min-max range; the candidate with the smallest sum of squared rounding errors of the group wins
+// (strict <, so the largest ratio on ties).  One warp per (output channel, group); a group of up to
+// 32 * CLIP_REG values is held in registers, longer ones are re-read (they stay in L1/L2).
+constexpr int CLIP_REG = 8;
+__global__ void grid_fit_mse_kernel(const float* __restrict__ W0, int p, int n, int gs, int levels,
+                                    int symmetric, int points, double min_ratio,
+                                    float* __restrict__ delta, float* __restrict__ zero) {
+  const int ng = n / gs;
+  const long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (gw >= (long long)p * ng) return;
+  const int j = (int)(gw / ng), g = (int)(gw % ng);
+  const float* w = W0 + (long long)j * n + (long long)g * gs;
+  const bool in_regs = gs <= 32 * CLIP_REG;
+  float wr[CLIP_REG];
+  float lo0 = INFINITY, hi0 = -INFINITY;
+  if (in_regs) {
+#pragma unroll
+    for (int q = 0; q < CLIP_REG; ++q) {
+      const int i = lane + 32 * q;
+      wr[q] = i < gs ? w[i] : NAN;
+      if (i < gs) {
+        lo0 = fminf(lo0, wr[q]);
+        hi0 = fmaxf(hi0, wr[q]);
+      }
+    }
+  } else {
+    for (int i = lane; i < gs; i += 32) {
+      const float v = w[i];
+      lo0 = fminf(lo0, v);
+      hi0 = fmaxf(hi0, v);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    lo0 = fminf(lo0, __shfl_xor_sync(0xffffffffu, lo0, o));
+    hi0 = fmaxf(hi0, __shfl_xor_sync(0xffffffffu, hi0, o));
+  }
+  if (symmetric) {
+    hi0 = fmaxf(fabsf(lo0), fabsf(hi0));
+    lo0 = -hi0;
+  }
+  const float fl = (float)levels;
+  double best = INFINITY;
+  float best_d = 1.f, best_lo = lo0;
+  const double step = points > 1 ? (1.0 - min_ratio) / (double)(points - 1) : 0.0;
+  for (int c = 0; c < points; ++c) {
+    const double r = 1.0 - step * (double)c;
+    const float lo = (float)(r * (double)lo0), hi = (float)(r * (double)hi0);
+    float d = (hi - lo) / fl;
+    if (hi - lo == 0.f) d = 1.f;
+    const float inv_d = 1.f / d;
+    double acc = 0.0;
+    if (in_regs) {
+#pragma unroll
+      for (int q = 0; q < CLIP_REG; ++q) {
+        if (lane + 32 * q < gs) {
+          const float k = fminf(fmaxf(rintf((wr[q] - lo) * inv_d), 0.f), fl);
+          const float e = fmaf(d, k, lo) - wr[q];
+          acc += (double)e * (double)e;
+        }
+      }
+    } else {
+      for (int i = lane; i < gs; i += 32) {
+        const float v = w[i];
+        const float k = fminf(fmaxf(rintf((v - lo) * inv_d), 0.f), fl);
+        const float e = fmaf(d, k, lo) - v;
+        acc += (double)e * (double)e;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (acc < best) {
+      best = acc;
+      best_d = d;
+      best_lo = lo;
+    }
+  }
+  if (lane == 0) {
+    delta[gw] = best_d;
+    zero[gw] = best_lo;
+  }
+}
+
+void launch_grid_fit_mse(Ctx* c, const float* W0, int p, int bits, int gs, int symmetric, int points,
+                         double min_ratio, float* delta, float* zero) {
+  const long long warps = (long long)p * (c->n / gs);
+  const int threads = 128;
+  const long long blocks = (warps * 32 + threads - 1) / threads;
+  grid_fit_mse_kernel<<<(unsigned)blocks, threads, 0, c->stream>>>(
+      W0, p, c->n, gs, (1 << bits) - 1, symmetric, points, min_ratio, delta, zero);
+  LAUNCH(c);
+}
+
 // W_hat' = Sigma^{-1} W_hat (Algorithm 1 line 2); V^(0) = 0; first right-hand side R = D^(0) - W_hat' = 0
 // (all-zero planes, row scale 1).
 __global__ void scale_weights_kernel(const float* __restrict__ W0, const float* __restrict__ s,

@@ -86,6 +86,8 @@ void launch_transpose_split(Ctx* c, const void* X, int is_bf16, long long rows, 
 void launch_finalize(Ctx* c, double damp_frac, int precondition);
 void launch_grid_fit(Ctx* c, const float* W0, int p, int bits, int gs, int symmetric, float* delta,
                      float* zero);
+void launch_grid_fit_mse(Ctx* c, const float* W0, int p, int bits, int gs, int symmetric, int points,
+                         double min_ratio, float* delta, float* zero);
 void launch_scale_weights(Ctx* c, const float* W0, int p);
 void launch_operand_scales(Ctx* c);   // fscal from diag(H)
 void launch_split_f64(Ctx* c, const double* src, int n, bf16* hi, bf16* lo, bf16* thi, bf16* tlo);

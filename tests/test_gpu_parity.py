@@ -441,3 +441,58 @@ def test_grid_refresh_parity(kw, attempts):
     with pytest.raises(B.AdmmqError) as e:
         sol.quantize_layer(W, spec.bits, 1, spec.symmetric, refresh_at=[3])
     assert e.value.status == B.ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------ MSE search for the clipping ratio (Sec. 3.4, App. D)
+@pytest.mark.parametrize("kw", [
+    dict(d_in=256, d_out=96, n_tokens=2048, bits=3, group_size=64),
+    dict(d_in=512, d_out=40, n_tokens=1536, bits=4, group_size=128, symmetric=True),
+    dict(d_in=264, d_out=70, n_tokens=3000, bits=2, group_size=0),              # one group per channel, ragged n
+    dict(d_in=384, d_out=33, n_tokens=1200, bits=3, group_size=384),           # group longer than the register path
+])
+def test_mse_clip_search_parity(kw):
+    spec = wl.small_case(**kw)
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(spec.d_in, spec.d_out, T_max=spec.T)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=spec.rho())
+    codes, scale, zero, rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, clip_points=100,
+                                                 clip_min_ratio=0.8)
+    assert sol.last_device_status() == B.OK
+    Wn = np64(W)
+    d_o, z_o = O.grid_fit_mse(Wn, spec.bits, spec.group_size, spec.symmetric, points=100, min_ratio=0.8)
+    d_g, z_g = np64(scale), np64(zero)
+    # The chosen candidate is an argmin over sums that can lie within rounding of each other: the grid must
+    # agree for almost every group, and where it does not the GPU's choice must be as good as the optimum.
+    same = np.isclose(d_g, d_o, rtol=1e-6, atol=0) & np.isclose(z_g, z_o, rtol=1e-6, atol=1e-12)
+    assert same.mean() >= 0.98, same.mean()
+    levels = (1 << spec.bits) - 1
+    gs = spec.d_in if spec.group_size in (0, spec.d_in) else spec.group_size
+    Wg = Wn.reshape(spec.d_out, spec.d_in // gs, gs)
+
+    def mse(d, z):
+        k = np.clip(np.rint((Wg - z[..., None]) / d[..., None]), 0, levels)
+        return ((z[..., None] + d[..., None] * k - Wg) ** 2).sum(axis=2)
+
+    e_g, e_o = mse(d_g, z_g), mse(d_o, z_o)
+    assert (e_g <= e_o * (1 + 1e-4) + 1e-30).all()
+    # every GPU grid is one of the candidates: ratio = Delta / Delta_minmax in [0.8, 1]
+    d_mm, _ = O.grid_fit(Wn, spec.bits, spec.group_size, spec.symmetric)
+    ratio = d_g / d_mm
+    assert (ratio >= 0.8 - 1e-6).all() and (ratio <= 1 + 1e-6).all()
+    assert (ratio < 0.999).mean() > 0.2                      # the search does clip on these weights
+    # the ADMM run on that grid matches the oracle's run on the same grid
+    H = oracle_hessian(spec, DEV)
+    ref = O.admm(H, Wn, spec.bits, spec.group_size, spec.symmetric, np.array(spec.rho()), grid=(d_g, z_g))
+    cg = codes.cpu().numpy()
+    assert (cg == ref.codes).mean() >= CODE_AGREEMENT
+    e_a = O.objective(H, Wn, O.dequantize(cg, d_g, z_g))
+    assert abs(e_a - O.objective(H, Wn, ref.Wq)) <= ERR_TOL * e_a
+    # one candidate is the min-max grid, bit for bit
+    _, s1, z1, _ = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, clip_points=1)
+    _, s0, z0, _ = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric)
+    assert torch.equal(s1, s0) and torch.equal(z1, z0)
+    with pytest.raises(B.AdmmqError):
+        sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, clip_points=100, clip_min_ratio=0.0)
