@@ -146,6 +146,11 @@ typedef struct {
                            r_i = 1 - (1 - clip_min_ratio) i / (clip_points - 1); each scales both ends of the group's
                            min-max range (symmetric: +-r max|w|), and the candidate with the smallest sum of squared
                            rounding errors of the group is kept (the largest ratio on ties). */
+  int fused_epilogue;   /* where the element update of Eq. 8-10 runs.  0 (default): the second product stores
+                           W^(t+1) - W_hat' and one row pass does projection, dual update, residual sums and the
+                           split of the next right-hand side (the faster of the two as measured on B200).
+                           1: inside the second product's epilogue, W never leaves the SM.  Same arithmetic per
+                           element, so both settings give the same codes. */
 } admmq_quant_cfg;
 typedef struct {
   double err_before;    /* Tr(E^T H E), E = W_q - W_hat, at entry (local search) / of the ADMM result */

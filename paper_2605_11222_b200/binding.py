@@ -45,7 +45,7 @@ class QuantCfg(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("bits", C.c_int), ("group_size", C.c_int),
                 ("symmetric", C.c_int), ("use_caller_grid", C.c_int), ("n_refresh", C.c_int),
                 ("h_refresh_iters", C.POINTER(C.c_int)), ("clip_points", C.c_int),
-                ("clip_min_ratio", C.c_double)]
+                ("clip_min_ratio", C.c_double), ("fused_epilogue", C.c_int)]
 
 
 class LsCfg(C.Structure):
@@ -212,7 +212,7 @@ class Solver:
     def quantize_layer(self, W0: torch.Tensor, bits: int, group_size: int = 0, symmetric: bool = False,
                        codes=None, scale=None, zero=None, Wq=None, resid=None, use_caller_grid=False,
                        report: bool = True, refresh_at: Sequence[int] = (), clip_points: int = 0,
-                       clip_min_ratio: float = 0.8):
+                       clip_min_ratio: float = 0.8, fused_epilogue: bool = False):
         p, n = W0.shape
         gs = n if group_size in (0, n) else group_size
         dev = W0.device
@@ -222,7 +222,7 @@ class Solver:
         iters = (C.c_int * max(1, len(refresh_at)))(*[int(t) for t in refresh_at])
         cfg = QuantCfg(C.sizeof(QuantCfg), bits, group_size, int(symmetric), int(use_caller_grid),
                        len(refresh_at), C.cast(iters, C.POINTER(C.c_int)) if len(refresh_at) else None,
-                       int(clip_points), float(clip_min_ratio))
+                       int(clip_points), float(clip_min_ratio), int(fused_epilogue))
         rep = Report()
         st = self.lib.admmq_quantize_layer(self.h, _ptr(W0), p, C.byref(cfg), _ptr(codes), _ptr(scale),
                                            _ptr(zero), _ptr(Wq), _ptr(resid),

@@ -435,12 +435,28 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
       w.ldc = n;
       if (w_update_products(ctx, p, t, w) != cudaSuccess) return ADMMQ_ERR_CUDA;
       launch_grid_refresh(c, e, p, cfg->bits, cfg->symmetric, t, d_scale, d_zero, refresh_flags);
-    } else if (w_update_products(ctx, p, t, e) != cudaSuccess) {
-      return ADMMQ_ERR_CUDA;
-    }
-    if (t + 1 < T) {
+      if (t + 1 < T) {
+        Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
+        launch_row_split(c, c->Y, p, c->R_hi, c->R_lo, c->rs_R);
+      }
+    } else if (cfg->fused_epilogue) {
+      // projection, dual update and residuals inside the second product's epilogue; the next right-hand side
+      // leaves it in fp32 and a row pass splits it into planes
+      if (w_update_products(ctx, p, t, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
+      if (t + 1 < T) {
+        Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
+        launch_row_split(c, c->Y, p, c->R_hi, c->R_lo, c->rs_R);
+      }
+    } else {
+      // the product stores z = W^(t+1) - W_hat'; one row pass does the element update and the plane split
+      EpiParams w = e;
+      w.kind = EPI_STORE;
+      w.C = c->Y;
+      w.ldc = n;
+      if (w_update_products(ctx, p, t, w) != cudaSuccess) return ADMMQ_ERR_CUDA;
       Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
-      launch_row_split(c, c->Y, p, c->R_hi, c->R_lo, c->rs_R);
+      w.kind = EPI_ADMM;
+      launch_admm_rows(c, w, p, c->R_hi, c->R_lo, c->rs_R);
     }
   }
   if (d_resid) launch_reduce_partials(c, T, d_resid);

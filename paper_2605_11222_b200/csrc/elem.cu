@@ -644,6 +644,85 @@ __global__ void __launch_bounds__(256) admm_elementwise_kernel(EpiParams P, long
   }
 }
 
+// The ADMM element update (Eq. 8-10) of whole rows from the stored product z = W^(t+1) - W_hat' (in P.C), merged
+// with the split of the next right-hand side into its scaled fp16 planes: the row of R = D - V/rho' - W_hat'
+// stays in shared memory between the two halves, so it makes no trip through memory of its own.
+__global__ void __launch_bounds__(ROW_THREADS)
+admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restrict__ lo,
+                float* __restrict__ row_inv) {
+  extern __shared__ float rowbuf[];
+  __shared__ float scratch[32];
+  float r2 = 0.f, s2 = 0.f;
+  const int gs = P.group_size;
+  for (int j = blockIdx.x; j < p; j += gridDim.x) {
+    const size_t base = (size_t)j * n;
+    const float* dlt = P.delta + (size_t)j * P.n_groups;
+    const float* zr = P.zero + (size_t)j * P.n_groups;
+    float m = 0.0f;
+    for (int i = threadIdx.x * 4; i < n; i += ROW_THREADS * 4) {          // n is a multiple of 8
+      const float4 z = *reinterpret_cast<const float4*>(P.C + base + i);
+      const float4 wh = *reinterpret_cast<const float4*>(P.Whs + base + i);
+      const float4 v = *reinterpret_cast<const float4*>(P.V + base + i);
+      const float4 sv = *reinterpret_cast<const float4*>(P.s + i);
+      const float4 si = *reinterpret_cast<const float4*>(P.inv_s + i);
+      uchar4 k = make_uchar4(0, 0, 0, 0);
+      if (!P.first_iter) k = *reinterpret_cast<const uchar4*>(P.codes + base + i);
+      const int g0 = i / gs, g3 = (i + 3) / gs;
+      const float d0 = dlt[g0], z0 = zr[g0], id0 = __frcp_rn(d0);
+      AdmmElem e0 = admm_elem(z.x, wh.x, v.x, k.x, sv.x, si.x, d0, id0, z0, P);
+      AdmmElem e1, e2, e3;
+      if (g3 == g0) {
+        e1 = admm_elem(z.y, wh.y, v.y, k.y, sv.y, si.y, d0, id0, z0, P);
+        e2 = admm_elem(z.z, wh.z, v.z, k.z, sv.z, si.z, d0, id0, z0, P);
+        e3 = admm_elem(z.w, wh.w, v.w, k.w, sv.w, si.w, d0, id0, z0, P);
+      } else {
+        const int g1 = (i + 1) / gs, g2 = (i + 2) / gs;
+        e1 = admm_elem(z.y, wh.y, v.y, k.y, sv.y, si.y, dlt[g1], __frcp_rn(dlt[g1]), zr[g1], P);
+        e2 = admm_elem(z.z, wh.z, v.z, k.z, sv.z, si.z, dlt[g2], __frcp_rn(dlt[g2]), zr[g2], P);
+        e3 = admm_elem(z.w, wh.w, v.w, k.w, sv.w, si.w, dlt[g3], __frcp_rn(dlt[g3]), zr[g3], P);
+      }
+      *reinterpret_cast<uchar4*>(P.codes + base + i) = make_uchar4(e0.code, e1.code, e2.code, e3.code);
+      *reinterpret_cast<float4*>(P.V + base + i) = make_float4(e0.v_new, e1.v_new, e2.v_new, e3.v_new);
+      *reinterpret_cast<float4*>(rowbuf + i) = make_float4(e0.r_next, e1.r_next, e2.r_next, e3.r_next);
+      m = fmaxf(fmaxf(fabsf(e0.r_next), fabsf(e1.r_next)), fmaxf(m, fmaxf(fabsf(e2.r_next), fabsf(e3.r_next))));
+      r2 += (e0.dr2 + e1.dr2) + (e2.dr2 + e3.dr2);
+      s2 += (e0.ds2 + e1.ds2) + (e2.ds2 + e3.ds2);
+    }
+    m = block_max(m, scratch);
+    float inv;
+    const float sc = pow2_scale_for(m, &inv);
+    if (threadIdx.x == 0) row_inv[j] = inv;
+    for (int i = threadIdx.x * 8; i < n; i += ROW_THREADS * 8) {
+      __align__(16) __half hh[8];
+      __align__(16) __half ll[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) split_f16(rowbuf[i + e] * sc, hh[e], ll[e]);
+      *reinterpret_cast<uint4*>(hi + base + i) = *reinterpret_cast<const uint4*>(hh);
+      *reinterpret_cast<uint4*>(lo + base + i) = *reinterpret_cast<const uint4*>(ll);
+    }
+    __syncthreads();
+  }
+  r2 = block_sum(r2, scratch);
+  s2 = block_sum(s2, scratch);
+  if (threadIdx.x == 0) {
+    P.partials[2 * blockIdx.x + 0] = r2;
+    P.partials[2 * blockIdx.x + 1] = s2;
+  }
+}
+
+void launch_admm_rows(Ctx* c, const EpiParams& P, int p, bf16* hi, bf16* lo, float* row_inv) {
+  const size_t smem = (size_t)c->n * sizeof(float);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaFuncSetAttribute(admm_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+    attr_set = true;
+  }
+  int blocks = row_pass_blocks(c, p, smem);
+  if (blocks > c->partial_slots) blocks = c->partial_slots;
+  admm_row_kernel<<<blocks, ROW_THREADS, smem, c->stream>>>(P, p, c->n, hi, lo, row_inv);
+  LAUNCH(c);
+}
+
 void launch_grid_refresh(Ctx* c, const EpiParams& P, int p, int bits, int symmetric, int iter, float* delta,
                          float* zero, int* flags) {
   const int n = c->n, gs = P.group_size, ng = n / gs;

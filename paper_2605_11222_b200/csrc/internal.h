@@ -86,6 +86,7 @@ void launch_transpose_split(Ctx* c, const void* X, int is_bf16, long long rows, 
 void launch_finalize(Ctx* c, double damp_frac, int precondition);
 void launch_grid_fit(Ctx* c, const float* W0, int p, int bits, int gs, int symmetric, float* delta,
                      float* zero);
+void launch_admm_rows(Ctx* c, const EpiParams& P, int p, bf16* hi, bf16* lo, float* row_inv);
 void launch_grid_fit_mse(Ctx* c, const float* W0, int p, int bits, int gs, int symmetric, int points,
                          double min_ratio, float* delta, float* zero);
 void launch_scale_weights(Ctx* c, const float* W0, int p);

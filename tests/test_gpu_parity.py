@@ -496,3 +496,26 @@ def test_mse_clip_search_parity(kw):
     assert torch.equal(s1, s0) and torch.equal(z1, z0)
     with pytest.raises(B.AdmmqError):
         sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, clip_points=100, clip_min_ratio=0.0)
+
+
+def test_fused_and_row_pass_element_update_agree():
+    """The element update of Eq. 8-10 inside the product's epilogue and in the row pass is the same arithmetic
+    on the same accumulators: codes, grid and residual trace are identical."""
+    spec = wl.small_case(d_in=520, d_out=200, n_tokens=2048, bits=3, group_size=0)
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(spec.d_in, spec.d_out, T_max=spec.T)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=spec.rho())
+    out = []
+    for fused in (False, True):
+        resid = torch.zeros(spec.T, 2, device=DEV)
+        codes, scale, zero, rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, resid=resid,
+                                                     fused_epilogue=fused)
+        assert sol.last_device_status() == B.OK
+        out.append((codes.clone(), scale.clone(), zero.clone(), resid.cpu().numpy(), rep.err_before))
+    assert torch.equal(out[0][0], out[1][0])
+    assert torch.equal(out[0][1], out[1][1]) and torch.equal(out[0][2], out[1][2])
+    assert np.allclose(out[0][3], out[1][3], rtol=1e-5, atol=0)
+    assert abs(out[0][4] - out[1][4]) <= 1e-12 * out[0][4]     # the error sum is accumulated atomically
