@@ -114,17 +114,15 @@ __device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t adesc, uint
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// 32 consecutive accumulator columns of this warp's 32 lanes (lane = row), issued without waiting.
-__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&v)[32]) {
+// 8 consecutive accumulator columns of this warp's 32 lanes (lane = row), issued without waiting.  The
+// drain uses this narrow form on purpose: a thread already holds 64 running sums, and with 16 or 32
+// temporaries on top the worker loop spills (the register file gives 96 registers per thread at 18 warps),
+// which cost 12 % of the launch.
+__device__ __forceinline__ void tc_ld8_issue(uint32_t taddr, uint32_t (&v)[8]) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),
-        "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]),
-        "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]),
-        "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      "tcgen05.ld.sync.aligned.32x32b.x8.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
       : "r"(taddr)
       : "memory");
 }
@@ -485,18 +483,28 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
         if (mine) {
           const uint32_t taddr = tmem_base + (uint32_t)pb * BN + (uint32_t)(cq * COLS_PER_THREAD) +
                                  ((uint32_t)(q * 32) << 16);
-          uint32_t v[32];
-          tc_ld32_issue(taddr, v);
-          tc_ld_wait();
+          // two alternating groups of 8 columns: the adds of one group run while the next load is in flight
+          uint32_t va[8], vb[8];
+          tc_ld8_issue(taddr, va);
 #pragma unroll
-          for (int e = 0; e < 32; ++e) sums[e] += __uint_as_float(v[e]);
-          tc_ld32_issue(taddr + 32, v);
+          for (int h = 0; h < 3; ++h) {
+            tc_ld8_issue(taddr + 16 * h + 8, vb);
+            tc_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sums[16 * h + e] += __uint_as_float(va[e]);
+            tc_ld8_issue(taddr + 16 * h + 16, va);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sums[16 * h + 8 + e] += __uint_as_float(vb[e]);
+          }
+          tc_ld8_issue(taddr + 56, vb);
           tc_ld_wait();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(pempty0 + 8 * pb);    // the partial is in registers: buffer free
 #pragma unroll
-          for (int e = 0; e < 32; ++e) sums[32 + e] += __uint_as_float(v[e]);
+          for (int e = 0; e < 8; ++e) sums[48 + e] += __uint_as_float(va[e]);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) sums[56 + e] += __uint_as_float(vb[e]);
         } else {
           tc_fence_before();
           if (lane == 0) mbar_arrive(pempty0 + 8 * pb);
