@@ -167,8 +167,11 @@ def run_reference(args, spec, wl):
 
 # ---------------------------------------------------------------------------------------------------
 def run_stack(args, wl):
-    """Config 5: every linear layer of the first B decoder blocks, each quantized once from its own seeded
-    calibration set (generated on the device, generation timed separately)."""
+    """Config 5: every linear layer of the first B decoder blocks, each quantized once from a seeded calibration
+    set generated on the device (generation timed separately).  Default: every layer has its own calibration set
+    and factorisation.  With --shared-h the projections that read the same activations in a decoder block
+    (q/k/v; gate/up) share one calibration set, one Hessian and one factorisation, and their weights are stacked
+    into one call: output channels are independent problems given H."""
     from paper_2605_11222_b200 import binding as B
     dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
     torch.cuda.set_device(dev)
@@ -177,16 +180,26 @@ def run_stack(args, wl):
         import dataclasses
         layers = [dataclasses.replace(l, n_tokens=args.tokens) for l in layers]
     T = layers[0].T
+    # groups of layers solved in one call: [q, k, v], [o], [gate, up], [down] per block when H is shared
+    groups = []
+    if args.shared_h:
+        per_block = 7
+        for b in range(0, len(layers), per_block):
+            blk = layers[b:b + per_block]
+            groups += [blk[0:3], blk[3:4], blk[4:6], blk[6:7]]
+    else:
+        groups = [[l] for l in layers]
     solvers = {}
-    for n in sorted({l.d_in for l in layers}):
-        solvers[n] = B.Solver(n, max(l.d_out for l in layers if l.d_in == n), T_max=T, device=dev)
+    for n in sorted({g[0].d_in for g in groups}):
+        solvers[n] = B.Solver(n, max(sum(l.d_out for l in g) for g in groups if g[0].d_in == n), T_max=T, device=dev)
     per_shape, gen_s, solve_ms, moves = {}, 0.0, 0.0, 0
     torch.cuda.synchronize(dev)
     t_wall = time.perf_counter()
-    for spec in layers:
+    for grp in groups:
+        spec = grp[0]                                       # its calibration set serves the whole group
         sol = solvers[spec.d_in]
         t0 = time.perf_counter()
-        W = wl.gen_weight(spec, dev)
+        W = torch.cat([wl.gen_weight(l, dev) for l in grp], dim=0) if len(grp) > 1 else wl.gen_weight(spec, dev)
         Xs = [wl.gen_x_chunk(spec, c, dev) for c in range(spec.n_chunks)]
         torch.cuda.synchronize(dev)
         gen_s += time.perf_counter() - t0
@@ -203,7 +216,7 @@ def run_stack(args, wl):
         ms = e0.elapsed_time(e1)
         solve_ms += ms
         moves += rep.moves
-        key = f"{spec.d_in}x{spec.d_out}"
+        key = f"{spec.d_in}x{W.shape[0]}"
         a = per_shape.setdefault(key, [0, 0.0])
         a[0] += 1
         a[1] += ms
@@ -213,9 +226,10 @@ def run_stack(args, wl):
         "metric": "admmq_stack_solve_time", "value": solve_ms / 1e3, "unit": "s", "n_gpus": 1,
         "higher_is_better": False, "data": "synthetic", "dtype": "f16x2-split (fp32 accumulate)",
         "config": {"workload": f"cfg5 first {args.stack_blocks} of 36 blocks", "layers": len(layers),
+                   "calls": len(groups), "shared_h": bool(args.shared_h),
                    "n_tokens": layers[0].n_tokens, "T": T, "bits": layers[0].bits, "group_size": layers[0].group_size},
         "wall_s_with_generation": wall, "generation_s": gen_s, "local_search_moves": moves,
-        "per_shape": {k: {"layers": v[0], "s_per_layer": v[1] / v[0] / 1e3} for k, v in per_shape.items()}}))
+        "per_shape": {k: {"calls": v[0], "s_per_call": v[1] / v[0] / 1e3} for k, v in per_shape.items()}}))
     return 0
 
 
@@ -233,6 +247,8 @@ def main():
     ap.add_argument("--stack-blocks", type=int, default=0,
                     help="instead of one layer: quantize the first B decoder blocks of config 5 (7 layers each, "
                          "36 = the whole stack), every layer once, and report the wall time")
+    ap.add_argument("--shared-h", action="store_true",
+                    help="with --stack-blocks: q/k/v and gate/up of a block share one Hessian and factorisation")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()

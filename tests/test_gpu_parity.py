@@ -519,3 +519,32 @@ def test_fused_and_row_pass_element_update_agree():
     assert torch.equal(out[0][1], out[1][1]) and torch.equal(out[0][2], out[1][2])
     assert np.allclose(out[0][3], out[1][3], rtol=1e-5, atol=0)
     assert abs(out[0][4] - out[1][4]) <= 1e-12 * out[0][4]     # the error sum is accumulated atomically
+
+
+def test_stacked_layers_share_one_factorisation():
+    """Projections that read the same activations share H: stacking their weights into one call gives, channel
+    by channel, exactly what separate calls on the same factorisation give (output channels are independent
+    problems given H; Sec. 3.1)."""
+    spec = wl.small_case(d_in=512, d_out=320, n_tokens=2048, bits=4, group_size=128)
+    sizes = [192, 64, 64]                                   # a q / k / v split
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(spec.d_in, spec.d_out, T_max=spec.T)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=spec.rho())
+    codes, scale, zero, rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric)
+    rep_ls, _ = sol.local_search(W, spec.bits, spec.group_size, codes, scale, zero)
+    r0, err_sum, err_ls_sum = 0, 0.0, 0.0
+    for p_i in sizes:
+        Wi = W[r0:r0 + p_i].contiguous()
+        ci, si, zi, ri = sol.quantize_layer(Wi, spec.bits, spec.group_size, spec.symmetric)
+        assert torch.equal(si, scale[r0:r0 + p_i]) and torch.equal(zi, zero[r0:r0 + p_i])
+        ri_ls, _ = sol.local_search(Wi, spec.bits, spec.group_size, ci, si, zi)
+        assert torch.equal(ci, codes[r0:r0 + p_i])
+        err_sum += ri.err_before
+        err_ls_sum += ri_ls.err_after
+        r0 += p_i
+    assert abs(err_sum - rep.err_before) <= 1e-9 * rep.err_before
+    assert abs(err_ls_sum - rep_ls.err_after) <= 1e-9 * rep_ls.err_after
+    assert sol.last_device_status() == B.OK
