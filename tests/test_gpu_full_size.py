@@ -207,3 +207,61 @@ def test_cfg3_down_proj_shape_w_update_sampled_rows():
     rel = np.linalg.norm(np64(Wg[rows]) - Wo) / np.linalg.norm(Wo)
     assert rel <= W_UPDATE_TOL, rel
     assert sol.last_device_status() == B.OK
+
+
+def _solve_and_compare_sampled_channels(spec, rows):
+    """One full-size layer on the GPU (Hessian -> factor -> ADMM -> local search) and the oracle's complete run
+    of a few of its output channels on the GPU's damped fp32 Hessian."""
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(spec.d_in, spec.d_out, T_max=spec.T)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=spec.rho())
+    Hd, _ = sol.get_hessian()
+    codes, scale, zero, rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric)
+    codes_admm = codes.clone()
+    rep_ls, st = sol.local_search(W, spec.bits, spec.group_size, codes, scale, zero)
+    assert st == B.OK and sol.last_device_status() == B.OK
+    H = np64(Hd)
+    Wn = np64(W)[rows]
+    res = O.quantize_layer(H, Wn, spec.bits, spec.group_size, spec.symmetric, np.array(spec.rho()))
+    ca = codes_admm[rows].cpu().numpy()
+    cf = codes[rows].cpu().numpy()
+    assert np.allclose(np64(scale)[rows], res.admm.delta, rtol=2e-7, atol=0)
+    assert (ca == res.admm.codes).mean() >= CODE_AGREEMENT, (ca == res.admm.codes).mean()
+    assert (cf == res.ls.codes).mean() >= CODE_AGREEMENT, (cf == res.ls.codes).mean()
+    e_a = O.objective(H, Wn, O.dequantize(ca, res.admm.delta, res.admm.z0))
+    e_f = O.objective(H, Wn, O.dequantize(cf, res.admm.delta, res.admm.z0))
+    assert abs(e_a - res.err_admm) <= ERR_TOL * res.err_admm
+    assert abs(e_f - res.err_final) <= ERR_TOL * res.err_final
+    assert int(codes.max()) <= (1 << spec.bits) - 1
+    assert rep_ls.err_after <= rep.err_before * (1 + 1e-6)
+    return rep, rep_ls
+
+
+def test_cfg3_gate_proj_sampled_channels_against_oracle():
+    """Config 3, gate_proj: 4096 -> 12288 (three times as many output channels as inputs), W3 g128, T = 300."""
+    spec = wl.config3()[0]
+    _solve_and_compare_sampled_channels(spec, [0, 4095, 4096, 8191, 10000, spec.d_out - 1])
+
+
+def test_cfg4_k_proj_sampled_channels_against_oracle():
+    """Config 4, k_proj: rotated inputs and weights, 4096 -> 1024, W2 symmetric per-channel grid, T = 500
+    (the penalty grows to ~5e19: the late iterations must leave the codes untouched)."""
+    spec = wl.config4()[0]
+    _solve_and_compare_sampled_channels(spec, [0, 1, 255, 512, 777, spec.d_out - 1])
+
+
+def test_cfg5_q_proj_sampled_channels_against_oracle():
+    """Config 5, q_proj of the first block: 131072 tokens, W4 g128, T = 300."""
+    spec = wl.config5(n_blocks=1)[0]
+    _solve_and_compare_sampled_channels(spec, [0, 63, 2048, 3001, spec.d_out - 1])
+
+
+def test_cfg3_down_proj_sampled_channels_against_oracle():
+    """Config 3, down_proj: d_in = 12288 (blocked reduction, 48 elements per thread in the tridiagonal solve),
+    post-SiLU-like activations, W3 g128, T = 300.  The oracle's eigendecomposition of the 12288 x 12288 matrix
+    takes a few minutes of host time; four channels keep the rest short."""
+    spec = wl.config3()[2]
+    _solve_and_compare_sampled_channels(spec, [0, 1234, 2048, spec.d_out - 1])
