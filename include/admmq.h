@@ -128,8 +128,7 @@ admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg);
  * Grid refresh: at the listed iterations, until one attempt is accepted, (Delta, z0) are refitted by the same
  * rule on the unscaled projection target (W + V/rho)/s, the target is projected on both grids, and the new grid
  * replaces the old one (in d_scale / d_zero) iff ||D_new - W~||_F^2 <= ||D_old - W~||_F^2 over the whole matrix;
- * the dual update then uses D_new.  Needs a group size >= 2.  At such an iteration W^(t+1) makes one trip through
- * memory (the epilogue is not fused).
+ * the dual update then uses D_new.  Needs a group size >= 2.
  * h_report NULL: nothing is synchronised.  Non-NULL: the call synchronises, fills the report and
  * returns the device status. */
 typedef struct {
@@ -244,10 +243,11 @@ typedef enum {
   ADMMQ_T_FACTOR = 2,           /* finalisation + tridiagonal reduction + Q + stage factors (step 2) */
   ADMMQ_T_WUPDATE_PRODUCT1 = 3, /* Y = R Q                                                (step 3) */
   ADMMQ_T_TRIDIAG_SOLVE = 4,    /* (T/rho + I)^{-1} row solve                             (step 3) */
-  ADMMQ_T_WUPDATE_PRODUCT2 = 5, /* Z = Y' Q^T with the fused projection/dual/residual epilogue */
+  ADMMQ_T_WUPDATE_PRODUCT2 = 5, /* Z = Y' Q^T (with fused_epilogue: plus projection/dual/residuals) (step 3) */
   ADMMQ_T_GRADIENT_PRODUCT = 6, /* g = E H                                                (step 4) */
   ADMMQ_T_LOCAL_SEARCH = 7,     /* move loop kernel                                       (step 4) */
-  ADMMQ_T_ROW_SPLIT = 8,        /* next right-hand side -> scaled fp16 operand planes     (step 3) */
+  ADMMQ_T_ROW_SPLIT = 8,        /* row pass: projection, dual update, residuals (unless fused into product 2) and
+                                   next right-hand side -> scaled fp16 operand planes     (step 3) */
   ADMMQ_T_KINDS = 9
 } admmq_timing_kind;
 admmq_status admmq_set_timing(admmq_ctx* ctx, int on);
