@@ -43,7 +43,7 @@ struct TrbArgs {
   double* beta;
   double* colbuf;     // [n] current column, brought up to date
   double* ybuf;       // [n] A22 v
-  double* part;       // [grid][TB_PART]
+  double* part;       // [TB_PART][grid]: the partials of one inner product are contiguous
   double* normpart;   // [grid]
   double* Vg;         // [n][TB_NB] finished panel, row-major
   double* Wg;         // [n][TB_NB]
@@ -191,14 +191,14 @@ __global__ void __launch_bounds__(TB_THREADS, 1) tridiag_blocked_kernel(TrbArgs 
         double s = 0.0;
         if (tid < i) {
           for (int t = 0; t < nr; ++t) s += Ws[(size_t)(tA + t) * TB_LDP + tid] * v[c + (tA + t) * G];
-          a.part[(size_t)c * TB_PART + tid] = s;
+          a.part[(size_t)tid * G + c] = s;
         } else if (tid < 2 * i) {
           const int j = tid - i;
           for (int t = 0; t < nr; ++t) s += Vs[(size_t)(tA + t) * TB_LDP + j] * v[c + (tA + t) * G];
-          a.part[(size_t)c * TB_PART + TB_NB + j] = s;
+          a.part[(size_t)(TB_NB + j) * G + c] = s;
         } else {
           for (int t = 0; t < nr; ++t) s += yown[tA + t] * v[c + (tA + t) * G];
-          a.part[(size_t)c * TB_PART + 2 * TB_NB] = s;
+          a.part[(size_t)(2 * TB_NB) * G + c] = s;
         }
       }
       grid.sync();
@@ -207,7 +207,7 @@ __global__ void __launch_bounds__(TB_THREADS, 1) tridiag_blocked_kernel(TrbArgs 
         const bool need = (o < TB_NB) ? (o < i) : (o < 2 * TB_NB ? (o - TB_NB < i) : true);
         if (!need) continue;
         double s = 0.0;
-        for (int b = lane; b < G; b += 32) s += __ldcg(a.part + (size_t)b * TB_PART + o);
+        for (int b = lane; b < G; b += 32) s += __ldcg(a.part + (size_t)o * G + b);
         s = warp_sum(s);
         if (lane == 0) red[o] = s;
       }
