@@ -31,7 +31,7 @@ namespace admmq {
 // Output: td/te (diagonal / off-diagonal of T), reflector k in A[k, k+1:], beta[k].
 // ------------------------------------------------------------------------------------------------
 constexpr int TRD_THREADS = 1024;
-constexpr int TRD_BLOCKED_FROM = 6144;
+constexpr int TRD_BLOCKED_FROM = 4096;
 constexpr int TRD_PSUM = 512;
 
 struct TrdArgs {
@@ -234,7 +234,8 @@ static int trd_cap(int n, int C) {
 cudaError_t tridiag_reduce(Ctx* c) {
   const int n = c->n;
   // The blocked kernel halves the traffic per column but pays a second grid barrier and more serial
-  // work per column; measured, it wins from about n = 6000 (n = 4096: 100 ms vs 84 ms; n = 12288: 1.4 s vs 2.0 s).
+  // work per column; measured, it wins from n = 4096 on (whole factorisation at n = 4096: 98.7 ms vs 102.0 ms;
+  // reduction alone at n = 12288: 1.36 s vs 2.0 s).
   if (n >= TRD_BLOCKED_FROM) {
     const cudaError_t eb = tridiag_reduce_blocked(c);
     if (eb != cudaErrorInvalidConfiguration) return eb;    // too large for its shared memory: fall through
