@@ -451,7 +451,7 @@ def main():
                  for k, v in timing.items()}
 
     cpu_baseline = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:            # the oracle is timed at N = 1 only
         est, desc, threads = oracle_sample_seconds(spec, wl)
         cpu_baseline = {"value": est, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
 
