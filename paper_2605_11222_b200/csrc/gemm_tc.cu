@@ -126,6 +126,16 @@ __device__ __forceinline__ void tc_ld8_issue(uint32_t taddr, uint32_t (&v)[8]) {
       : "r"(taddr)
       : "memory");
 }
+// sums[0..7] += v[0..7] as four packed fp32 additions (round to nearest, the same result as eight scalar ones).
+__device__ __forceinline__ void add8(float* sums, const uint32_t (&v)[8]) {
+#pragma unroll
+  for (int e = 0; e < 8; e += 2) {
+    const float2 r = __fadd2_rn(make_float2(sums[e], sums[e + 1]),
+                                make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])));
+    sums[e] = r.x;
+    sums[e + 1] = r.y;
+  }
+}
 __device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major tile with 128-byte rows and 128B swizzle: groups of
@@ -490,21 +500,17 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
           for (int h = 0; h < 3; ++h) {
             tc_ld8_issue(taddr + 16 * h + 8, vb);
             tc_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 8; ++e) sums[16 * h + e] += __uint_as_float(va[e]);
+            add8(sums + 16 * h, va);
             tc_ld8_issue(taddr + 16 * h + 16, va);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) sums[16 * h + 8 + e] += __uint_as_float(vb[e]);
+            add8(sums + 16 * h + 8, vb);
           }
           tc_ld8_issue(taddr + 56, vb);
           tc_ld_wait();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(pempty0 + 8 * pb);    // the partial is in registers: buffer free
-#pragma unroll
-          for (int e = 0; e < 8; ++e) sums[48 + e] += __uint_as_float(va[e]);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) sums[56 + e] += __uint_as_float(vb[e]);
+          add8(sums + 48, va);
+          add8(sums + 56, vb);
         } else {
           tc_fence_before();
           if (lane == 0) mbar_arrive(pempty0 + 8 * pb);
