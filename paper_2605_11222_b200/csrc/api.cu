@@ -375,6 +375,16 @@ static cudaError_t w_update_products(admmq_ctx* a, int p, int stage, const EpiPa
   return product(c, op_Y(c), op_Q(c), p, n, n, epi);
 }
 
+// Two events for the device time of a call; destroyed on every exit path.
+struct CallEvents {
+  cudaEvent_t a = nullptr, b = nullptr;
+  bool create() { return cudaEventCreate(&a) == cudaSuccess && cudaEventCreate(&b) == cudaSuccess; }
+  ~CallEvents() {
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+  }
+};
+
 admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, const admmq_quant_cfg* cfg,
                                   unsigned char* d_codes, float* d_scale, float* d_zero, float* d_Wq,
                                   float* d_resid, admmq_report* h_report) {
@@ -388,10 +398,10 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   if (cfg->n_refresh > 0 && group_of(ctx->c.n, cfg->group_size) < 2) return ADMMQ_ERR_UNSUPPORTED;
   Ctx* c = &ctx->c;
   const int n = c->n, p = d_out, gs = group_of(n, cfg->group_size), T = c->T;
-  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  CallEvents ev;
   if (h_report) {
-    if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return ADMMQ_ERR_CUDA;
-    cudaEventRecord(ev0, c->stream);
+    if (!ev.create()) return ADMMQ_ERR_CUDA;
+    cudaEventRecord(ev.a, c->stream);
   }
   if (!cfg->use_caller_grid) {
     if (cfg->clip_points > 0)
@@ -463,16 +473,14 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   if (d_Wq) launch_dequant(c, p, gs, d_codes, d_scale, d_zero, d_Wq);
   if (cudaGetLastError() != cudaSuccess) return ADMMQ_ERR_CUDA;
   if (!h_report) return ADMMQ_OK;
-  cudaEventRecord(ev1, c->stream);
+  cudaEventRecord(ev.b, c->stream);
   memset(h_report, 0, sizeof(*h_report));
   if (gradient(ctx, d_W0, p, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
   launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 1);
   st = read_status(ctx);
   double err = 0.0;
   cudaMemcpy(&err, c->scal + 1, sizeof(double), cudaMemcpyDeviceToHost);
-  cudaEventElapsedTime(&h_report->ms, ev0, ev1);
-  cudaEventDestroy(ev0);
-  cudaEventDestroy(ev1);
+  cudaEventElapsedTime(&h_report->ms, ev.a, ev.b);
   int flags[2] = {0, 0};
   cudaMemcpy(flags, refresh_flags, sizeof(flags), cudaMemcpyDeviceToHost);
   h_report->err_before = err;
@@ -520,10 +528,10 @@ admmq_status admmq_local_search(admmq_ctx* ctx, const float* d_W0, int d_out, co
   Ctx* c = &ctx->c;
   const int n = c->n, p = d_out, gs = group_of(n, cfg->group_size);
   const long long cap = cfg->max_moves_per_col > 0 ? cfg->max_moves_per_col : 8LL * n;
-  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  CallEvents ev;
   if (h_report) {
-    if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return ADMMQ_ERR_CUDA;
-    cudaEventRecord(ev0, c->stream);
+    if (!ev.create()) return ADMMQ_ERR_CUDA;
+    cudaEventRecord(ev.a, c->stream);
   }
   if (gradient(ctx, d_W0, p, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
   if (h_report) launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 1);
@@ -536,7 +544,7 @@ admmq_status admmq_local_search(admmq_ctx* ctx, const float* d_W0, int d_out, co
       return ADMMQ_ERR_CUDA;
   }
   if (!h_report) return ADMMQ_OK;
-  cudaEventRecord(ev1, c->stream);
+  cudaEventRecord(ev.b, c->stream);
   memset(h_report, 0, sizeof(*h_report));
   if (gradient(ctx, d_W0, p, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
   launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 2);
@@ -547,9 +555,7 @@ admmq_status admmq_local_search(admmq_ctx* ctx, const float* d_W0, int d_out, co
   cudaMemcpy(errs, c->scal + 1, 2 * sizeof(double), cudaMemcpyDeviceToHost);
   cudaMemcpy(&moves, ctx->d_moves, sizeof(long long), cudaMemcpyDeviceToHost);
   cudaMemcpy(&capped, ctx->d_capped, sizeof(int), cudaMemcpyDeviceToHost);
-  cudaEventElapsedTime(&h_report->ms, ev0, ev1);
-  cudaEventDestroy(ev0);
-  cudaEventDestroy(ev1);
+  cudaEventElapsedTime(&h_report->ms, ev.a, ev.b);
   h_report->err_before = errs[0];
   h_report->err_after = errs[1];
   h_report->moves = moves;
@@ -570,10 +576,10 @@ admmq_status admmq_pair_swap(admmq_ctx* ctx, const float* d_W0, int d_out, const
   if (cfg->rounds > 0 && cfg->batch > 0 && (!cfg->d_pairs || !aligned16(cfg->d_pairs))) return ADMMQ_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
   const int n = c->n, p = d_out, gs = group_of(n, cfg->group_size);
-  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  CallEvents ev;
   if (h_report) {
-    if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return ADMMQ_ERR_CUDA;
-    cudaEventRecord(ev0, c->stream);
+    if (!ev.create()) return ADMMQ_ERR_CUDA;
+    cudaEventRecord(ev.a, c->stream);
   }
   if (gradient(ctx, d_W0, p, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
   if (h_report) launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 1);
@@ -585,7 +591,7 @@ admmq_status admmq_pair_swap(admmq_ctx* ctx, const float* d_W0, int d_out, const
                           ctx->d_capped) != cudaSuccess)
       return ADMMQ_ERR_CUDA;
   if (!h_report) return ADMMQ_OK;
-  cudaEventRecord(ev1, c->stream);
+  cudaEventRecord(ev.b, c->stream);
   memset(h_report, 0, sizeof(*h_report));
   if (gradient(ctx, d_W0, p, gs, d_codes, d_scale, d_zero) != cudaSuccess) return ADMMQ_ERR_CUDA;
   launch_objective_dot(c, d_W0, p, gs, d_codes, d_scale, d_zero, c->Y, c->scal + 2);
@@ -596,9 +602,7 @@ admmq_status admmq_pair_swap(admmq_ctx* ctx, const float* d_W0, int d_out, const
   cudaMemcpy(errs, c->scal + 1, 2 * sizeof(double), cudaMemcpyDeviceToHost);
   cudaMemcpy(&moves, ctx->d_moves, sizeof(long long), cudaMemcpyDeviceToHost);
   cudaMemcpy(&rounds_applied, ctx->d_capped, sizeof(int), cudaMemcpyDeviceToHost);
-  cudaEventElapsedTime(&h_report->ms, ev0, ev1);
-  cudaEventDestroy(ev0);
-  cudaEventDestroy(ev1);
+  cudaEventElapsedTime(&h_report->ms, ev.a, ev.b);
   h_report->err_before = errs[0];
   h_report->err_after = errs[1];
   h_report->moves = moves;
