@@ -52,11 +52,11 @@ def _check_factor(sol, H, s, tol_orth=1e-10, tol_rec=1e-10):
     assert te[-1].item() == 0.0
 
 
-@pytest.mark.parametrize("n", [8, 72, 264, 1000, 4096, 6144, 12288, 14336])
+@pytest.mark.parametrize("n", [8, 72, 264, 1000, 4096, 4104, 6144, 12288, 14336])
 def test_factorisation_properties(n):
     """The one-time factorisation at sizes that cover every code path: one partial reflector block,
     ragged blocks (one-pass reduction), the benchmark sizes (4096, 12288: blocked reduction, also taken at
-    6144), and the largest supported size, where the one-pass reduction works on column chunks."""
+    6144 and at 4104, which is no multiple of the segment and panel widths), and the largest supported size, where the one-pass reduction works on column chunks."""
     p = 8
     N = 2 * wl.CHUNK_ROWS if n >= 4096 else 3 * n + 40
     spec = wl.small_case(n, p, N, group_size=0, T=2)
