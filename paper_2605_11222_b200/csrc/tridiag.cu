@@ -504,6 +504,7 @@ cudaError_t tridiag_form_qt(Ctx* c) {
 // i = t * ept + e (thread t, e-th element of its segment) at [e * SOLVE_THREADS + t].
 // ------------------------------------------------------------------------------------------------
 constexpr int SOLVE_THREADS = 256;
+constexpr int SOLVE_ROWS = 2;               // rows solved together by the register-resident kernel
 
 // elements per thread of the solve kernel: n / 256 rounded up to a multiple of 8 (16-byte plane stores)
 int solve_ept(int n) { return (((n + SOLVE_THREADS - 1) / SOLVE_THREADS) + 7) & ~7; }
@@ -690,6 +691,208 @@ tridiag_solve_kernel(const float* __restrict__ Y, int p, int n, const float* __r
   }
 }
 
+// The same solve for R rows at a time, for d_in <= 4096 (EPT <= 16).  The one-row kernel is bound by latency,
+// not by memory: every step of its four recurrences waits for the previous one (and for a shared-memory load of
+// the factor).  Here the thread's part of the factor sits in registers for all rows, and the R rows give every
+// step R independent chains; the multipliers of the affine maps, the barriers and the loop overhead are shared by
+// the rows.  Every row sees exactly the operations, in the same order, as in the one-row kernel.
+template <int R>
+struct AffineR {
+  float c[R];
+  float m;
+};
+
+template <int EPT, int R>
+__global__ void __launch_bounds__(SOLVE_THREADS, 3)
+tridiag_solve_rows_kernel(const float* __restrict__ Y, int p, int n, const float* __restrict__ lT,
+                          const float* __restrict__ dT, bf16* __restrict__ Yhi, bf16* __restrict__ Ylo,
+                          float* __restrict__ row_inv) {
+  __shared__ AffineR<R> wtot[SOLVE_THREADS / 32];
+  __shared__ float mscratch[R][32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  float sl[EPT], sd[EPT];
+#pragma unroll
+  for (int t = 0; t < EPT; ++t) {
+    sl[t] = lT[t * SOLVE_THREADS + tid];
+    sd[t] = dT[t * SOLVE_THREADS + tid];
+  }
+  const int a0 = tid * EPT;
+  const int len = a0 >= n ? 0 : (n - a0 < EPT ? n - a0 : EPT);      // a multiple of 8
+  const float l_before = (tid > 0 && len > 0) ? lT[(EPT - 1) * SOLVE_THREADS + tid - 1] : 0.0f;
+  const int groups = (p + R - 1) / R;
+
+  for (int jg = blockIdx.x; jg < groups; jg += gridDim.x) {
+    const int j0 = jg * R;
+    float x[R][EPT];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const int j = j0 + r < p ? j0 + r : p - 1;           // rows past the end repeat the last one, unsaved
+      const float* y = Y + (size_t)j * n + a0;
+#pragma unroll
+      for (int e = 0; e < EPT; e += 4) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e < len) v = *reinterpret_cast<const float4*>(y + e);
+        x[r][e] = v.x; x[r][e + 1] = v.y; x[r][e + 2] = v.z; x[r][e + 3] = v.w;
+      }
+    }
+    // ---- forward substitution x_i = y_i - l_{i-1} x_{i-1}, then the diagonal ----
+    {
+      AffineR<R> f;
+#pragma unroll
+      for (int r = 0; r < R; ++r) f.c[r] = 0.0f;
+      f.m = 1.0f;
+      float lp = l_before;
+#pragma unroll
+      for (int t = 0; t < EPT; ++t)
+        if (t < len) {
+#pragma unroll
+          for (int r = 0; r < R; ++r) f.c[r] = fmaf(-lp, f.c[r], x[r][t]);
+          f.m *= -lp;
+          lp = sl[t];
+        }
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        float oc[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) oc[r] = __shfl_up_sync(0xffffffffu, f.c[r], off);
+        const float om = __shfl_up_sync(0xffffffffu, f.m, off);
+        if (lane >= off) {
+#pragma unroll
+          for (int r = 0; r < R; ++r) f.c[r] = fmaf(f.m, oc[r], f.c[r]);
+          f.m = f.m * om;
+        }
+      }
+      if (lane == 31) wtot[warp] = f;
+      __syncthreads();
+      float prec[R], prem = 1.0f;
+#pragma unroll
+      for (int r = 0; r < R; ++r) prec[r] = 0.0f;
+      for (int w = 0; w < warp; ++w) {
+        const float wm = wtot[w].m;
+#pragma unroll
+        for (int r = 0; r < R; ++r) prec[r] = fmaf(wm, prec[r], wtot[w].c[r]);
+        prem = wm * prem;
+      }
+      float xin[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const float tot = fmaf(f.m, prec[r], f.c[r]);      // map of everything up to this thread
+        xin[r] = __shfl_up_sync(0xffffffffu, tot, 1);
+        if (lane == 0) xin[r] = prec[r];
+      }
+      lp = l_before;
+#pragma unroll
+      for (int t = 0; t < EPT; ++t)
+        if (t < len) {
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            xin[r] = fmaf(-lp, xin[r], x[r][t]);
+            x[r][t] = xin[r] * sd[t];
+          }
+          lp = sl[t];
+        }
+      __syncthreads();
+    }
+    // ---- backward substitution z_i = x_i - l_i z_{i+1} ----
+    float zmax[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) zmax[r] = 0.0f;
+    {
+      AffineR<R> f;
+#pragma unroll
+      for (int r = 0; r < R; ++r) f.c[r] = 0.0f;
+      f.m = 1.0f;
+#pragma unroll
+      for (int t = EPT - 1; t >= 0; --t)
+        if (t < len) {
+#pragma unroll
+          for (int r = 0; r < R; ++r) f.c[r] = fmaf(-sl[t], f.c[r], x[r][t]);
+          f.m *= -sl[t];
+        }
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        float oc[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) oc[r] = __shfl_down_sync(0xffffffffu, f.c[r], off);
+        const float om = __shfl_down_sync(0xffffffffu, f.m, off);
+        if (lane + off < 32) {
+#pragma unroll
+          for (int r = 0; r < R; ++r) f.c[r] = fmaf(f.m, oc[r], f.c[r]);
+          f.m = f.m * om;
+        }
+      }
+      if (lane == 0) wtot[warp] = f;
+      __syncthreads();
+      float postc[R], postm = 1.0f;
+#pragma unroll
+      for (int r = 0; r < R; ++r) postc[r] = 0.0f;
+      for (int w = SOLVE_THREADS / 32 - 1; w > warp; --w) {
+        const float wm = wtot[w].m;
+#pragma unroll
+        for (int r = 0; r < R; ++r) postc[r] = fmaf(wm, postc[r], wtot[w].c[r]);
+        postm = wm * postm;
+      }
+      float z[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const float tot = fmaf(f.m, postc[r], f.c[r]);
+        z[r] = __shfl_down_sync(0xffffffffu, tot, 1);
+        if (lane == 31) z[r] = postc[r];
+      }
+#pragma unroll
+      for (int t = EPT - 1; t >= 0; --t)
+        if (t < len) {
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            z[r] = fmaf(-sl[t], z[r], x[r][t]);
+            x[r][t] = z[r];
+            zmax[r] = fmaxf(zmax[r], fabsf(z[r]));
+          }
+        }
+    }
+    // all row maxima through one pair of barriers (they also separate the row groups' use of wtot)
+#pragma unroll
+    for (int r = 0; r < R; ++r) zmax[r] = warp_max(zmax[r]);
+    __syncthreads();
+    if (lane == 0) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) mscratch[r][warp] = zmax[r];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      if (j0 + r >= p) break;
+      const int j = j0 + r;
+      const float zm = warp_max(lane < SOLVE_THREADS / 32 ? mscratch[r][lane] : 0.0f);
+      float inv;
+      const float sc = pow2_scale_for(zm, &inv);
+      if (tid == 0) row_inv[j] = inv;
+#pragma unroll
+      for (int e = 0; e < EPT; e += 8) {
+        if (e < len) {
+          __align__(16) __half hh[8];
+          __align__(16) __half ll[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) split_f16(x[r][e + k] * sc, hh[k], ll[k]);
+          *reinterpret_cast<uint4*>(Yhi + (size_t)j * n + a0 + e) = *reinterpret_cast<const uint4*>(hh);
+          *reinterpret_cast<uint4*>(Ylo + (size_t)j * n + a0 + e) = *reinterpret_cast<const uint4*>(ll);
+        }
+      }
+    }
+  }
+}
+
+template <int EPT, int R>
+static void launch_solve_rows_t(Ctx* c, int p, int stage, int ctas_per_sm) {
+  const size_t fs = stage_factor_stride(c->n);
+  const int groups = (p + R - 1) / R;
+  int blocks = c->num_sms * ctas_per_sm;
+  if (blocks > groups) blocks = groups;
+  tridiag_solve_rows_kernel<EPT, R><<<blocks, SOLVE_THREADS, 0, c->stream>>>(
+      c->Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi, c->Y_lo,
+      c->rs_Y);
+}
+
 template <int EPT>
 static void launch_solve_t(Ctx* c, int p, int stage, int blocks) {
   const size_t fs = stage_factor_stride(c->n);
@@ -708,8 +911,8 @@ void launch_tridiag_solve(Ctx* c, int p, int stage) {
   int blocks = c->num_sms * 3;                             // resident CTAs; each loads the factor once
   if (blocks > p) blocks = p;
   switch (solve_ept(c->n)) {
-    case 8: launch_solve_t<8>(c, p, stage, blocks); break;
-    case 16: launch_solve_t<16>(c, p, stage, blocks); break;
+    case 8: launch_solve_rows_t<8, SOLVE_ROWS>(c, p, stage, 3); break;
+    case 16: launch_solve_rows_t<16, SOLVE_ROWS>(c, p, stage, 3); break;
     case 24: launch_solve_t<24>(c, p, stage, blocks); break;
     case 32: launch_solve_t<32>(c, p, stage, blocks); break;
     case 40: launch_solve_t<40>(c, p, stage, blocks); break;
