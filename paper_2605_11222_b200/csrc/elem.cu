@@ -654,6 +654,7 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
   __shared__ float scratch[32];
   float r2 = 0.f, s2 = 0.f;
   const int gs = P.group_size;
+  const int gsh = (gs & (gs - 1)) == 0 ? 31 - __clz(gs) : -1;      // group index by shift when the size allows
   for (int j = blockIdx.x; j < p; j += gridDim.x) {
     const size_t base = (size_t)j * n;
     const float* dlt = P.delta + (size_t)j * P.n_groups;
@@ -667,7 +668,8 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
       const float4 si = *reinterpret_cast<const float4*>(P.inv_s + i);
       uchar4 k = make_uchar4(0, 0, 0, 0);
       if (!P.first_iter) k = *reinterpret_cast<const uchar4*>(P.codes + base + i);
-      const int g0 = i / gs, g3 = (i + 3) / gs;
+      const int g0 = gsh >= 0 ? i >> gsh : i / gs;
+      const int g3 = gsh >= 0 ? (i + 3) >> gsh : (i + 3) / gs;
       const float d0 = dlt[g0], z0 = zr[g0], id0 = __frcp_rn(d0);
       AdmmElem e0 = admm_elem(z.x, wh.x, v.x, k.x, sv.x, si.x, d0, id0, z0, P);
       AdmmElem e1, e2, e3;
