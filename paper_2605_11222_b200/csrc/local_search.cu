@@ -45,16 +45,30 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
   long long moves = 0;
   int capped = 0;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  // The gradient update of the move just applied and the scan for the next move share one sweep over the
+  // entries: d_move = 0 on the first sweep (nothing to apply yet).
+  int i_move = -1, k_step = 0;
+  float d_move = 0.0f;
+  const float* hrow = H;
   while (true) {
     Cand best;
     best.cost = INFINITY;
     best.idx = 0x7fffffff;
     // a thread meets its candidates in increasing index order, so a strict "<" keeps the earliest
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      float gi = g[i];
+      int k = kc[i];
+      if (i_move >= 0) {
+        gi = fmaf(d_move, hrow[i], gi);                    // g += d H[:, i_move] (row of the symmetric H)
+        g[i] = gi;
+        if (i == i_move) {
+          k += k_step;
+          kc[i] = (unsigned char)k;
+        }
+      }
       const float d = sdl[shift >= 0 ? (i >> shift) : (i / gs)];
       const float q = quad[i];
-      const float lin = 2.0f * d * g[i];
-      const int k = kc[i];
+      const float lin = 2.0f * d * gi;
       const float cp = lin + q, cm = q - lin;
       if (k < kmax && cp < best.cost) {
         best.cost = cp;
@@ -87,19 +101,16 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
     }
     __syncthreads();
     const Cand c = chosen;
-    if (c.idx < 0) break;
-    const int i = c.idx >> 1;
-    const float sgn = (c.idx & 1) ? -1.0f : 1.0f;
-    const float d = sgn * dl[i / gs];
-    const float* hrow = H + (long long)i * n;
-    for (int t = threadIdx.x; t < n; t += blockDim.x) g[t] = fmaf(d, hrow[t], g[t]);
-    if (threadIdx.x == 0) kc[i] = (unsigned char)((int)kc[i] + ((c.idx & 1) ? -1 : 1));
-    ++moves;
-    __syncthreads();
-    if (moves >= max_moves) {
+    if (moves >= max_moves) {                              // the move that reached the cap has been applied
       capped = 1;
       break;
     }
+    if (c.idx < 0) break;
+    i_move = c.idx >> 1;
+    k_step = (c.idx & 1) ? -1 : 1;
+    d_move = (float)k_step * dl[i_move / gs];
+    hrow = H + (long long)i_move * n;
+    ++moves;
   }
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
     const long long idx = (long long)j * n + i;
