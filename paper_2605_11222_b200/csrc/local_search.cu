@@ -54,29 +54,46 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
     Cand best;
     best.cost = INFINITY;
     best.idx = 0x7fffffff;
-    // a thread meets its candidates in increasing index order, so a strict "<" keeps the earliest
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-      float gi = g[i];
-      int k = kc[i];
+    // a thread meets its candidates in increasing index order, so a strict "<" keeps the earliest;
+    // four consecutive entries per step (n is a multiple of 8)
+    for (int i4 = threadIdx.x * 4; i4 < n; i4 += blockDim.x * 4) {
+      float4 g4 = *reinterpret_cast<const float4*>(g + i4);
+      const float4 q4 = *reinterpret_cast<const float4*>(quad + i4);
+      uchar4 k4 = *reinterpret_cast<const uchar4*>(kc + i4);
       if (i_move >= 0) {
-        gi = fmaf(d_move, hrow[i], gi);                    // g += d H[:, i_move] (row of the symmetric H)
-        g[i] = gi;
-        if (i == i_move) {
-          k += k_step;
-          kc[i] = (unsigned char)k;
+        const float4 h4 = *reinterpret_cast<const float4*>(hrow + i4);   // g += d H[:, i_move] (H symmetric)
+        g4.x = fmaf(d_move, h4.x, g4.x);
+        g4.y = fmaf(d_move, h4.y, g4.y);
+        g4.z = fmaf(d_move, h4.z, g4.z);
+        g4.w = fmaf(d_move, h4.w, g4.w);
+        *reinterpret_cast<float4*>(g + i4) = g4;
+        if ((i_move & ~3) == i4) {
+          const int e = i_move & 3;
+          if (e == 0) k4.x = (unsigned char)((int)k4.x + k_step);
+          if (e == 1) k4.y = (unsigned char)((int)k4.y + k_step);
+          if (e == 2) k4.z = (unsigned char)((int)k4.z + k_step);
+          if (e == 3) k4.w = (unsigned char)((int)k4.w + k_step);
+          *reinterpret_cast<uchar4*>(kc + i4) = k4;
         }
       }
-      const float d = sdl[shift >= 0 ? (i >> shift) : (i / gs)];
-      const float q = quad[i];
-      const float lin = 2.0f * d * gi;
-      const float cp = lin + q, cm = q - lin;
-      if (k < kmax && cp < best.cost) {
-        best.cost = cp;
-        best.idx = 2 * i;
-      }
-      if (k > 0 && cm < best.cost) {
-        best.cost = cm;
-        best.idx = 2 * i + 1;
+      const float gv[4] = {g4.x, g4.y, g4.z, g4.w};
+      const float qv[4] = {q4.x, q4.y, q4.z, q4.w};
+      const int kv[4] = {k4.x, k4.y, k4.z, k4.w};
+      float d = sdl[shift >= 0 ? (i4 >> shift) : (i4 / gs)];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int i = i4 + e;
+        if (e > 0 && (gs & 3) != 0) d = sdl[shift >= 0 ? (i >> shift) : (i / gs)];
+        const float lin = 2.0f * d * gv[e];
+        const float cp = lin + qv[e], cm = qv[e] - lin;
+        if (kv[e] < kmax && cp < best.cost) {
+          best.cost = cp;
+          best.idx = 2 * i;
+        }
+        if (kv[e] > 0 && cm < best.cost) {
+          best.cost = cm;
+          best.idx = 2 * i + 1;
+        }
       }
     }
 #pragma unroll
