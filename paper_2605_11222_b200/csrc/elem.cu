@@ -46,8 +46,43 @@ __global__ void transpose_split_kernel(const TIn* __restrict__ X, long long rows
   }
 }
 
+// The bf16 case on 64 x 64 tiles, two elements per thread: every warp access is 128 contiguous bytes on both
+// sides (the generic kernel moves 64).  Needs even leading dimensions (4-byte accesses).
+__global__ void transpose_bf16_kernel(const bf16* __restrict__ X, long long rows, long long ldx, int n,
+                                      bf16* __restrict__ T, long long ldt) {
+  __shared__ unsigned short tile[64][66];
+  const long long r0 = (long long)blockIdx.x * 64;
+  const int c0 = blockIdx.y * 64;
+  const int tx = threadIdx.x;
+  for (int i = threadIdx.y; i < 64; i += blockDim.y) {
+    const long long r = r0 + i;
+    const int cc = c0 + 2 * tx;
+    unsigned int v = 0u;
+    if (r < rows && cc < n) v = *reinterpret_cast<const unsigned int*>(X + r * ldx + cc);   // n is even
+    tile[i][2 * tx] = (unsigned short)(v & 0xffffu);
+    tile[i][2 * tx + 1] = (unsigned short)(v >> 16);
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 64; i += blockDim.y) {
+    const int cc = c0 + i;
+    const long long r = r0 + 2 * tx;
+    if (cc < n && r < rows) {
+      const unsigned int lo = tile[2 * tx][i], hi = tile[2 * tx + 1][i];
+      bf16* dst = T + (long long)cc * ldt + r;
+      if (r + 1 < rows) *reinterpret_cast<unsigned int*>(dst) = lo | (hi << 16);
+      else *reinterpret_cast<unsigned short*>(dst) = (unsigned short)lo;
+    }
+  }
+}
+
 void launch_transpose_split(Ctx* c, const void* X, int is_bf16, long long rows, long long ldx, int n,
                             bf16* XT_hi, bf16* XT_lo, long long ldt) {
+  if (is_bf16 && (ldx & 1) == 0 && (ldt & 1) == 0 && (reinterpret_cast<uintptr_t>(X) & 3) == 0) {
+    dim3 grid64((unsigned)((rows + 63) / 64), (unsigned)((n + 63) / 64)), block64(32, 8);
+    transpose_bf16_kernel<<<grid64, block64, 0, c->stream>>>((const bf16*)X, rows, ldx, n, XT_hi, ldt);
+    LAUNCH(c);
+    return;
+  }
   dim3 grid((unsigned)((rows + 31) / 32), (unsigned)((n + 31) / 32)), block(32, 8);
   if (is_bf16)
     transpose_split_kernel<bf16><<<grid, block, 0, c->stream>>>((const bf16*)X, rows, ldx, n, XT_hi,
