@@ -450,6 +450,32 @@ def main():
     breakdown = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
                  for k, v in timing.items()}
 
+    # ---- the other timed kernels against their own rooflines (algorithmic bytes or executed flops per launch;
+    #      times are CUDA events around each launch, so short kernels carry a few microseconds of launch gap) ----
+    x_bytes = 2 if spec.x_dtype == "bf16" else 4
+    chunk_rows = spec.n_tokens / max(1, spec.n_chunks)
+
+    def _hbm(kind, bytes_per_launch):
+        ms, cnt = timing[kind]
+        if cnt == 0 or ms <= 0:
+            return None
+        gbs = bytes_per_launch * cnt / (ms * 1e-3) / 1e9
+        return {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / peaks["hbm_gbs"], "launches": cnt, "avg_launch_ms": ms / cnt}
+
+    kernel_rooflines = {
+        "tridiag_solve": _hbm("tridiag_solve", 8.0 * p * n),          # read Y fp32, write two fp16 planes
+        "row_split": _hbm("row_split", 22.0 * p * n),                 # element update + plane split
+        "transpose": _hbm("transpose", 2.0 * x_bytes * chunk_rows * n),
+    }
+    ms_h, n_h = timing["hessian_product"]
+    if n_h:
+        planes = 1 if spec.x_dtype == "bf16" else 3
+        tf = planes * 1.0 * chunk_rows * n * n * n_h / (ms_h * 1e-3) / 1e12   # lower-triangle tiles only
+        kernel_rooflines["hessian_product"] = {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_sustained"],
+                                               "unit": "TFLOP/s", "frac": tf / peaks["bf16_sustained"],
+                                               "launches": n_h, "avg_launch_ms": ms_h / n_h}
+
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:            # the oracle is timed at N = 1 only
         est, desc, threads = oracle_sample_seconds(spec, wl)
@@ -469,7 +495,8 @@ def main():
         "local_search_moves": rep.moves, "pair_swap_after_local_search": pair_swap, "admm_with_grid_refresh": grid_refresh,
         "admm_with_mse_clip_search": mse_clip, "admm_with_fused_epilogue": fused_variant,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-        "roofline": roofline, "cpu_baseline": cpu_baseline, "breakdown": breakdown,
+        "roofline": roofline, "kernel_rooflines": kernel_rooflines, "cpu_baseline": cpu_baseline,
+        "breakdown": breakdown,
     }
     print(json.dumps(line))
     if world > 1:
