@@ -702,7 +702,7 @@ struct AffineR {
   float m;
 };
 
-template <int EPT, int R>
+template <int EPT, int R, bool FULL>
 __global__ void __launch_bounds__(SOLVE_THREADS, 3)
 tridiag_solve_rows_kernel(const float* __restrict__ Y, int p, int n, const float* __restrict__ lT,
                           const float* __restrict__ dT, bf16* __restrict__ Yhi, bf16* __restrict__ Ylo,
@@ -717,7 +717,8 @@ tridiag_solve_rows_kernel(const float* __restrict__ Y, int p, int n, const float
     sd[t] = dT[t * SOLVE_THREADS + tid];
   }
   const int a0 = tid * EPT;
-  const int len = a0 >= n ? 0 : (n - a0 < EPT ? n - a0 : EPT);      // a multiple of 8
+  // FULL: d_in = EPT * SOLVE_THREADS, every thread has a whole segment and the guards below fold away
+  const int len = FULL ? EPT : (a0 >= n ? 0 : (n - a0 < EPT ? n - a0 : EPT));      // a multiple of 8
   const float l_before = (tid > 0 && len > 0) ? lT[(EPT - 1) * SOLVE_THREADS + tid - 1] : 0.0f;
   const int groups = (p + R - 1) / R;
 
@@ -888,9 +889,14 @@ static void launch_solve_rows_t(Ctx* c, int p, int stage, int ctas_per_sm) {
   const int groups = (p + R - 1) / R;
   int blocks = c->num_sms * ctas_per_sm;
   if (blocks > groups) blocks = groups;
-  tridiag_solve_rows_kernel<EPT, R><<<blocks, SOLVE_THREADS, 0, c->stream>>>(
-      c->Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi, c->Y_lo,
-      c->rs_Y);
+  if (c->n == EPT * SOLVE_THREADS)
+    tridiag_solve_rows_kernel<EPT, R, true><<<blocks, SOLVE_THREADS, 0, c->stream>>>(
+        c->Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi, c->Y_lo,
+        c->rs_Y);
+  else
+    tridiag_solve_rows_kernel<EPT, R, false><<<blocks, SOLVE_THREADS, 0, c->stream>>>(
+        c->Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi, c->Y_lo,
+        c->rs_Y);
 }
 
 template <int EPT>
