@@ -475,6 +475,178 @@ form_qt_kernel(const double* __restrict__ A, const double* __restrict__ Sall, in
   }
 }
 
+// ---- the same accumulation for CTAs with at most QT_PIPE_ROWS own rows (d_in <= QT_PIPE_ROWS x CTAs): the
+// chunks of Y and X are staged by asynchronous copies several chunks ahead, so that the sweep over the columns
+// no longer waits for a round trip to L2 at every chunk.
+constexpr int QT_PIPE_ROWS = 32;
+constexpr int QT_PIPE_DEPTH = 3;
+__device__ __forceinline__ void cp_async8(double* dst_smem, const double* src, bool valid) {
+  const unsigned int d = (unsigned int)__cvta_generic_to_shared(dst_smem);
+  const int bytes = valid ? 8 : 0;                         // 0: the destination is filled with zeros
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+__global__ void __launch_bounds__(QT_THREADS, 1)
+form_qt_pipe_kernel(const double* __restrict__ A, const double* __restrict__ Sall, int n, int nblk,
+               double* __restrict__ P) {
+  extern __shared__ double smq[];
+  constexpr int BUF = (WY_NB + QT_PIPE_ROWS) * QT_LD;      // one staged chunk: Y block, then the own rows of X
+  double* Zp = smq + QT_PIPE_DEPTH * BUF;                  // [ks][RS][QT_LDZ], ks * RS <= 128
+  double* Z1 = Zp + QT_RS_MAX * QT_LDZ;                    // [RS][QT_LDZ]  (X Y), then -(X Y) S^T
+  double* Ss = Z1 + QT_PIPE_ROWS * QT_LDZ;                 // [WY_NB][WY_NB + 1]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gid = lane >> 2, tig = lane & 3;
+  const int G = gridDim.x, c = blockIdx.x;
+  if (c >= n) return;
+  const int Rtot = (n - c + G - 1) / G;                    // rows c, c + G, c + 2G, ...
+  const int nrefl = n - 2;
+
+  for (int b = nblk - 1; b >= 0; --b) {
+    const int kb = b * WY_NB;
+    const int nbk = nrefl - kb < WY_NB ? nrefl - kb : WY_NB;
+    int t0 = (kb + 1 - c + G - 1) / G;                     // first own row with r >= kb + 1
+    if (kb + 1 - c <= 0) t0 = 0;
+    const int Ract = Rtot - t0;
+    if (Ract <= 0) continue;                               // uniform in the CTA
+    const int RS = (Ract + 7) & ~7;
+    const int nrt = RS >> 3;
+    int KS = 1;
+    while (KS < 4 && 2 * KS * RS <= QT_RS_MAX) KS <<= 1;
+    const int kspan = QT_KC / KS;
+    const int cbeg = ((kb + 1) / QT_KC) * QT_KC;
+
+    for (int idx = tid; idx < WY_NB * WY_NB; idx += QT_THREADS)
+      Ss[(idx >> 5) * (WY_NB + 1) + (idx & 31)] = Sall[(size_t)b * WY_NB * WY_NB + idx];
+
+    // ---------------- Z = X Y ----------------
+    const int units_z = nrt * 4 * KS;                      // (k split, row tile, column tile of 8)
+    double z00 = 0.0, z01 = 0.0, z10 = 0.0, z11 = 0.0;     // accumulators of units warp and warp + 32
+    const int nch = (n - cbeg + QT_KC - 1) / QT_KC;
+    // chunk ci of the columns, staged by asynchronous copies QT_PIPE_DEPTH - 1 chunks ahead of its use
+    auto issue = [&](int ci, bool with_x) {
+      if (ci < nch) {
+        const int cs = cbeg + ci * QT_KC;
+        double* Yb = smq + (ci % QT_PIPE_DEPTH) * BUF;
+        double* Xb = Yb + WY_NB * QT_LD;
+        for (int idx = tid; idx < WY_NB * QT_KC; idx += QT_THREADS) {
+          const int j = idx >> 6, cl = idx & 63, cc = cs + cl;
+          const bool ok = j < nbk && cc < n && cc >= kb + j + 1;
+          cp_async8(Yb + j * QT_LD + cl, ok ? A + (size_t)(kb + j) * n + cc : A, ok);
+        }
+        if (with_x)
+          for (int idx = tid; idx < RS * QT_KC; idx += QT_THREADS) {
+            const int rl = idx >> 6, cl = idx & 63, cc = cs + cl;
+            const bool ok = rl < Ract && cc < n;
+            cp_async8(Xb + rl * QT_LD + cl, ok ? P + (size_t)(c + (size_t)(t0 + rl) * G) * n + cc : P, ok);
+          }
+      }
+      cp_async_commit();                                   // an empty group keeps the count uniform
+    };
+    for (int d = 0; d < QT_PIPE_DEPTH - 1; ++d) issue(d, true);
+    for (int ci = 0; ci < nch; ++ci) {
+      issue(ci + QT_PIPE_DEPTH - 1, true);                 // its buffer was released by the barrier below
+      cp_async_wait<QT_PIPE_DEPTH - 1>();
+      __syncthreads();
+      const double* Ys = smq + (ci % QT_PIPE_DEPTH) * BUF;
+      const double* Xs = Ys + WY_NB * QT_LD;
+#pragma unroll
+      for (int s = 0; s < 2; ++s) {
+        const int u = warp + 32 * s;
+        if (u < units_z) {
+          const int ks = u / (nrt * 4), rem = u - ks * nrt * 4;
+          const int rt = rem >> 2, jt = rem & 3;
+          const double* xa = Xs + (rt * 8 + gid) * QT_LD + ks * kspan + tig;
+          const double* yb = Ys + (jt * 8 + gid) * QT_LD + ks * kspan + tig;
+          double d0 = s ? z10 : z00, d1 = s ? z11 : z01;
+          for (int kk = 0; kk < kspan; kk += 4) dmma_8x8x4(d0, d1, xa[kk], yb[kk]);
+          if (s) {
+            z10 = d0;
+            z11 = d1;
+          } else {
+            z00 = d0;
+            z01 = d1;
+          }
+        }
+      }
+      __syncthreads();
+    }
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      const int u = warp + 32 * s;
+      if (u < units_z) {
+        const int ks = u / (nrt * 4), rem = u - ks * nrt * 4;
+        const int rt = rem >> 2, jt = rem & 3;
+        double* zp = Zp + (ks * RS + rt * 8 + gid) * QT_LDZ + jt * 8 + 2 * tig;
+        zp[0] = s ? z10 : z00;
+        zp[1] = s ? z11 : z01;
+      }
+    }
+    __syncthreads();
+    for (int idx = tid; idx < RS * WY_NB; idx += QT_THREADS) {
+      const int rl = idx >> 5, j = idx & 31;
+      double z = 0.0;
+      for (int ks = 0; ks < KS; ++ks) z += Zp[(ks * RS + rl) * QT_LDZ + j];
+      Z1[rl * QT_LDZ + j] = z;
+    }
+    __syncthreads();
+    // ---------------- Z2 = -(Z S^T):  Z2[rl][j] = -sum_{j' >= j} Z[rl][j'] S[j][j'] ----------------
+    double z2v[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int idx = tid + q * QT_THREADS;
+      z2v[q] = 0.0;
+      if (idx < RS * WY_NB) {
+        const int rl = idx >> 5, j = idx & 31;
+        double z = 0.0;
+        for (int jp = j; jp < WY_NB; ++jp) z += Z1[rl * QT_LDZ + jp] * Ss[j * (WY_NB + 1) + jp];
+        z2v[q] = -z;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int idx = tid + q * QT_THREADS;
+      if (idx < RS * WY_NB) Z1[(idx >> 5) * QT_LDZ + (idx & 31)] = z2v[q];
+    }
+    __syncthreads();
+    // ---------------- X += Z2 Y^T ----------------
+    const int units_u = nrt * 8;                           // (row tile, column tile of 8 inside the chunk)
+    __syncthreads();                                       // every warp is done with the buffers of the first sweep
+    // one unit per warp at most (QT_PIPE_ROWS = 32 rows): its tile of X for the next chunk is loaded a chunk ahead
+    const int rt_u = warp >> 3, nt_u = warp & 7;
+    const int rl_u = rt_u * 8 + gid;
+    const bool has_u = warp < units_u;
+    auto xptr = [&](int ci) {
+      return P + (size_t)(c + (size_t)(t0 + (rl_u < Ract ? rl_u : 0)) * G) * n + cbeg + ci * QT_KC + nt_u * 8 + 2 * tig;
+    };
+    auto xlive = [&](int ci) { return has_u && rl_u < Ract && cbeg + ci * QT_KC + nt_u * 8 + 2 * tig < n; };
+    double2 cvn = make_double2(0.0, 0.0);
+    if (xlive(0)) cvn = *reinterpret_cast<const double2*>(xptr(0));
+    for (int d = 0; d < QT_PIPE_DEPTH - 1; ++d) issue(d, false);
+    for (int ci = 0; ci < nch; ++ci) {
+      issue(ci + QT_PIPE_DEPTH - 1, false);
+      cp_async_wait<QT_PIPE_DEPTH - 1>();
+      __syncthreads();
+      const double* Ys = smq + (ci % QT_PIPE_DEPTH) * BUF;
+      double2 cv = cvn;
+      if (ci + 1 < nch && xlive(ci + 1)) cvn = *reinterpret_cast<const double2*>(xptr(ci + 1));
+      if (has_u) {
+        const double* za = Z1 + rl_u * QT_LDZ + tig;
+        const double* yb = Ys + tig * QT_LD + nt_u * 8 + gid;
+#pragma unroll
+        for (int kk = 0; kk < WY_NB; kk += 4) dmma_8x8x4(cv.x, cv.y, za[kk], yb[kk * QT_LD]);
+        if (xlive(ci)) *reinterpret_cast<double2*>(xptr(ci)) = cv;
+      }
+      __syncthreads();
+    }
+  }
+}
+
 cudaError_t tridiag_form_qt(Ctx* c) {
   const int n = c->n;
   const int nrefl = n - 2;
@@ -491,6 +663,15 @@ cudaError_t tridiag_form_qt(Ctx* c) {
   e = cudaFuncSetAttribute(form_qt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   int grid = c->num_sms;
+  if ((n + grid - 1) / grid <= QT_PIPE_ROWS) {
+    const size_t smem_p = (size_t)(QT_PIPE_DEPTH * (WY_NB + QT_PIPE_ROWS) * QT_LD + QT_RS_MAX * QT_LDZ +
+                                   QT_PIPE_ROWS * QT_LDZ + WY_NB * (WY_NB + 1)) * sizeof(double);
+    e = cudaFuncSetAttribute(form_qt_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_p);
+    if (e != cudaSuccess) return e;
+    form_qt_pipe_kernel<<<grid, QT_THREADS, smem_p, c->stream>>>(c->A64, Sall, n, nblk, c->P64);
+    c->launches++;
+    return cudaGetLastError();
+  }
   while ((n + grid - 1) / grid > QT_RS_MAX) grid += c->num_sms;   // at most 128 rows per CTA
   form_qt_kernel<<<grid, QT_THREADS, smem, c->stream>>>(c->A64, Sall, n, nblk, c->P64);
   c->launches++;
