@@ -203,7 +203,14 @@ __global__ void __launch_bounds__(TB_THREADS, 1) tridiag_blocked_kernel(TrbArgs 
       }
       grid.sync();
       // ================= D: w, own rows and the panel's broadcast rows =================
-      for (int o = warp; o <= 2 * TB_NB; o += 32) {
+      // sums o < i (W^T v), TB_NB + o < TB_NB + i (V^T v) and 2 TB_NB (v^T A22 v): warp w takes w and TB_NB + w; the
+      // last warp, whose two are never needed (i < TB_NB), takes the third kind, so that no warp runs three rounds
+      for (int q = 0; q < 2; ++q) {
+        int o = warp + TB_NB * q;
+        if (warp == 31) {
+          if (q == 1) break;
+          o = 2 * TB_NB;
+        }
         const bool need = (o < TB_NB) ? (o < i) : (o < 2 * TB_NB ? (o - TB_NB < i) : true);
         if (!need) continue;
         double s = 0.0;
