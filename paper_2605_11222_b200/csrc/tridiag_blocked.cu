@@ -203,20 +203,21 @@ __global__ void __launch_bounds__(TB_THREADS, 1) tridiag_blocked_kernel(TrbArgs 
       }
       grid.sync();
       // ================= D: w, own rows and the panel's broadcast rows =================
-      // sums o < i (W^T v), TB_NB + o < TB_NB + i (V^T v) and 2 TB_NB (v^T A22 v): warp w takes w and TB_NB + w; the
-      // last warp, whose two are never needed (i < TB_NB), takes the third kind, so that no warp runs three rounds
-      for (int q = 0; q < 2; ++q) {
-        int o = warp + TB_NB * q;
-        if (warp == 31) {
-          if (q == 1) break;
-          o = 2 * TB_NB;
-        }
+      // sums o < i (W^T v), TB_NB + o < TB_NB + i (V^T v) and 2 TB_NB (v^T A22 v) in one round: the two halves of
+      // warp w take w and TB_NB + w; the last warp, whose two are never needed (i < TB_NB), takes the third kind
+      {
+        const int half = lane >> 4, sub = lane & 15;
+        int o = warp + TB_NB * half;
+        if (warp == 31) o = 2 * TB_NB;                   // both halves: the same sum, written once
         const bool need = (o < TB_NB) ? (o < i) : (o < 2 * TB_NB ? (o - TB_NB < i) : true);
-        if (!need) continue;
         double s = 0.0;
-        for (int b = lane; b < G; b += 32) s += __ldcg(a.part + (size_t)o * G + b);
-        s = warp_sum(s);
-        if (lane == 0) red[o] = s;
+        if (need)
+          for (int b = sub; b < G; b += 16) s += __ldcg(a.part + (size_t)o * G + b);
+        s += __shfl_xor_sync(0xffffffffu, s, 8);
+        s += __shfl_xor_sync(0xffffffffu, s, 4);
+        s += __shfl_xor_sync(0xffffffffu, s, 2);
+        s += __shfl_xor_sync(0xffffffffu, s, 1);
+        if (need && sub == 0 && (warp != 31 || half == 0)) red[o] = s;
       }
       __syncthreads();
       const double* Wv = red;                            // W^T v
