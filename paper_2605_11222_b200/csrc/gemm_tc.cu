@@ -17,7 +17,9 @@
 //
 // One persistent CTA per SM, 576 threads:
 //   warp 0       TMA producer: cp.async.bulk.tensor loads of 128B-swizzled K-major tiles into a ring
-//                of shared-memory stages, completion counted by mbarriers;
+//                of shared-memory stages, completion counted by mbarriers; with two planes the lo planes of
+//                a stage are refilled as soon as the cross products of its K block are done, the hi planes
+//                after the hi x hi products (only two stages fit, so every cycle of head start counts);
 //   warp 1       MMA issuer: one elected thread issues tcgen05.mma (M = 128, N = 256 or 128, K = 16 per
 //                instruction) and tcgen05.commit, which releases stages and publishes partials;
 //   warps 2-17   workers: warp w owns tensor-memory lanes 32 (w mod 4) .. +31 (output rows) and 64 of
@@ -341,7 +343,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
   constexpr int STAGES = (NP == 1) ? 4 : 2;
   constexpr int KB_PER_FLUSH = (NP == 1) ? 3 : 1;        // 12 accumulating MMA steps per flush either way
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * STAGES + 2 * NPART];
+  __shared__ __align__(8) uint64_t bars[3 * STAGES + 2 * NPART];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ float red[WORKER_WARPS * 2];
@@ -355,12 +357,14 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
   const uint32_t empty0 = smem_u32(&bars[STAGES]);
   const uint32_t pfull0 = smem_u32(&bars[2 * STAGES]);
   const uint32_t pempty0 = smem_u32(&bars[2 * STAGES + NPART]);
+  const uint32_t elo0 = smem_u32(&bars[2 * STAGES + 2 * NPART]);   // two planes: the lo planes of a stage are free
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(full0 + 8 * s, 1);
+      mbar_init(full0 + 8 * s, NP == 2 ? 2 : 1);           // two planes: the lo and the hi half arrive separately
       mbar_init(empty0 + 8 * s, 1);
+      mbar_init(elo0 + 8 * s, 1);
     }
     for (int a = 0; a < NPART; ++a) {
       mbar_init(pfull0 + 8 * a, 1);
@@ -395,18 +399,25 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
         if (lower && un.col0 > un.tm * BM + BM - 1) continue;
         const int boxes = un.ncols / BN_BOX;
         for (int kb = 0; kb < num_kb; ++kb) {
-          ok = mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag, status);
-          if (!ok) break;
           const uint32_t sbase = tiles_base + stage * STAGE_BYTES;
           const uint32_t fb = full0 + 8 * stage;
-          mbar_expect_tx(fb, NP * (A_BYTES + boxes * BOX_BYTES));
-#pragma unroll
-          for (int pl = 0; pl < NP; ++pl) tma_load_2d(sbase + pl * A_BYTES, &maps.a[pl], fb, kb * BK, un.tm * BM);
-#pragma unroll
-          for (int pl = 0; pl < NP; ++pl)
+          if (NP == 2) {
+            // the lo planes of a stage are released after the two cross products of its K block, a third of the
+            // block's MMA time before the hi planes: their refill starts that much earlier
+            ok = mbar_wait(elo0 + 8 * stage, phase ^ 1u, abort_flag, status);
+            if (!ok) break;
+            mbar_expect_tx(fb, A_BYTES + boxes * BOX_BYTES);
+            tma_load_2d(sbase + A_BYTES, &maps.a[1], fb, kb * BK, un.tm * BM);
             for (int bx = 0; bx < boxes; ++bx)
-              tma_load_2d(sbase + NP * A_BYTES + pl * B_BYTES + bx * BOX_BYTES, &maps.b[pl], fb, kb * BK,
+              tma_load_2d(sbase + NP * A_BYTES + B_BYTES + bx * BOX_BYTES, &maps.b[1], fb, kb * BK,
                           un.col0 + bx * BN_BOX);
+          }
+          ok = mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag, status);
+          if (!ok) break;
+          mbar_expect_tx(fb, A_BYTES + boxes * BOX_BYTES);
+          tma_load_2d(sbase, &maps.a[0], fb, kb * BK, un.tm * BM);
+          for (int bx = 0; bx < boxes; ++bx)
+            tma_load_2d(sbase + NP * A_BYTES + bx * BOX_BYTES, &maps.b[0], fb, kb * BK, un.col0 + bx * BN_BOX);
           if (++stage == STAGES) {
             stage = 0;
             phase ^= 1u;
@@ -444,15 +455,21 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
           const uint64_t a_lo = make_kmajor_sw128_desc(sbase + A_BYTES);
           const uint64_t b_hi = make_kmajor_sw128_desc(sbase + NP * A_BYTES);
           const uint64_t b_lo = make_kmajor_sw128_desc(sbase + NP * A_BYTES + B_BYTES);
+          // the small cross terms of the whole K block first (they meet a small accumulator, and the lo planes
+          // become free for the next load), then the hi x hi terms
+          if (NP == 2) {
 #pragma unroll
-          for (int k16 = 0; k16 < BK / 16; ++k16) {
-            const uint64_t koff = (uint64_t)((k16 * 32) >> 4);   // 16 elements = 32 bytes along K
-            // small terms first, so that they meet a small accumulator
-            if (NP == 2) {
+            for (int k16 = 0; k16 < BK / 16; ++k16) {
+              const uint64_t koff = (uint64_t)((k16 * 32) >> 4);   // 16 elements = 32 bytes along K
               tc_mma_f16(d_tmem, a_hi + koff, b_lo + koff, idesc, accumulate);
               tc_mma_f16(d_tmem, a_lo + koff, b_hi + koff, idesc, 1);
               accumulate = 1;
             }
+            tc_commit(elo0 + 8 * stage);
+          }
+#pragma unroll
+          for (int k16 = 0; k16 < BK / 16; ++k16) {
+            const uint64_t koff = (uint64_t)((k16 * 32) >> 4);
             tc_mma_f16(d_tmem, a_hi + koff, b_hi + koff, idesc, accumulate);
             accumulate = 1;
           }
