@@ -21,8 +21,12 @@
  *    enqueued.  Numerical failures found on the device (non-finite input, a
  *    non-positive Hessian diagonal or pivot, a wait that ran out) are recorded in a
  *    device status word: admmq_last_device_status synchronises and returns it, and a
- *    call given a non-NULL host report returns it too.  Outputs are unspecified
- *    after an error.
+ *    call given a non-NULL host report returns it too.  The word keeps the first error
+ *    raised since it was last read, and reading it clears it: the error is returned
+ *    once, and the next call on the context (for example quantize_layer with a valid
+ *    weight matrix after one that held a NaN, on the same factorisation) starts from
+ *    ADMMQ_OK.  admmq_hessian_reset and admmq_hessian_set clear it as well.  Outputs
+ *    are unspecified after an error.
  *  - Device pointers must be 16-byte aligned; d_in must be a multiple of 8 and at
  *    most ADMMQ_MAX_D_IN; d_in must be a multiple of the group size.
  *  - Call order: create -> hessian_reset -> hessian_accumulate* -> factor ->
@@ -62,8 +66,9 @@ typedef enum { ADMMQ_F32 = 0, ADMMQ_BF16 = 1 } admmq_dtype;
 /* How the product (H~ + rho I)^{-1} of the W-update (Eq. 7) is applied.
  * TRIDIAG: one orthogonal reduction H~ = Q T Q^T (T tridiagonal), reused for every rho, with an O(n)
  *          LDL^T of T + rho I per penalty value -- the role the single eigendecomposition plays in
- *          Algorithm 1 line 3.  The only kind implemented. */
-typedef enum { ADMMQ_FACTOR_TRIDIAG = 0, ADMMQ_FACTOR_CHOLESKY = 1, ADMMQ_FACTOR_EIG = 2 } admmq_factor_kind;
+ *          Algorithm 1 line 3.  It is the only kind; the field exists so that the struct need not
+ *          change if another is added. */
+typedef enum { ADMMQ_FACTOR_TRIDIAG = 0 } admmq_factor_kind;
 
 /* Which matrix-product kernels run.  TENSOR: tcgen05 tensor-core kernels on two-plane 16-bit operands
  * (power-of-two scaled fp16 hi + lo for the W-update and gradient products, bf16 for the calibration
@@ -85,7 +90,7 @@ admmq_status admmq_create(admmq_ctx** ctx, int d_in, int d_out_max, int T_max, v
 admmq_status admmq_destroy(admmq_ctx* ctx); /* frees the host struct only */
 admmq_status admmq_set_gemm_kind(admmq_ctx* ctx, admmq_gemm_kind kind);
 
-/* Synchronises the stream and returns the device status word (ADMMQ_OK if none was raised). */
+/* Synchronises the stream, returns the device status word (ADMMQ_OK if none was raised) and clears it. */
 admmq_status admmq_last_device_status(admmq_ctx* ctx);
 
 /* ---- Step 1: Hessian accumulation, H_raw += X^T X, N += n_tokens  (Sec. 3.1: H = X^T X). ----------
@@ -108,7 +113,7 @@ typedef struct {
   size_t struct_size;     /* sizeof(admmq_factor_cfg) */
   double damp_frac;       /* 0.01 in the paper */
   int precondition;       /* 1: diagonal scaling on (paper default); 0: s_i = 1 */
-  int kind;               /* admmq_factor_kind */
+  int kind;               /* admmq_factor_kind; any other value: ADMMQ_ERR_INVALID_ARG */
   int T;                  /* number of ADMM iterations, 1..T_max */
   const double* h_rho;    /* host array [T] or NULL */
   double rho0, gamma;     /* used when h_rho == NULL */
@@ -272,7 +277,10 @@ admmq_status admmq_get_timing(admmq_ctx* ctx, int kind, double* h_total_ms, long
  * entries it later reads, so nothing needs clearing): calls that overlap on the GPU -- different
  * streams or threads without an ordering between them -- race; serialise them.  The first call on a
  * device also looks up the scratch address and raises the kernel's shared-memory limit; make that first
- * call outside any stream capture. */
+ * call outside any stream capture.  The device that owns the pointers and the stream must be the
+ * current device of the calling thread: the scratch address is looked up for the current device.  With
+ * lazy module loading the array and the kernels are placed in device memory at that first call, so a
+ * caller that expects a co-tenant to claim the remaining HBM should make it before that happens. */
 #define ADMMQ_STATIC_MAX_D_OUT 16384
 admmq_status admmq_objective_static(const float* d_H, int d_in, const float* d_W0, int d_out,
                                     int group_size, const unsigned char* d_codes, const float* d_scale,

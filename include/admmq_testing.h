@@ -1,0 +1,29 @@
+/*
+ * admmq_testing.h -- hooks for tests of the library's failure handling.  Not part of the solver's
+ * contract: nothing here is needed to quantize a layer, and the paper has no counterpart.
+ */
+#ifndef ADMMQ_TESTING_H_
+#define ADMMQ_TESTING_H_
+
+#include "admmq.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Every device-side wait of the tensor-core product kernel (on a shared-memory barrier that a copy or a
+ * tensor-core operation completes) is bounded: when the bound runs out the kernel records
+ * ADMMQ_ERR_TIMEOUT in the device status word, stops issuing work, waits for what it has in flight,
+ * frees its tensor memory and returns, and the context stays usable.
+ * This call sets that bound for the context, in SM clock cycles (wait_limit_cycles >= 1000; the default is
+ * 2e9, about a second), and, with hold_loads != 0, makes the kernel's producer warp issue no loads at
+ * all, so that the first wait of every CTA runs out with nothing in flight: the safe way to see the
+ * time-out path execute.  hold_loads = 0 and the default bound restore normal operation.  Host-side
+ * only; takes effect from the next launch.  Returns ADMMQ_ERR_INVALID_ARG for a NULL context or a bound
+ * below 1000 cycles. */
+admmq_status admmq_test_set_wait(admmq_ctx* ctx, long long wait_limit_cycles, int hold_loads);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADMMQ_TESTING_H_ */

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libadmmq.so")
 OK, ERR_INVALID_ARG, ERR_SHAPE, ERR_STATE, ERR_WORKSPACE, ERR_NOT_SPD, ERR_NONFINITE, ERR_TIMEOUT, \
     ERR_CUDA, ERR_UNSUPPORTED, WARN_MOVE_CAP = range(11)
 F32, BF16 = 0, 1
-FACTOR_TRIDIAG, FACTOR_CHOLESKY, FACTOR_EIG = 0, 1, 2
+FACTOR_TRIDIAG = 0
 GEMM_TENSOR, GEMM_SIMT = 0, 1
 
 EXPORTS = [
@@ -27,7 +27,7 @@ EXPORTS = [
     "admmq_hessian_accumulate", "admmq_hessian_set", "admmq_factor", "admmq_quantize_layer",
     "admmq_w_update", "admmq_local_search", "admmq_objective", "admmq_get_hessian",
     "admmq_launch_count", "admmq_set_timing", "admmq_reset_timing", "admmq_get_timing",
-    "admmq_objective_static", "admmq_get_factor", "admmq_pair_swap",
+    "admmq_objective_static", "admmq_get_factor", "admmq_pair_swap", "admmq_test_set_wait",
 ]
 T_HESSIAN_PRODUCT, T_TRANSPOSE, T_FACTOR, T_WUPDATE_PRODUCT1, T_TRIDIAG_SOLVE, T_WUPDATE_PRODUCT2, \
     T_GRADIENT_PRODUCT, T_LOCAL_SEARCH, T_ROW_SPLIT = range(9)
@@ -109,6 +109,7 @@ def load_library(path: Optional[str] = None):
     lib.admmq_reset_timing.argtypes = [vp]
     lib.admmq_get_timing.argtypes = [vp, ci, C.POINTER(cd), C.POINTER(cll)]
     lib.admmq_objective_static.argtypes = [vp, ci, vp, ci, ci, vp, vp, vp, vp, vp]
+    lib.admmq_test_set_wait.argtypes = [vp, cll, ci]
     lib.admmq_launch_count.restype = cll
     lib.admmq_launch_count.argtypes = [vp]
     for name in EXPORTS:
@@ -296,16 +297,24 @@ class Solver:
     def launch_count(self) -> int:
         return int(self.lib.admmq_launch_count(self.h))
 
+    def test_set_wait(self, wait_limit_cycles: int = 2_000_000_000, hold_loads: bool = False):
+        """Failure-handling tests only: bound of the product kernel's device-side waits, and whether its
+        producer withholds every load (admmq_testing.h)."""
+        _check(self.lib.admmq_test_set_wait(self.h, int(wait_limit_cycles), int(hold_loads)),
+               "admmq_test_set_wait")
+
 
 def objective_static(H: torch.Tensor, W0: torch.Tensor, group_size: int, codes: torch.Tensor,
                      scale: torch.Tensor, zero: torch.Tensor, out: torch.Tensor,
                      stream: Optional[torch.cuda.Stream] = None) -> int:
     """admmq_objective_static: the layer error into `out` (one device double) without any context,
     workspace or allocation inside the library -- for callers whose device memory is all spoken for.
-    Returns the status; asynchronous on `stream` (default: the current stream)."""
+    Returns the status; asynchronous on `stream` (default: the current stream).  The call is made with the
+    tensors' device current, as the entry point requires."""
     lib = load_library()
     assert out.dtype == torch.float64 and out.is_cuda and out.numel() == 1
-    sp = C.c_void_p(stream.cuda_stream if stream is not None else
-                    torch.cuda.current_stream(W0.device).cuda_stream)
-    return lib.admmq_objective_static(_ptr(H), H.shape[0], _ptr(W0), W0.shape[0], group_size, _ptr(codes),
-                                      _ptr(scale), _ptr(zero), _ptr(out), sp)
+    with torch.cuda.device(W0.device):
+        sp = C.c_void_p(stream.cuda_stream if stream is not None else
+                        torch.cuda.current_stream(W0.device).cuda_stream)
+        return lib.admmq_objective_static(_ptr(H), H.shape[0], _ptr(W0), W0.shape[0], group_size, _ptr(codes),
+                                          _ptr(scale), _ptr(zero), _ptr(out), sp)

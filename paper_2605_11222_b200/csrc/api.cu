@@ -1,14 +1,34 @@
 // extern "C" entry points of libadmmq: argument checks, workspace carve-up and the host-side
 // sequencing of the kernels.  All numerical work runs in the CUDA kernels of this library.
 #include <math.h>
+#include <map>
+#include <mutex>
 #include <new>
 #include <string.h>
+#include <utility>
 #include <vector>
 
 #include "../../include/admmq.h"
+#include "../../include/admmq_testing.h"
 #include "internal.h"
 
 using namespace admmq;
+
+namespace admmq {
+cudaError_t ensure_dynamic_smem(const void* kernel, int bytes) {
+  static std::mutex mu;
+  static std::map<std::pair<const void*, int>, int> done;   // (kernel, device) -> limit already set
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> lock(mu);
+  int& have = done[std::make_pair(kernel, dev)];
+  if (have >= bytes) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) have = bytes;
+  return e;
+}
+}  // namespace admmq
 
 struct admmq_ctx {
   Ctx c;
@@ -115,10 +135,13 @@ cudaError_t product(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiPa
   return c->gemm_kind == ADMMQ_GEMM_SIMT ? gemm_simt(c, A, B, M, N, K, e) : gemm_tc(c, A, B, M, N, K, e);
 }
 
+// Reads the device status word and clears it: an error is reported once, by the first call that reads
+// it, and later calls on the context start from ADMMQ_OK again.
 admmq_status read_status(admmq_ctx* a) {
   int st = 0;
   if (cudaStreamSynchronize(a->c.stream) != cudaSuccess) return ADMMQ_ERR_CUDA;
   if (cudaMemcpy(&st, a->c.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  if (st != 0 && cudaMemsetAsync(a->c.status, 0, sizeof(int), a->c.stream) != cudaSuccess) return ADMMQ_ERR_CUDA;
   if (cudaGetLastError() != cudaSuccess) return ADMMQ_ERR_CUDA;
   return (admmq_status)st;
 }
@@ -251,6 +274,13 @@ admmq_status admmq_last_device_status(admmq_ctx* ctx) {
 
 long long admmq_launch_count(const admmq_ctx* ctx) { return ctx ? ctx->c.launches : 0; }
 
+admmq_status admmq_test_set_wait(admmq_ctx* ctx, long long wait_limit_cycles, int hold_loads) {
+  if (!ctx || wait_limit_cycles < 1000) return ADMMQ_ERR_INVALID_ARG;
+  ctx->c.wait_limit_cycles = wait_limit_cycles;
+  ctx->c.hold_loads = hold_loads ? 1 : 0;
+  return ADMMQ_OK;
+}
+
 admmq_status admmq_hessian_reset(admmq_ctx* ctx) {
   if (!ctx) return ADMMQ_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
@@ -309,7 +339,6 @@ admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg) {
   if (!ctx || !cfg || cfg->struct_size != sizeof(admmq_factor_cfg)) return ADMMQ_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
   if (c->state < 1 || c->n_tokens < 1) return ADMMQ_ERR_STATE;
-  if (cfg->kind == ADMMQ_FACTOR_CHOLESKY || cfg->kind == ADMMQ_FACTOR_EIG) return ADMMQ_ERR_UNSUPPORTED;
   if (cfg->kind != ADMMQ_FACTOR_TRIDIAG) return ADMMQ_ERR_INVALID_ARG;
   if (cfg->T < 1 || cfg->T > c->T_max) return ADMMQ_ERR_SHAPE;
   if (!(cfg->damp_frac >= 0.0) || !isfinite(cfg->damp_frac)) return ADMMQ_ERR_INVALID_ARG;

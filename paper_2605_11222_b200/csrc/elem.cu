@@ -446,11 +446,7 @@ static int row_pass_blocks(Ctx* c, int p, size_t smem) {
 
 void launch_row_split(Ctx* c, const float* src, int p, bf16* hi, bf16* lo, float* row_inv) {
   const size_t smem = (size_t)c->n * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(row_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-    attr_set = true;
-  }
+  if (ensure_dynamic_smem((const void*)row_split_kernel, 64 * 1024) != cudaSuccess) return;   // the launch error check reports it
   row_split_kernel<<<row_pass_blocks(c, p, smem), ROW_THREADS, smem, c->stream>>>(src, p, c->n, hi, lo, row_inv);
   LAUNCH(c);
 }
@@ -549,11 +545,7 @@ error_planes_kernel(int p, int n, int gs, int ng, const float* __restrict__ W0,
 void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes,
                          const float* delta, const float* zero, bf16* Ehi, bf16* Elo, float* row_inv) {
   const size_t smem = (size_t)c->n * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(error_planes_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-    attr_set = true;
-  }
+  if (ensure_dynamic_smem((const void*)error_planes_kernel, 64 * 1024) != cudaSuccess) return;   // the launch error check reports it
   error_planes_kernel<<<row_pass_blocks(c, p, smem), ROW_THREADS, smem, c->stream>>>(
       p, c->n, gs, c->n / gs, W0, codes, delta, zero, Ehi, Elo, row_inv);
   LAUNCH(c);
@@ -749,11 +741,7 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
 
 void launch_admm_rows(Ctx* c, const EpiParams& P, int p, bf16* hi, bf16* lo, float* row_inv) {
   const size_t smem = (size_t)c->n * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(admm_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
-    attr_set = true;
-  }
+  if (ensure_dynamic_smem((const void*)admm_row_kernel, 64 * 1024) != cudaSuccess) return;   // the launch error check reports it
   int blocks = row_pass_blocks(c, p, smem);
   if (blocks > c->partial_slots) blocks = c->partial_slots;
   admm_row_kernel<<<blocks, ROW_THREADS, smem, c->stream>>>(P, p, c->n, hi, lo, row_inv);

@@ -28,8 +28,8 @@
 //                ADMM iteration the projection, dual update, residual sums and the next right-hand
 //                side -- through a per-warp staging buffer that makes the global accesses coalesced.
 //                The issuer runs up to two flushes into the next tile meanwhile.
-// Every wait is bounded: on expiry the kernel records ADMMQ_ERR_TIMEOUT, stops issuing work, lets
-// copies in flight land, frees tensor memory and returns.
+// Every wait is bounded: on expiry the kernel records ADMMQ_ERR_TIMEOUT, stops issuing work, waits (again
+// bounded) until the stage fills and MMAs already issued have completed, frees tensor memory and returns.
 #include <cuda.h>
 
 #include "internal.h"
@@ -42,7 +42,7 @@ constexpr int NPART = 2;                 // partial accumulators in tensor memor
 constexpr int WORKER_WARPS = 16;
 constexpr int TC_THREADS = 32 * (2 + WORKER_WARPS);
 constexpr int COLS_PER_THREAD = BN / 4;  // 64
-constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // about a second
+constexpr long long DRAIN_LIMIT_CYCLES = 20000000LL;    // bound of each wait of the abort path (~10 ms)
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -70,14 +70,14 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 // Bounded wait.  Returns false (and raises the abort flag + device status) when the limit runs out.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status) {
+                                          int* status, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   int spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if (++spins >= 32) {
       spins = 0;
-      if (*abort_flag || clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      if (*abort_flag || clock64() - t0 > limit) {
         *abort_flag = 1;
         raise_status(status, ST_TIMEOUT);
         return false;
@@ -89,10 +89,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // The same wait for a whole warp: lane 0 polls, the others sleep at the shuffle, so that the 16 worker
 // warps do not all hammer one barrier word.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                               int* status) {
+                                               int* status, long long limit) {
   int ok = 1;
-  if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status) ? 1 : 0;
+  if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, status, limit) ? 1 : 0;
   return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+// Wait of the abort path: bounded, raises nothing (the status is already set).
+__device__ __forceinline__ void mbar_wait_quiet(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity) && clock64() - t0 < DRAIN_LIMIT_CYCLES) {
+  }
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x,
                                             int y) {
@@ -337,15 +343,16 @@ __device__ __forceinline__ void epilogue_block(const EpiParams& P, int row0, int
 template <int NP, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_t fmt, EpiParams epi,
-               int* status) {
+               int* status, long long wait_limit, int hold_loads) {
   constexpr int A_BYTES = BM * BK * 2, BOX_BYTES = BN_BOX * BK * 2, B_BYTES = 2 * BOX_BYTES;
   constexpr int STAGE_BYTES = NP * (A_BYTES + B_BYTES);
   constexpr int STAGES = (NP == 1) ? 4 : 2;
   constexpr int KB_PER_FLUSH = (NP == 1) ? 3 : 1;        // 12 accumulating MMA steps per flush either way
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[3 * STAGES + 2 * NPART];
+  __shared__ __align__(8) uint64_t bars[3 * STAGES + 2 * NPART + 1];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
+  __shared__ uint32_t fill_state[3];       // producer's record for the abort path: armed / parity / half-armed stages
   __shared__ float red[WORKER_WARPS * 2];
   __shared__ __align__(16) float stage_all[WORKER_WARPS * STAGE_FLOATS];
 
@@ -358,9 +365,12 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
   const uint32_t pfull0 = smem_u32(&bars[2 * STAGES]);
   const uint32_t pempty0 = smem_u32(&bars[2 * STAGES + NPART]);
   const uint32_t elo0 = smem_u32(&bars[2 * STAGES + 2 * NPART]);   // two planes: the lo planes of a stage are free
+  const uint32_t drain_bar = smem_u32(&bars[3 * STAGES + 2 * NPART]);  // abort path: all issued MMAs have completed
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
+    fill_state[0] = fill_state[1] = fill_state[2] = 0u;
+    mbar_init(drain_bar, 1);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(full0 + 8 * s, NP == 2 ? 2 : 1);           // two planes: the lo and the hi half arrive separately
       mbar_init(empty0 + 8 * s, 1);
@@ -390,10 +400,15 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
 
   if (warp == 0) {
     // ===================== TMA producer =====================
-    if (lane == 0) {
+    // hold_loads (failure-handling tests only): the producer issues nothing, so the issuer's first wait runs out
+    // with no copy in flight.
+    if (lane == 0 && !hold_loads) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      // latest fill of every stage, for the abort path: bit s of `armed`: stage s was armed, of `par`: with which
+      // phase parity, of `half`: only the first of its two arrivals has been made
+      uint32_t armed = 0u, par = 0u, half = 0u;
       for (int u = blockIdx.x; u < sched.num_units && ok; u += gridDim.x) {
         const Unit un = unit_of(sched, u);
         if (lower && un.col0 > un.tm * BM + BM - 1) continue;
@@ -401,20 +416,27 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
         for (int kb = 0; kb < num_kb; ++kb) {
           const uint32_t sbase = tiles_base + stage * STAGE_BYTES;
           const uint32_t fb = full0 + 8 * stage;
+          const uint32_t bit = 1u << stage;
           if (NP == 2) {
             // the lo planes of a stage are released after the two cross products of its K block, a third of the
             // block's MMA time before the hi planes: their refill starts that much earlier
-            ok = mbar_wait(elo0 + 8 * stage, phase ^ 1u, abort_flag, status);
+            ok = mbar_wait(elo0 + 8 * stage, phase ^ 1u, abort_flag, status, wait_limit);
             if (!ok) break;
             mbar_expect_tx(fb, A_BYTES + boxes * BOX_BYTES);
+            armed |= bit;
+            half |= bit;
+            par = (par & ~bit) | (phase << stage);
             tma_load_2d(sbase + A_BYTES, &maps.a[1], fb, kb * BK, un.tm * BM);
             for (int bx = 0; bx < boxes; ++bx)
               tma_load_2d(sbase + NP * A_BYTES + B_BYTES + bx * BOX_BYTES, &maps.b[1], fb, kb * BK,
                           un.col0 + bx * BN_BOX);
           }
-          ok = mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag, status);
+          ok = mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag, status, wait_limit);
           if (!ok) break;
           mbar_expect_tx(fb, A_BYTES + boxes * BOX_BYTES);
+          armed |= bit;
+          half &= ~bit;
+          par = (par & ~bit) | (phase << stage);
           tma_load_2d(sbase, &maps.a[0], fb, kb * BK, un.tm * BM);
           for (int bx = 0; bx < boxes; ++bx)
             tma_load_2d(sbase + NP * A_BYTES + bx * BOX_BYTES, &maps.b[0], fb, kb * BK, un.col0 + bx * BN_BOX);
@@ -424,6 +446,9 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
           }
         }
       }
+      fill_state[0] = armed;
+      fill_state[1] = par;
+      fill_state[2] = half;
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
@@ -441,13 +466,13 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
         for (int kb = 0; kb < num_kb; ++kb) {
           if (kb % KB_PER_FLUSH == 0) {
             pb = (int)(g % NPART);
-            ok = mbar_wait(pempty0 + 8 * pb, ((g / NPART) & 1u) ^ 1u, abort_flag, status);
+            ok = mbar_wait(pempty0 + 8 * pb, ((g / NPART) & 1u) ^ 1u, abort_flag, status, wait_limit);
             if (!ok) break;
             tc_fence_after();
             d_tmem = tmem_base + (uint32_t)pb * BN;
             accumulate = 0;
           }
-          ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, status);
+          ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, status, wait_limit);
           if (!ok) break;
           tc_fence_after();
           const uint32_t sbase = tiles_base + stage * STAGE_BYTES;
@@ -504,7 +529,7 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
       for (int f = 0; f < num_flush; ++f) {
         if (f == pf_at && mine) epilogue_prefetch<EPI>(epi, row0 + lane, col0, M, N);
         const int pb = (int)(g % NPART);
-        ok = mbar_wait_warp(pfull0 + 8 * pb, (g / NPART) & 1u, abort_flag, status);
+        ok = mbar_wait_warp(pfull0 + 8 * pb, (g / NPART) & 1u, abort_flag, status, wait_limit);
         if (!ok) break;
         tc_fence_after();
         if (mine) {
@@ -549,9 +574,23 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
   }
   tc_fence_before();
   __syncthreads();
-  if (abort_flag_s) {                        // give copies in flight time to land before the CTA exits
-    const long long t0 = clock64();
-    while (clock64() - t0 < 2000000LL) {
+  if (abort_flag_s) {
+    // A wait ran out and every role has stopped.  Before shared and tensor memory are given back: (thread 0, the
+    // producer) every stage fill that was armed must have landed -- a stage with only the first of its two
+    // arrivals gets the second one here, without bytes, so that its barrier can complete; (thread 32, the
+    // issuer) every MMA issued so far must have completed, which a commit to a barrier of its own reports.
+    // These waits are bounded as well and raise nothing: the status word already holds the timeout.
+    if (threadIdx.x == 0) {
+      const uint32_t armed = fill_state[0], par = fill_state[1], half = fill_state[2];
+      for (int s = 0; s < STAGES; ++s)
+        if (armed >> s & 1u) {
+          if (half >> s & 1u) mbar_arrive(full0 + 8 * s);
+          mbar_wait_quiet(full0 + 8 * s, par >> s & 1u);
+        }
+    }
+    if (threadIdx.x == 32) {
+      tc_commit(drain_bar);
+      mbar_wait_quiet(drain_bar, 0u);
     }
     __syncthreads();
   }
@@ -612,16 +651,12 @@ static cudaError_t launch_tc(Ctx* c, const TcMaps& maps, int M, int N, int K, ui
   constexpr int STAGE_BYTES = NP * (BM * BK * 2 + BN * BK * 2);
   constexpr int STAGES = (NP == 1) ? 4 : 2;
   const size_t smem = (size_t)STAGES * STAGE_BYTES + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<NP, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  const cudaError_t ea = ensure_dynamic_smem((const void*)gemm_tc_kernel<NP, EPI>, (int)smem);
+  if (ea != cudaSuccess) return ea;
   const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = tiles < c->num_sms ? tiles : c->num_sms;
-  gemm_tc_kernel<NP, EPI><<<grid, TC_THREADS, smem, c->stream>>>(maps, M, N, K, fmt, epi, c->status);
+  gemm_tc_kernel<NP, EPI><<<grid, TC_THREADS, smem, c->stream>>>(maps, M, N, K, fmt, epi, c->status,
+                                                                   c->wait_limit_cycles, c->hold_loads);
   c->launches++;
   return cudaGetLastError();
 }

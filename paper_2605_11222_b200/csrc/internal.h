@@ -37,6 +37,8 @@ struct Ctx {
   int precondition = 1;
   double rho_host[4096];
   long long launches = 0;
+  long long wait_limit_cycles = 2000000000LL;   // bound of every device-side wait, about a second
+  int hold_loads = 0;           // failure-handling tests only: the product kernel's producer issues no loads
   // ---- workspace carve-up (device) ----
   char* ws = nullptr;
   size_t ws_bytes = 0;
@@ -78,6 +80,11 @@ struct Ctx {
 };
 
 constexpr int XT_ROWS = 16384;   // calibration rows handled per Hessian launch
+
+// Raises a kernel's dynamic shared-memory limit to at least `bytes` on the CURRENT device.  The attribute
+// belongs to a (kernel, device) pair, so the record of what was already set is kept per pair, under a
+// mutex: contexts on several GPUs of one process, and host threads, each get a correctly set-up kernel.
+cudaError_t ensure_dynamic_smem(const void* kernel, int bytes);
 
 // ---- elem.cu ----
 void launch_zero(Ctx* c, void* ptr, size_t bytes);

@@ -124,14 +124,16 @@ pair_gradient_kernel(const float* __restrict__ H, int n, int p, const int* __res
                      const float* __restrict__ d2buf, float* __restrict__ g) {
   const int b = chosen[0];
   if (b < 0) return;
-  const int j = blockIdx.y;
-  const float d1 = d1buf[j], d2 = d2buf[j];
-  if (d1 == 0.0f && d2 == 0.0f) return;
   const float* h1 = H + (size_t)pairs[2 * b] * n;
   const float* h2 = H + (size_t)pairs[2 * b + 1] * n;
-  float* gr = g + (size_t)j * n;
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
-    gr[i] = fmaf(d2, h2[i], fmaf(d1, h1[i], gr[i]));
+  // channels on grid.x (any d_out), column segments on grid.y
+  for (int j = blockIdx.x; j < p; j += gridDim.x) {
+    const float d1 = d1buf[j], d2 = d2buf[j];
+    if (d1 == 0.0f && d2 == 0.0f) continue;
+    float* gr = g + (size_t)j * n;
+    for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < n; i += gridDim.y * blockDim.x)
+      gr[i] = fmaf(d2, h2[i], fmaf(d1, h1[i], gr[i]));
+  }
 }
 
 cudaError_t launch_pair_round(Ctx* c, int p, int bits, int gs, float tau, unsigned char* codes,
@@ -144,7 +146,7 @@ cudaError_t launch_pair_round(Ctx* c, int p, int bits, int gs, float tau, unsign
   pair_apply_kernel<<<(p + 255) / 256, 256, 0, c->stream>>>(c->H, c->hdiag, n, p, gs, kmax, tau, codes, delta,
                                                             zero, Wq, g, pairs, c->ps_chosen, c->ps_d,
                                                             c->ps_d + p, d_moves, d_rounds);
-  dim3 grid((n + 1023) / 1024, p);
+  dim3 grid(p, (n + 1023) / 1024);
   pair_gradient_kernel<<<grid, 256, 0, c->stream>>>(c->H, n, p, pairs, c->ps_chosen, c->ps_d, c->ps_d + p, g);
   c->launches += 4;
   return cudaGetLastError();

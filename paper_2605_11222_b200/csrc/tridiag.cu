@@ -1084,11 +1084,7 @@ template <int EPT>
 static void launch_solve_t(Ctx* c, int p, int stage, int blocks) {
   const size_t fs = stage_factor_stride(c->n);
   const size_t smem = (size_t)2 * EPT * SOLVE_THREADS * sizeof(float);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaFuncSetAttribute(tridiag_solve_kernel<EPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    attr_set = true;
-  }
+  if (ensure_dynamic_smem((const void*)tridiag_solve_kernel<EPT>, (int)smem) != cudaSuccess) return;
   tridiag_solve_kernel<EPT><<<blocks, SOLVE_THREADS, smem, c->stream>>>(
       c->Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi, c->Y_lo,
       c->rs_Y);

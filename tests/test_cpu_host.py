@@ -22,7 +22,8 @@ def lib():
 
 def test_library_exports_every_declared_symbol(lib):
     from paper_2605_11222_b200 import binding
-    header = open(os.path.join(ROOT, "include", "admmq.h")).read()
+    inc = os.path.join(ROOT, "include")
+    header = "".join(open(os.path.join(inc, f)).read() for f in sorted(os.listdir(inc)) if f.endswith(".h"))
     declared = sorted(set(re.findall(r"\b(admmq_[a-z_0-9]+)\s*\(", header)))
     assert len(declared) >= 16
     for name in declared:
