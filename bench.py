@@ -5,9 +5,17 @@ One "step" = one pass of the whole hot path over one layer's calibration set:
 Hessian accumulation -> damping / scaling / factorisation -> T ADMM iterations -> local search
 (with the error report).  The workload at N = 1 is the Qwen3-8B q_proj-shaped layer
 (d_in = d_out = 4096, 262144 bf16 calibration rows, W3 asymmetric g128, T = 300).  With N > 1
-ranks every rank solves its own layer (independent problems, no data-path collective).
+ranks (one process per GPU; started by torchrun, or by this script itself when --gpus N > 1 is given
+without a launcher around it) there are three modes:
+  * default: every rank solves its own copy of the layer (independent problems, no data-path
+    collective, "scaling": "weak");
+  * --shard channels: ONE layer on all ranks -- token-sharded Hessian, one all-reduce of the n x n
+    accumulator, replicated factorisation, channel-sharded ADMM loop and local search ("strong");
+  * --stack-blocks B: the 7 B layers of config 5 dealt out to the ranks, wall time = slowest rank ("strong").
 
     python bench.py --gpus 1 --steps 3 --warmup 3
+    python bench.py --gpus 8 --stack-blocks 36
+    python bench.py --gpus 8 --workload cfg3_down --shard channels
     python bench.py --impl reference ...     # the fp64 CPU oracle on the host cores, bounded sample
 """
 from __future__ import annotations
@@ -29,6 +37,9 @@ import torch  # noqa: E402
 
 METRIC = "admmq_layer_solve_time"
 UNIT = "s"
+# ncu counters of gemm_tc_kernel<2, EPI_STORE> per launch, keyed by (d_in, d_out); the capture and its command
+# are summarised in profiles/gemm_tc_wupdate_4096x4096_ncu_full.txt
+PRODUCT_DRAM_BYTES_PER_LAUNCH = {(4096, 4096): 381.0e6}
 
 
 def load_peaks():
@@ -150,13 +161,15 @@ def run_reference(args, spec, wl):
         vals.append(est)
     wall = time.perf_counter() - t0
     v = float(np.mean(vals))
+    # `value` and `ms_per_step` are the whole-layer time the sample's pieces scale to (the metric is a layer's
+    # solve time, and the oracle needs minutes per layer); what one step really ran is under its own key
+    desc += f"; value = the pieces scaled to the whole layer, one sampled step itself ran {wall / args.steps:.2f} s"
     line = {
-        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * wall / args.steps,
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * v,
+        "sample_wall_ms_per_step": 1e3 * wall / args.steps,
         "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": spec.name, "d_in": spec.d_in, "d_out": spec.d_out,
-                                        "n_tokens": spec.n_tokens, "T": spec.T, "bits": spec.bits,
-                                        "group_size": spec.group_size},
+        "data": "synthetic", "config": layer_config(spec, 1),
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -165,16 +178,71 @@ def run_reference(args, spec, wl):
     return 0
 
 
+def layer_config(spec, world, parallelism=None):
+    """The `config` object of a one-layer line (the same keys in both arms)."""
+    return {"workload": spec.name, "d_in": spec.d_in, "d_out": spec.d_out, "n_tokens": spec.n_tokens, "T": spec.T,
+            "bits": spec.bits, "group_size": spec.group_size, "layers_per_step": world,
+            "l2": "inputs_exceed_l2", "parallelism": parallelism or f"layer-parallel x{world}"}
+
+
+def spawn_ranks(n: int) -> int:
+    """`--gpus N` with no launcher around this process: start N ranks of this same command line under
+    torch.distributed.run (one process per GPU, rendezvous on 127.0.0.1) and wait for them."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "WARN")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
+
+
+def init_ranks(args):
+    """(rank, world, local_rank, device or None).  NCCL on GPUs; gloo for --dry-run, which touches no GPU."""
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = None
+    if not args.dry_run:
+        torch.cuda.set_device(local_rank)
+        dev = torch.device("cuda", local_rank)
+    if world > 1 and not dist.is_initialized():
+        if args.dry_run:
+            dist.init_process_group("gloo")
+        else:
+            dist.init_process_group("nccl", device_id=dev)
+    return rank, world, local_rank, dev
+
+
+def finish_ranks():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.destroy_process_group()
+
+
+def gather_objects(obj, world):
+    import torch.distributed as dist
+    if world == 1:
+        return [obj]
+    out = [None] * world
+    dist.all_gather_object(out, obj)
+    return out
+
+
 # ---------------------------------------------------------------------------------------------------
 def run_stack(args, wl):
     """Config 5: every linear layer of the first B decoder blocks, each quantized once from a seeded calibration
     set generated on the device (generation timed separately).  Default: every layer has its own calibration set
     and factorisation.  With --shared-h the projections that read the same activations in a decoder block
     (q/k/v; gate/up) share one calibration set, one Hessian and one factorisation, and their weights are stacked
-    into one call: output channels are independent problems given H."""
-    from paper_2605_11222_b200 import binding as B
-    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
-    torch.cuda.set_device(dev)
+    into one call: output channels are independent problems given H.
+    With N > 1 ranks the calls are dealt out to the ranks (sharding.shard_layers: largest first, to the least
+    loaded rank); every rank solves its share, and the time reported is the slowest rank's."""
+    from paper_2605_11222_b200 import sharding
+    rank, world, local_rank, dev = init_ranks(args)
     layers = wl.config5(n_blocks=args.stack_blocks)
     if args.tokens > 0:
         import dataclasses
@@ -189,13 +257,32 @@ def run_stack(args, wl):
             groups += [blk[0:3], blk[3:4], blk[4:6], blk[6:7]]
     else:
         groups = [[l] for l in layers]
+    import dataclasses
+    # one cost-bearing stand-in per call (its d_out = the stacked width), dealt out like layers
+    calls = [dataclasses.replace(g[0], d_out=sum(l.d_out for l in g), name="+".join(l.name for l in g)) for g in groups]
+    mine = {c.name for c in sharding.shard_layers(calls, rank, world)}
+    my_groups = [g for g, c in zip(groups, calls) if c.name in mine]
+    config = {"workload": f"cfg5 first {args.stack_blocks} of 36 blocks", "layers": len(layers),
+              "calls": len(groups), "shared_h": bool(args.shared_h), "n_tokens": layers[0].n_tokens, "T": T,
+              "bits": layers[0].bits, "group_size": layers[0].group_size,
+              "parallelism": f"layers dealt to {world} rank(s), no data-path collective"}
+    if args.dry_run:
+        names = gather_objects([l.name for g in my_groups for l in g], world)
+        if rank == 0:
+            print(json.dumps({"metric": "admmq_stack_solve_time", "value": None, "unit": "s", "n_gpus": world,
+                              "scaling": "strong", "dry_run": True, "config": config, "layers_by_rank": names}))
+        finish_ranks()
+        return 0
+    from paper_2605_11222_b200 import binding as B
     solvers = {}
-    for n in sorted({g[0].d_in for g in groups}):
-        solvers[n] = B.Solver(n, max(sum(l.d_out for l in g) for g in groups if g[0].d_in == n), T_max=T, device=dev)
+    for n in sorted({g[0].d_in for g in my_groups}):
+        solvers[n] = B.Solver(n, max(sum(l.d_out for l in g) for g in my_groups if g[0].d_in == n), T_max=T, device=dev)
     per_shape, gen_s, solve_ms, moves = {}, 0.0, 0.0, 0
     torch.cuda.synchronize(dev)
+    if world > 1:
+        torch.distributed.barrier()
     t_wall = time.perf_counter()
-    for grp in groups:
+    for grp in my_groups:
         spec = grp[0]                                       # its calibration set serves the whole group
         sol = solvers[spec.d_in]
         t0 = time.perf_counter()
@@ -222,14 +309,82 @@ def run_stack(args, wl):
         a[1] += ms
         del Xs, W
     wall = time.perf_counter() - t_wall
-    print(json.dumps({
-        "metric": "admmq_stack_solve_time", "value": solve_ms / 1e3, "unit": "s", "n_gpus": 1,
-        "higher_is_better": False, "data": "synthetic", "dtype": "f16x2-split (fp32 accumulate)",
-        "config": {"workload": f"cfg5 first {args.stack_blocks} of 36 blocks", "layers": len(layers),
-                   "calls": len(groups), "shared_h": bool(args.shared_h),
-                   "n_tokens": layers[0].n_tokens, "T": T, "bits": layers[0].bits, "group_size": layers[0].group_size},
-        "wall_s_with_generation": wall, "generation_s": gen_s, "local_search_moves": moves,
-        "per_shape": {k: {"calls": v[0], "s_per_call": v[1] / v[0] / 1e3} for k, v in per_shape.items()}}))
+    solve_s = sharding.max_over_ranks(solve_ms / 1e3)       # the job ends with its slowest rank
+    wall_s = sharding.max_over_ranks(wall)
+    per_rank = gather_objects({"solve_s": solve_ms / 1e3, "calls": len(my_groups), "generation_s": gen_s}, world)
+    total_moves = int(sharding.sum_over_ranks(moves))
+    if rank == 0:
+        print(json.dumps({
+            "metric": "admmq_stack_solve_time", "value": solve_s, "unit": "s", "n_gpus": world,
+            "higher_is_better": False, "scaling": "strong", "data": "synthetic",
+            "dtype": "f16x2-split (fp32 accumulate)", "config": config,
+            "wall_s_with_generation": wall_s, "generation_s": gen_s, "local_search_moves": total_moves,
+            "per_rank": per_rank,
+            "per_shape": {k: {"calls": v[0], "s_per_call": v[1] / v[0] / 1e3} for k, v in per_shape.items()}}))
+    finish_ranks()
+    return 0
+
+
+def run_channel_sharded(args, spec, wl):
+    """ONE layer on all ranks (--shard channels): every rank accumulates the Hessian of its share of the
+    calibration chunks, one all-reduce(sum) of the n x n fp32 accumulator gives every rank the whole H, the
+    factorisation is replicated, and each rank runs the ADMM loop and the local search on its slice of output
+    channels.  A step is the whole layer; its time is the slowest rank's."""
+    from paper_2605_11222_b200 import sharding
+    rank, world, local_rank, dev = init_ranks(args)
+    slices = [list(sharding.channel_shard(spec.d_out, r, world)) for r in range(world)]
+    chunks = [[sharding.token_shard(spec.n_chunks, r, world).start, sharding.token_shard(spec.n_chunks, r, world).stop]
+              for r in range(world)]
+    config = layer_config(spec, 1, f"one layer on {world} rank(s): token-sharded Hessian + all-reduce, "
+                                   "replicated factorisation, channel-sharded ADMM and local search")
+    if args.dry_run:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT, "n_gpus": world, "scaling": "strong",
+                              "dry_run": True, "config": config, "channel_slices": slices, "token_chunks": chunks}))
+        finish_ranks()
+        return 0
+    from paper_2605_11222_b200 import binding as B
+    j0, j1 = slices[rank]
+    W = wl.gen_weight(spec, dev)
+    mine = sharding.token_shard(spec.n_chunks, rank, world)
+    Xs = {c: wl.gen_x_chunk(spec, c, dev) for c in mine}                  # this rank's token shard, resident
+    sol = B.Solver(spec.d_in, j1 - j0, T_max=spec.T, device=dev)
+    last = {}
+
+    def step():
+        out = sharding.solve_layer_sharded(sol, spec, W, lambda c: Xs[c])
+        last["info"] = out[3]
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize(dev)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_step = sharding.max_over_ranks(e0.elapsed_time(e1) / args.steps)
+    err = sharding.layer_error(last["info"])
+    moves = int(sharding.sum_over_ranks(last["info"]["rep_ls"].moves))
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": ms_step / 1e3, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f16x2-split (fp32 accumulate)", "data": "synthetic", "config": config,
+            "channel_slices": slices, "token_chunks": chunks, "allreduce_bytes_per_step": 4 * spec.d_in ** 2,
+            "err_after_local_search": err, "local_search_moves": moves, "clocks": clocks}))
+    finish_ranks()
     return 0
 
 
@@ -249,10 +404,19 @@ def main():
                          "36 = the whole stack), every layer once, and report the wall time")
     ap.add_argument("--shared-h", action="store_true",
                     help="with --stack-blocks: q/k/v and gate/up of a block share one Hessian and factorisation")
+    ap.add_argument("--shard", default="layers", choices=["layers", "channels"],
+                    help="with --gpus N > 1 and one layer: 'layers' = every rank its own layer (weak scaling), "
+                         "'channels' = one layer on all ranks (token-sharded Hessian, channel-sharded solve)")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="multi-rank plumbing only (gloo, no GPU, nothing solved): print what every rank would do")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    # --gpus N > 1 without a launcher around this process: start the N ranks here
+    if args.impl == "ours" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(args.gpus)
 
     from paper_2605_11222_b200 import workloads as wl
     rank = int(os.environ.get("RANK", "0"))
@@ -262,21 +426,20 @@ def main():
     base = wl.named_workload(args.workload)
     if args.tokens > 0:
         base = dataclasses.replace(base, n_tokens=args.tokens)
-    spec = dataclasses.replace(base, seed=base.seed + rank)
     if args.iters > 0:
-        spec = dataclasses.replace(spec, T=args.iters)
+        base = dataclasses.replace(base, T=args.iters)
 
     if args.impl == "reference":
-        return run_reference(args, spec, wl)
+        return run_reference(args, base, wl)
     if args.stack_blocks > 0:
         return run_stack(args, wl)
+    if args.shard == "channels":
+        return run_channel_sharded(args, base, wl)
+    spec = dataclasses.replace(base, seed=base.seed + rank)   # layer-parallel replicas: every rank its own layer
 
     from paper_2605_11222_b200 import binding as B, sharding
     import torch.distributed as dist
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    rank, world, local_rank, dev = init_ranks(args)
     peaks = load_peaks()
 
     n, p, T = spec.d_in, spec.d_out, spec.T
@@ -431,16 +594,9 @@ def main():
     flops_launch = 3 * 2.0 * p * n * n                     # three 16-bit MMAs per K step of the 2-plane split
     avg_ms = (ms_p1 + ms_p2) / max(1, n_p1 + n_p2)
     achieved = flops_launch / (avg_ms * 1e-3) / 1e12
-    # DRAM bytes per launch from the committed ncu summary (both products store their result: the plain epilogue)
-    traffic = None
-    prof = os.path.join(ROOT, "profiles", "gemm_tc_wupdate_4096x4096_ncu_full.txt")
-    if os.path.exists(prof) and (n, p) == (4096, 4096):
-        vals = {}
-        for ln in open(prof):
-            if ln.startswith("traffic_bytes_per_launch_"):
-                k, v = ln.strip().split("=")
-                vals[k] = float(v)
-        traffic = vals.get("traffic_bytes_per_launch_plain")
+    # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of this kernel from its ncu capture;
+    # known for the shape that was captured, null for every other
+    traffic = PRODUCT_DRAM_BYTES_PER_LAUNCH.get((n, p))
     roofline = {"kernel": "gemm_tc_kernel<2,*> (W-update products: two-plane fp16, 3 MMAs per K step)", "bound": "tensor",
                 "achieved": achieved, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
                 "frac": achieved / peaks["bf16_sustained"], "peak_source": peaks["source"] + ", bf16 sustained (fp16 and bf16 share the dense 16-bit peak)",
@@ -465,7 +621,8 @@ def main():
 
     kernel_rooflines = {
         "tridiag_solve": _hbm("tridiag_solve", 8.0 * p * n),          # read Y fp32, write two fp16 planes
-        "row_split": _hbm("row_split", 22.0 * p * n),                 # element update + plane split
+        # row pass: reads z 4, w_hat 4, V 4, codes 1; writes V 4, codes 1, two fp16 planes 4 bytes per element
+        "row_split": _hbm("row_split", 22.0 * p * n),
         "transpose": _hbm("transpose", 2.0 * x_bytes * chunk_rows * n),
     }
     ms_h, n_h = timing["hessian_product"]
@@ -485,9 +642,7 @@ def main():
         "metric": METRIC, "value": ms_step / 1e3, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "f16x2-split (fp32 accumulate)", "data": "synthetic",
-        "config": {"workload": spec.name, "d_in": n, "d_out": p, "n_tokens": spec.n_tokens, "T": T,
-                   "bits": spec.bits, "group_size": spec.group_size, "layers_per_step": world,
-                   "l2": "inputs_exceed_l2", "parallelism": f"layer-parallel x{world}"},
+        "config": layer_config(spec, world),
         "layers_per_s": world / (ms_step / 1e3),
         "w_update_useful_tflops": 4.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
         "w_update_executed_tflops": 12.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,

@@ -104,6 +104,18 @@ admmq_status admmq_hessian_accumulate(admmq_ctx* ctx, const void* d_X, admmq_dty
  * (Algorithm 1 takes H as its input).  d_H: [d_in][d_in] fp32, symmetric.  Counts as N = 1. */
 admmq_status admmq_hessian_set(admmq_ctx* ctx, const float* d_H);
 
+/* The accumulated state of step 1, for a Hessian whose calibration rows are spread over several contexts
+ * (for instance one per GPU, each fed its share of the tokens): every context exports its sum, the caller
+ * adds the sums element by element (an all-reduce) and imports the total, with the total row count, into
+ * every context before admmq_factor.  H = X^T X is a plain sum over the rows (Sec. 3.1), so the result is
+ * the Hessian of all rows.
+ * export: d_Hraw_out [d_in][d_in] fp32 receives sum_t x_t x_t^T of the rows accumulated so far (full
+ *         symmetric matrix, not divided by N); *h_tokens (host) receives the row count.  Synchronises.
+ * import: replaces the accumulated sum by d_Hraw (symmetric, same meaning) and the row count by n_tokens
+ *         (>= 1); like admmq_hessian_reset it may be the first call after admmq_create.  Asynchronous. */
+admmq_status admmq_hessian_export(admmq_ctx* ctx, float* d_Hraw_out, long long* h_tokens);
+admmq_status admmq_hessian_import(admmq_ctx* ctx, const float* d_Hraw, long long n_tokens);
+
 /* ---- Step 2: damping, diagonal scaling, factorisation. ---------------------------------------------
  * H = H_raw / N + damp_frac * mean(diag(H_raw / N)) I                         (App. D, damping)
  * s_i = sqrt(H_ii),  H~ = diag(1/s) H diag(1/s)                   (Sec. 3.2; Algorithm 1 lines 1-2)

@@ -28,6 +28,7 @@ EXPORTS = [
     "admmq_w_update", "admmq_local_search", "admmq_objective", "admmq_get_hessian",
     "admmq_launch_count", "admmq_set_timing", "admmq_reset_timing", "admmq_get_timing",
     "admmq_objective_static", "admmq_get_factor", "admmq_pair_swap", "admmq_test_set_wait",
+    "admmq_hessian_export", "admmq_hessian_import",
 ]
 T_HESSIAN_PRODUCT, T_TRANSPOSE, T_FACTOR, T_WUPDATE_PRODUCT1, T_TRIDIAG_SOLVE, T_WUPDATE_PRODUCT2, \
     T_GRADIENT_PRODUCT, T_LOCAL_SEARCH, T_ROW_SPLIT = range(9)
@@ -96,6 +97,8 @@ def load_library(path: Optional[str] = None):
     lib.admmq_hessian_reset.argtypes = [vp]
     lib.admmq_hessian_accumulate.argtypes = [vp, vp, ci, cll, cll]
     lib.admmq_hessian_set.argtypes = [vp, vp]
+    lib.admmq_hessian_export.argtypes = [vp, vp, C.POINTER(cll)]
+    lib.admmq_hessian_import.argtypes = [vp, vp, cll]
     lib.admmq_factor.argtypes = [vp, C.POINTER(FactorCfg)]
     lib.admmq_quantize_layer.argtypes = [vp, vp, ci, C.POINTER(QuantCfg), vp, vp, vp, vp, vp,
                                          C.POINTER(Report)]
@@ -189,6 +192,16 @@ class Solver:
 
     def hessian_set(self, H: torch.Tensor):
         _check(self.lib.admmq_hessian_set(self.h, _ptr(H)), "admmq_hessian_set")
+
+    def hessian_export(self):
+        """(sum_t x_t x_t^T as a full symmetric fp32 matrix, rows accumulated so far)."""
+        H = torch.empty(self.d_in, self.d_in, dtype=torch.float32, device=self.device)
+        ntok = C.c_longlong(0)
+        _check(self.lib.admmq_hessian_export(self.h, _ptr(H), C.byref(ntok)), "admmq_hessian_export")
+        return H, int(ntok.value)
+
+    def hessian_import(self, H_raw: torch.Tensor, n_tokens: int):
+        _check(self.lib.admmq_hessian_import(self.h, _ptr(H_raw), int(n_tokens)), "admmq_hessian_import")
 
     def factor(self, rho: Optional[Sequence[float]] = None, T: int = 0, rho0: float = 0.1,
                gamma: float = 1.1, damp_frac: float = 0.01, precondition: bool = True,

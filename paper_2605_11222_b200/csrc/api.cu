@@ -335,6 +335,29 @@ admmq_status admmq_hessian_set(admmq_ctx* ctx, const float* d_H) {
   return ADMMQ_OK;
 }
 
+admmq_status admmq_hessian_export(admmq_ctx* ctx, float* d_Hraw_out, long long* h_tokens) {
+  if (!ctx || !d_Hraw_out || !h_tokens || !aligned16(d_Hraw_out)) return ADMMQ_ERR_INVALID_ARG;
+  Ctx* c = &ctx->c;
+  if (c->state < 1) return ADMMQ_ERR_STATE;
+  launch_symmetric_copy(c, d_Hraw_out);
+  *h_tokens = c->n_tokens;
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) return ADMMQ_ERR_CUDA;
+  return ADMMQ_OK;
+}
+
+admmq_status admmq_hessian_import(admmq_ctx* ctx, const float* d_Hraw, long long n_tokens) {
+  if (!ctx || !d_Hraw || !aligned16(d_Hraw)) return ADMMQ_ERR_INVALID_ARG;
+  if (n_tokens < 1) return ADMMQ_ERR_SHAPE;
+  Ctx* c = &ctx->c;
+  if (cudaMemcpyAsync(c->H_raw, d_Hraw, (size_t)c->n * c->n * sizeof(float), cudaMemcpyDeviceToDevice,
+                      c->stream) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
+  launch_zero(c, c->status, 256);
+  c->n_tokens = n_tokens;
+  c->state = 1;
+  return ADMMQ_OK;
+}
+
 admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg) {
   if (!ctx || !cfg || cfg->struct_size != sizeof(admmq_factor_cfg)) return ADMMQ_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
@@ -446,6 +469,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   EpiParams e{};
   e.kind = EPI_ADMM;
   e.Whs = c->Whs;
+  e.W0 = d_W0;
   e.V = c->V;
   e.codes = d_codes;
   e.s = c->s;
@@ -467,9 +491,9 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     bool refresh = false;
     for (int q = 0; q < cfg->n_refresh; ++q) refresh = refresh || (cfg->h_refresh_iters[q] == t);
     if (refresh) {
-      // grid refresh attempt: W^(t+1) is stored by the plain epilogue, then evaluated on both grids
+      // grid refresh attempt: z = W^(t+1) - W_hat' is stored by the plain epilogue, then evaluated on both grids
       EpiParams w = e;
-      w.kind = EPI_WOUT;
+      w.kind = EPI_STORE;
       w.C = c->Y;
       w.ldc = n;
       if (w_update_products(ctx, p, t, w) != cudaSuccess) return ADMMQ_ERR_CUDA;
@@ -529,7 +553,7 @@ admmq_status admmq_w_update(admmq_ctx* ctx, const float* d_W0, int d_out, int gr
   Ctx* c = &ctx->c;
   const int n = c->n, p = d_out, gs = group_of(n, group_size);
   launch_scale_weights(c, d_W0, p);
-  launch_init_rhs(c, p, gs, d_codes, d_scale, d_zero, d_V, (float)(1.0 / rho), c->Y);
+  launch_init_rhs(c, d_W0, p, gs, d_codes, d_scale, d_zero, d_V, (float)(1.0 / rho), c->Y);
   launch_row_split(c, c->Y, p, c->R_hi, c->R_lo, c->rs_R);
   const int stage = c->T_max;                              // spare slot for an ad-hoc penalty
   ctx->rho_adhoc = rho;

@@ -141,6 +141,21 @@ __global__ void finalize_full_kernel(const float* __restrict__ Hraw, int n, doub
   A64[(long long)a * n + b] = (double)h / (s64[a] * s64[b]);
 }
 
+// Full symmetric copy of the accumulator, whose lower triangle is the valid half.
+__global__ void symmetric_copy_kernel(const float* __restrict__ Hraw, int n, float* __restrict__ out) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  const int a = blockIdx.y;
+  if (b >= n) return;
+  const int lo = min(a, b), hi = max(a, b);
+  out[(long long)a * n + b] = Hraw[(long long)hi * n + lo];
+}
+
+void launch_symmetric_copy(Ctx* c, float* out) {
+  dim3 grid((c->n + 255) / 256, c->n);
+  symmetric_copy_kernel<<<grid, 256, 0, c->stream>>>(c->H_raw, c->n, out);
+  LAUNCH(c);
+}
+
 void launch_finalize(Ctx* c, double damp_frac, int precondition) {
   const int n = c->n;
   const double inv_N = 1.0 / (double)c->n_tokens;
@@ -457,21 +472,22 @@ __global__ void init_rhs_kernel(long long total, int n, int gs, int ng,
                                 const unsigned char* __restrict__ codes,
                                 const float* __restrict__ delta, const float* __restrict__ zero,
                                 const float* __restrict__ V, float inv_rho, const float* __restrict__ s,
-                                const float* __restrict__ Whs, float* __restrict__ R) {
+                                const float* __restrict__ W0, float* __restrict__ R) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
   const int col = (int)(idx % n);
   const long long row = idx / n;
   const long long gi = row * ng + col / gs;
-  const float d = s[col] * (zero[gi] + delta[gi] * (float)codes[idx]);
-  R[idx] = d - V[idx] * inv_rho - Whs[idx];
+  // D - W_hat' = s (z0 + Delta k - w_hat): the difference of weight-sized numbers is taken in fp64
+  const double e = (double)s[col] * fma((double)delta[gi], (double)codes[idx], (double)zero[gi] - (double)W0[idx]);
+  R[idx] = fmaf(-V[idx], inv_rho, (float)e);
 }
 
-void launch_init_rhs(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
+void launch_init_rhs(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes, const float* delta,
                      const float* zero, const float* V_in, float inv_rho, float* R_out) {
   const long long total = (long long)p * c->n;
   init_rhs_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
-      total, c->n, gs, c->n / gs, codes, delta, zero, V_in, inv_rho, c->s, c->Whs, R_out);
+      total, c->n, gs, c->n / gs, codes, delta, zero, V_in, inv_rho, c->s, W0, R_out);
   LAUNCH(c);
 }
 
@@ -552,17 +568,18 @@ void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned 
 }
 
 // ------------------------------------------------------------------------------------------------
-// Grid refresh (Sec. 3.3 "Grid refresh", App. B) at one iteration, from the stored W^(t+1):
-//   eval:   per (channel, group) refit (Delta', z0') on the unscaled target (W + V/rho)/s by the initial
-//           fitting rule, project the target on the old and on the new grid, sum both squared distances;
+// Grid refresh (Sec. 3.3 "Grid refresh", App. B) at one iteration, from the stored product z = W^(t+1) - W_hat':
+//   eval:   per (channel, group) refit (Delta', z0') on the unscaled target Sigma W~ = w_hat + (z + V/rho)/s by
+//           the initial fitting rule, project the target on the old and on the new grid, sum both squared distances;
 //   decide: new grid kept iff its sum <= the old one (Eq. of App. B) and no refresh was accepted before;
 //   apply:  the ADMM element update (projection, dual, residual sums, next right-hand side) with the grid
-//           that was kept.  Same arithmetic as the fused epilogue.
+//           that was kept.  Same arithmetic as the row pass: targets and grid points relative to the weight,
+//           weight-sized differences and the rounding decisions in fp64.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-refresh_eval_kernel(const float* __restrict__ Wc, const float* __restrict__ V, const float* __restrict__ s,
-                    const float* __restrict__ inv_s, int p, int n, int gs, int kmax, int symmetric,
-                    float inv_rho, const float* __restrict__ delta, const float* __restrict__ zero,
+refresh_eval_kernel(const float* __restrict__ Zc, const float* __restrict__ W0, const float* __restrict__ V,
+                    const float* __restrict__ s, const float* __restrict__ inv_s, int p, int n, int gs, int kmax,
+                    int symmetric, float inv_rho, const float* __restrict__ delta, const float* __restrict__ zero,
                     float* __restrict__ cand_delta, float* __restrict__ cand_zero, double* __restrict__ partial) {
   __shared__ double scratch[32];
   const int ng = n / gs, lane = threadIdx.x & 31;
@@ -572,43 +589,46 @@ refresh_eval_kernel(const float* __restrict__ Wc, const float* __restrict__ V, c
        gw += ((long long)gridDim.x * blockDim.x) >> 5) {
     const int j = (int)(gw / ng), gq = (int)(gw % ng);
     const size_t base = (size_t)j * n + (size_t)gq * gs;
-    float lo = INFINITY, hi = -INFINITY;
+    double lo = INFINITY, hi = -INFINITY;
     for (int i = lane; i < gs; i += 32) {
-      const float y = fmaf(V[base + i], inv_rho, Wc[base + i]) * inv_s[gq * gs + i];
-      lo = fminf(lo, y);
-      hi = fmaxf(hi, y);
+      const float u = fmaf(V[base + i], inv_rho, Zc[base + i]) * inv_s[gq * gs + i];
+      const double y = (double)W0[base + i] + (double)u;
+      lo = fmin(lo, y);
+      hi = fmax(hi, y);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-      lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
-      hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+      lo = fmin(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+      hi = fmax(hi, __shfl_xor_sync(0xffffffffu, hi, o));
     }
     if (symmetric) {
-      hi = fmaxf(fabsf(lo), fabsf(hi));
+      hi = fmax(fabs(lo), fabs(hi));
       lo = -hi;
     }
-    float dn = (hi - lo) / (float)kmax;
-    if (hi - lo == 0.f) dn = 1.f;
-    const float zn = lo;
+    float dn = (float)((hi - lo) / (double)kmax);          // the grid is stored in fp32
+    if (hi - lo == 0.0) dn = 1.f;
+    const float zn = (float)lo;
     if (lane == 0) {
       cand_delta[gw] = dn;
       cand_zero[gw] = zn;
     }
     const float d0 = delta[gw], z0 = zero[gw];
-    const float id0 = __frcp_rn(d0), idn = __frcp_rn(dn);
-    float a = 0.f, b = 0.f;
+    const double id0 = 1.0 / (double)d0, idn = 1.0 / (double)dn;
+    double a = 0.0, b = 0.0;
     for (int i = lane; i < gs; i += 32) {
-      const float sv = s[gq * gs + i];
-      const float wt = fmaf(V[base + i], inv_rho, Wc[base + i]);
-      const float y = wt * inv_s[gq * gs + i];
-      const float k0 = fminf(fmaxf(rintf((y - z0) * id0), 0.f), (float)kmax);
-      const float kn = fminf(fmaxf(rintf((y - zn) * idn), 0.f), (float)kmax);
-      const float eo = sv * (z0 + d0 * k0) - wt, en = sv * (zn + dn * kn) - wt;
-      a = fmaf(eo, eo, a);
-      b = fmaf(en, en, b);
+      const double sv = (double)s[gq * gs + i];
+      const double u = (double)(fmaf(V[base + i], inv_rho, Zc[base + i]) * inv_s[gq * gs + i]);
+      const double w = (double)W0[base + i];
+      const double k0 = fmin(fmax(rint(((w - (double)z0) + u) * id0), 0.0), (double)kmax);
+      const double kn = fmin(fmax(rint(((w - (double)zn) + u) * idn), 0.0), (double)kmax);
+      // D - W~ in scaled coordinates: s ((z0 + Delta k - w_hat) - u)
+      const double eo = sv * (fma((double)d0, k0, (double)z0 - w) - u);
+      const double en = sv * (fma((double)dn, kn, (double)zn - w) - u);
+      a = fma(eo, eo, a);
+      b = fma(en, en, b);
     }
-    e_old += (double)warp_sum(a);
-    e_new += (double)warp_sum(b);
+    e_old += warp_sum(a);
+    e_new += warp_sum(b);
   }
   e_old = block_sum(e_old, scratch);       // every lane of a warp carries its warp's sums: divide by 32 below
   e_new = block_sum(e_new, scratch);
@@ -644,7 +664,8 @@ __global__ void refresh_commit_kernel(long long groups, const int* __restrict__ 
   zero[i] = cand_zero[i];
 }
 
-// The ADMM element update from a stored W^(t+1) (in P.Rnext, overwritten by the next right-hand side).
+// The ADMM element update from the stored product z = W^(t+1) - W_hat' (in P.Rnext, overwritten by the next
+// right-hand side).
 __global__ void __launch_bounds__(256) admm_elementwise_kernel(EpiParams P, long long total, int n) {
   __shared__ float red[32];
   float r2 = 0.f, s2 = 0.f;
@@ -653,10 +674,8 @@ __global__ void __launch_bounds__(256) admm_elementwise_kernel(EpiParams P, long
     const int col = (int)(idx % n);
     const long long row = idx / n;
     const long long gi = row * P.n_groups + col / P.group_size;
-    const float dl = P.delta[gi], z0 = P.zero[gi];
-    const float wh = P.Whs[idx];
-    AdmmElem e = admm_elem(P.Rnext[idx] - wh, wh, P.V[idx], P.first_iter ? 0 : (int)P.codes[idx], P.s[col],
-                           P.inv_s[col], dl, __frcp_rn(dl), z0, P);
+    AdmmElem e = admm_elem(P.Rnext[idx], P.W0[idx], P.V[idx], P.first_iter ? 0 : (int)P.codes[idx], P.s[col],
+                           P.inv_s[col], grid_g(P.delta[gi], P.zero[gi]), P);
     P.codes[idx] = e.code;
     P.V[idx] = e.v_new;
     P.Rnext[idx] = e.r_next;
@@ -689,7 +708,7 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
     float m = 0.0f;
     for (int i = threadIdx.x * 4; i < n; i += ROW_THREADS * 4) {          // n is a multiple of 8
       const float4 z = *reinterpret_cast<const float4*>(P.C + base + i);
-      const float4 wh = *reinterpret_cast<const float4*>(P.Whs + base + i);
+      const float4 wh = *reinterpret_cast<const float4*>(P.W0 + base + i);
       const float4 v = *reinterpret_cast<const float4*>(P.V + base + i);
       const float4 sv = *reinterpret_cast<const float4*>(P.s + i);
       const float4 si = *reinterpret_cast<const float4*>(P.inv_s + i);
@@ -697,18 +716,18 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
       if (!P.first_iter) k = *reinterpret_cast<const uchar4*>(P.codes + base + i);
       const int g0 = gsh >= 0 ? i >> gsh : i / gs;
       const int g3 = gsh >= 0 ? (i + 3) >> gsh : (i + 3) / gs;
-      const float d0 = dlt[g0], z0 = zr[g0], id0 = __frcp_rn(d0);
-      AdmmElem e0 = admm_elem(z.x, wh.x, v.x, k.x, sv.x, si.x, d0, id0, z0, P);
+      const GridG gg = grid_g(dlt[g0], zr[g0]);
+      AdmmElem e0 = admm_elem(z.x, wh.x, v.x, k.x, sv.x, si.x, gg, P);
       AdmmElem e1, e2, e3;
       if (g3 == g0) {
-        e1 = admm_elem(z.y, wh.y, v.y, k.y, sv.y, si.y, d0, id0, z0, P);
-        e2 = admm_elem(z.z, wh.z, v.z, k.z, sv.z, si.z, d0, id0, z0, P);
-        e3 = admm_elem(z.w, wh.w, v.w, k.w, sv.w, si.w, d0, id0, z0, P);
+        e1 = admm_elem(z.y, wh.y, v.y, k.y, sv.y, si.y, gg, P);
+        e2 = admm_elem(z.z, wh.z, v.z, k.z, sv.z, si.z, gg, P);
+        e3 = admm_elem(z.w, wh.w, v.w, k.w, sv.w, si.w, gg, P);
       } else {
         const int g1 = (i + 1) / gs, g2 = (i + 2) / gs;
-        e1 = admm_elem(z.y, wh.y, v.y, k.y, sv.y, si.y, dlt[g1], __frcp_rn(dlt[g1]), zr[g1], P);
-        e2 = admm_elem(z.z, wh.z, v.z, k.z, sv.z, si.z, dlt[g2], __frcp_rn(dlt[g2]), zr[g2], P);
-        e3 = admm_elem(z.w, wh.w, v.w, k.w, sv.w, si.w, dlt[g3], __frcp_rn(dlt[g3]), zr[g3], P);
+        e1 = admm_elem(z.y, wh.y, v.y, k.y, sv.y, si.y, grid_g(dlt[g1], zr[g1]), P);
+        e2 = admm_elem(z.z, wh.z, v.z, k.z, sv.z, si.z, grid_g(dlt[g2], zr[g2]), P);
+        e3 = admm_elem(z.w, wh.w, v.w, k.w, sv.w, si.w, grid_g(dlt[g3], zr[g3]), P);
       }
       *reinterpret_cast<uchar4*>(P.codes + base + i) = make_uchar4(e0.code, e1.code, e2.code, e3.code);
       *reinterpret_cast<float4*>(P.V + base + i) = make_float4(e0.v_new, e1.v_new, e2.v_new, e3.v_new);
@@ -756,7 +775,7 @@ void launch_grid_refresh(Ctx* c, const EpiParams& P, int p, int bits, int symmet
   float* cand_zero = reinterpret_cast<float*>(c->R_lo);       // and the row pass that rewrites them
   long long want = (groups * 32 + 255) / 256;
   const int blocks = (int)(want < 1184 ? want : 1184);
-  refresh_eval_kernel<<<blocks, 256, 0, c->stream>>>(P.Rnext, P.V, P.s, P.inv_s, p, n, gs, (1 << bits) - 1,
+  refresh_eval_kernel<<<blocks, 256, 0, c->stream>>>(P.Rnext, P.W0, P.V, P.s, P.inv_s, p, n, gs, (1 << bits) - 1,
                                                      symmetric, P.inv_rho, delta, zero, cand_delta, cand_zero,
                                                      c->ps_totals);
   refresh_decide_kernel<<<1, 256, 0, c->stream>>>(c->ps_totals, blocks, iter, flags);

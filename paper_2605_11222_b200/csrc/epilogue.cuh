@@ -19,7 +19,8 @@ struct EpiParams {
   long long ldc;
   int lower_only;           // ACCUM: skip elements with col > row (symmetric product)
   // ---- ADMM state, all [p][n] row-major with leading dimension n ----
-  const float* Whs;         // W_hat' = s_i * W_hat  (scaled pre-trained weights)
+  const float* Whs;         // W_hat' = s_i * W_hat  (scaled pre-trained weights; WOUT only)
+  const float* W0;          // W_hat, unscaled, as the caller passed it (ADMM element update)
   float* V;                 // dual V (in/out)
   unsigned char* codes;     // codes of D (in: D^(t), out: D^(t+1))
   const float* s;           // [n] s_i = sqrt(H_ii)
@@ -47,30 +48,50 @@ __device__ __forceinline__ float epi_row_factor(const EpiParams& P, int row) {
   return f;
 }
 
-// One element of the fused ADMM epilogue.  z = [Q (T/rho + I)^{-1} Q^T R]_{ji} is the accumulator, so
+// One element of the ADMM update (Eq. 8-10).  z = [Q (T/rho + I)^{-1} Q^T R]_{ji} is the product's output, so
 // that W = W_hat' + z is the W-update of Eq. 7 written for the error W - W_hat'.
+//
+// Every quantity here is kept RELATIVE to the pre-trained weight, i.e. at the size of a grid step, never at
+// the size of the weight itself: in unscaled coordinates the projection target is
+//     Sigma W~ = w_hat + (z + V/rho) / s,
+// so the code is k = rint(((w_hat - z0) + (z + V/rho)/s) / Delta), and the grid point enters only through its
+// distance from the weight, D - W_hat' = s (z0 + Delta k - w_hat).  The two places where numbers of the
+// weight's size meet -- (w_hat - z0) and (Delta k - (w_hat - z0)) -- are evaluated in fp64, where both are
+// exact; the rounding decision of Eq. 10 is taken in fp64 like the oracle's.  (In plain fp32 the sums
+// W_hat' + z, s (z0 + Delta k) and y - z0 each round at the weight's magnitude, up to 2^(bits-1) grid steps:
+// ~1e-6 of a step per iteration at 4 bits, which is what decided most of the codes that differed from an
+// fp64 run.)
 struct AdmmElem {
   unsigned char code;
   float v_new, r_next, dr2, ds2;
 };
-// The two divisions of the projection are taken as products with 1 / s_i and 1 / Delta (each correctly
-// rounded): the epilogue runs on the critical path of every tile, and a full-precision division costs as
-// much as the rest of the element.
-__device__ __forceinline__ AdmmElem admm_elem(float z, float wh, float v, int code_old, float s, float inv_s,
-                                              float dl, float inv_dl, float z0, const EpiParams& P) {
+// Constants of one (channel, group): Delta, z0 and 1 / Delta in fp64.
+struct GridG {
+  float dl, z0;
+  double inv_dl;
+};
+__device__ __forceinline__ GridG grid_g(float dl, float z0) {
+  GridG g;
+  g.dl = dl;
+  g.z0 = z0;
+  g.inv_dl = 1.0 / (double)dl;
+  return g;
+}
+__device__ __forceinline__ AdmmElem admm_elem(float z, float w0, float v, int code_old, float s, float inv_s,
+                                              const GridG& g, const EpiParams& P) {
   AdmmElem o;
-  const float w = wh + z;                                  // W^(t+1)
-  const float wt = fmaf(v, P.inv_rho, w);                  // target W~ = W + V/rho          (Eq. 8)
-  const float y = wt * inv_s;                              // unscaled coordinate Sigma W~
-  float k = rintf((y - z0) * inv_dl);                      // nearest level, ties to even    (Eq. 10)
-  k = fminf(fmaxf(k, 0.0f), (float)P.kmax);
-  const float d_new = s * (z0 + dl * k);                   // D^(t+1), scaled coordinates
-  const float d_old = P.first_iter ? wh : s * (z0 + dl * (float)code_old);
-  const float wd = w - d_new;
-  const float dd = d_new - d_old;
-  o.code = (unsigned char)k;
-  o.v_new = v + P.rho * wd;                                // V += rho (W - D)               (Eq. 9)
-  o.r_next = d_new - o.v_new * P.inv_rho_next - wh;        // next R = D - V/rho' - W_hat'
+  const double a = (double)w0 - (double)g.z0;              // w_hat - z0, exact
+  const float u = fmaf(v, P.inv_rho, z) * inv_s;           // (W~ - W_hat') / s: target minus weight  (Eq. 8)
+  double k = rint((a + (double)u) * g.inv_dl);             // nearest level, ties to even    (Eq. 10)
+  k = fmin(fmax(k, 0.0), (double)P.kmax);
+  const float e_new = (float)((double)s * fma((double)g.dl, k, -a));        // D^(t+1) - W_hat'
+  const float e_old = P.first_iter ? 0.0f                                   // D^(0) = W_hat'
+                                   : (float)((double)s * fma((double)g.dl, (double)code_old, -a));
+  const float wd = z - e_new;                              // W^(t+1) - D^(t+1)
+  const float dd = e_new - e_old;                          // D^(t+1) - D^(t)
+  o.code = (unsigned char)(int)k;
+  o.v_new = fmaf(P.rho, wd, v);                            // V += rho (W - D)               (Eq. 9)
+  o.r_next = fmaf(-o.v_new, P.inv_rho_next, e_new);        // next R = D - V/rho' - W_hat'
   o.dr2 = wd * wd;
   o.ds2 = dd * dd;
   return o;
@@ -91,8 +112,8 @@ __device__ __forceinline__ void epi_scalar(const EpiParams& P, int row, int col,
     const int g = col / P.group_size;
     const float dl = P.delta[(long long)row * P.n_groups + g];
     const float z0 = P.zero[(long long)row * P.n_groups + g];
-    AdmmElem e = admm_elem(acc, P.Whs[idx], P.V[idx], P.first_iter ? 0 : (int)P.codes[idx], P.s[col],
-                           P.inv_s[col], dl, __frcp_rn(dl), z0, P);
+    AdmmElem e = admm_elem(acc, P.W0[idx], P.V[idx], P.first_iter ? 0 : (int)P.codes[idx], P.s[col],
+                           P.inv_s[col], grid_g(dl, z0), P);
     P.codes[idx] = e.code;
     P.V[idx] = e.v_new;
     P.Rnext[idx] = e.r_next;

@@ -234,7 +234,7 @@ __device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, 
   const float a[4] = {acc.x, acc.y, acc.z, acc.w};
   if (EPI == EPI_ADMM) {
     const long long o = (long long)row * N + col;
-    const float4 w = *reinterpret_cast<const float4*>(P.Whs + o);
+    const float4 w = *reinterpret_cast<const float4*>(P.W0 + o);
     const float4 v = *reinterpret_cast<const float4*>(P.V + o);
     const float4 s = *reinterpret_cast<const float4*>(P.s + col);
     const float4 is = *reinterpret_cast<const float4*>(P.inv_s + col);
@@ -246,20 +246,17 @@ __device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, 
     const float si[4] = {is.x, is.y, is.z, is.w};
     const bool one_group = (P.group_size & 3) == 0;        // then the 4 columns share (Delta, z0)
     long long gi = (long long)row * P.n_groups + col / P.group_size;
-    float dl = P.delta[gi], z0 = P.zero[gi];
-    float inv_dl = __frcp_rn(dl);
+    GridG gg = grid_g(P.delta[gi], P.zero[gi]);
     float vn[4], rn[4];
     uint32_t cn = 0u;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       if (!one_group && e > 0) {
         gi = (long long)row * P.n_groups + (col + e) / P.group_size;
-        dl = P.delta[gi];
-        z0 = P.zero[gi];
-        inv_dl = __frcp_rn(dl);
+        gg = grid_g(P.delta[gi], P.zero[gi]);
       }
       const int code_old = (int)((codes >> (8 * e)) & 0xffu);
-      AdmmElem r = admm_elem(a[e], wh[e], vv[e], code_old, ss[e], si[e], dl, inv_dl, z0, P);
+      AdmmElem r = admm_elem(a[e], wh[e], vv[e], code_old, ss[e], si[e], gg, P);
       vn[e] = r.v_new;
       cn |= (uint32_t)r.code << (8 * e);
       rn[e] = r.r_next;
@@ -296,8 +293,8 @@ __device__ __forceinline__ void epilogue_prefetch(const EpiParams& P, int row, i
   if (row >= M || col0 + COLS_PER_THREAD > N) return;
   if (EPI == EPI_ADMM) {
     const long long o = (long long)row * N + col0;
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(P.Whs + o));
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(P.Whs + o + 32));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(P.W0 + o));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(P.W0 + o + 32));
     asm volatile("prefetch.global.L2 [%0];" ::"l"(P.V + o));
     asm volatile("prefetch.global.L2 [%0];" ::"l"(P.V + o + 32));
     if (!P.first_iter) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.codes + o));

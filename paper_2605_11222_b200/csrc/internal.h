@@ -91,6 +91,7 @@ void launch_zero(Ctx* c, void* ptr, size_t bytes);
 void launch_transpose_split(Ctx* c, const void* X, int is_bf16, long long rows, long long ldx, int n,
                             bf16* XT_hi, bf16* XT_lo, long long ldt);
 void launch_finalize(Ctx* c, double damp_frac, int precondition);
+void launch_symmetric_copy(Ctx* c, float* out);      // H_raw (lower triangle valid) -> full symmetric matrix
 void launch_grid_fit(Ctx* c, const float* W0, int p, int bits, int gs, int symmetric, float* delta,
                      float* zero);
 void launch_admm_rows(Ctx* c, const EpiParams& P, int p, bf16* hi, bf16* lo, float* row_inv);
@@ -101,7 +102,7 @@ void launch_operand_scales(Ctx* c);   // fscal from diag(H)
 void launch_split_f64(Ctx* c, const double* src, int n, bf16* hi, bf16* lo, bf16* thi, bf16* tlo);
 void launch_split_f32(Ctx* c, const float* src, long long count, bf16* hi, bf16* lo);
 void launch_row_split(Ctx* c, const float* src, int p, bf16* hi, bf16* lo, float* row_inv);
-void launch_init_rhs(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
+void launch_init_rhs(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes, const float* delta,
                      const float* zero, const float* V_in, float inv_rho, float* R_out);
 void launch_reduce_partials(Ctx* c, int T, float* resid);
 void launch_dequant(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
