@@ -35,6 +35,7 @@ sys.path.insert(0, ROOT)
 import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
+DTYPE = "f16x2-split (fp32 accumulate; one fp16 plane in the late iterations, where it resolves the products below fp32)"
 METRIC = "admmq_layer_solve_time"
 UNIT = "s"
 # ncu counters of gemm_tc_kernel<2, EPI_STORE> per launch, keyed by (d_in, d_out); the capture and its command
@@ -317,7 +318,7 @@ def run_stack(args, wl):
         print(json.dumps({
             "metric": "admmq_stack_solve_time", "value": solve_s, "unit": "s", "n_gpus": world,
             "higher_is_better": False, "scaling": "strong", "data": "synthetic",
-            "dtype": "f16x2-split (fp32 accumulate)", "config": config,
+            "dtype": DTYPE, "config": config,
             "wall_s_with_generation": wall_s, "generation_s": gen_s, "local_search_moves": total_moves,
             "per_rank": per_rank,
             "per_shape": {k: {"calls": v[0], "s_per_call": v[1] / v[0] / 1e3} for k, v in per_shape.items()}}))
@@ -381,7 +382,7 @@ def run_channel_sharded(args, spec, wl):
         print(json.dumps({
             "metric": METRIC, "value": ms_step / 1e3, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": False, "scaling": "strong",
-            "vs_baseline": None, "dtype": "f16x2-split (fp32 accumulate)", "data": "synthetic", "config": config,
+            "vs_baseline": None, "dtype": DTYPE, "data": "synthetic", "config": config,
             "channel_slices": slices, "token_chunks": chunks, "allreduce_bytes_per_step": 4 * spec.d_in ** 2,
             "err_after_local_search": err, "local_search_moves": moves, "clocks": clocks}))
     finish_ranks()
@@ -525,6 +526,17 @@ def main():
                                          zero=zero, resid=resid, fused_epilogue=True)
     fused_variant = {"quantize_layer_ms": fu_rep.ms, "err_admm": fu_rep.err_before}
 
+    # ---- the same run with two operand planes in every iteration, and the default run through the same call ----
+    _, _, _, tp_rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, codes=codes, scale=scale,
+                                         zero=zero, resid=resid, product_planes=2)
+    c_two = codes.clone()
+    _, _, _, df_rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, codes=codes, scale=scale,
+                                         zero=zero, resid=resid)
+    planes_variant = {"two_planes_always_ms": tp_rep.ms, "default_ms": df_rep.ms,
+                      "default_one_plane_iterations": df_rep.one_plane_iters,
+                      "err_admm_two_planes": tp_rep.err_before, "err_admm_default": df_rep.err_before,
+                      "codes_equal_fraction": float((c_two == codes).float().mean().item())}
+
     # ---- a run whose grid comes from the MSE search for the clipping ratio, 100 candidates down to 0.8
     #      (another widened row: measured, not part of `value`), followed by the local search ----
     _, _, _, cl_rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, codes=codes, scale=scale,
@@ -588,12 +600,18 @@ def main():
             dist.destroy_process_group()
         return 0
 
-    # ---- roofline of the dominant kernel: the split-bf16 tcgen05 product of the W-update ----
+    # ---- roofline of the dominant kernel: the two-plane fp16 tcgen05 product of the W-update ----
+    # With d_out >= 1.5 d_in the library forms the n x n operator each iteration (first product: n rows) and applies
+    # it in the second; otherwise both products have d_out rows.
+    explicit_route = 2 * p >= 3 * n
     ms_p1, n_p1 = timing["wupdate_product1"]
     ms_p2, n_p2 = timing["wupdate_product2"]
-    flops_launch = 3 * 2.0 * p * n * n                     # three 16-bit MMAs per K step of the 2-plane split
+    ms_1p, n_1p = timing["wupdate_one_plane"]
+    rows_p1 = n if explicit_route else p
+    flops_two_plane = 3 * 2.0 * n * n * (rows_p1 * n_p1 + p * n_p2)   # three 16-bit MMAs per K step of the 2-plane split
+    flops_launch = 3 * 2.0 * p * n * n                               # of a launch with d_out rows
     avg_ms = (ms_p1 + ms_p2) / max(1, n_p1 + n_p2)
-    achieved = flops_launch / (avg_ms * 1e-3) / 1e12
+    achieved = flops_two_plane / max(1e-9, (ms_p1 + ms_p2) * 1e-3) / 1e12
     # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of this kernel from its ncu capture;
     # known for the shape that was captured, null for every other
     traffic = PRODUCT_DRAM_BYTES_PER_LAUNCH.get((n, p))
@@ -601,8 +619,12 @@ def main():
                 "achieved": achieved, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
                 "frac": achieved / peaks["bf16_sustained"], "peak_source": peaks["source"] + ", bf16 sustained (fp16 and bf16 share the dense 16-bit peak)",
                 "traffic": traffic, "launches": n_p1 + n_p2, "avg_launch_ms": avg_ms,
+                "flops_per_full_launch": flops_launch,
                 "product1_launch_ms": ms_p1 / max(1, n_p1), "product2_launch_ms": ms_p2 / max(1, n_p2)}
-    w_update_ms = (ms_p1 + ms_p2 + timing["tridiag_solve"][0] + timing["row_split"][0]) / args.steps
+    w_update_ms = (ms_p1 + ms_p2 + ms_1p + timing["tridiag_solve"][0] + timing["row_split"][0]) / args.steps
+    # one-plane launches: both products of an iteration, so half of them have rows_p1 rows
+    flops_one_plane = 2.0 * n * n * (rows_p1 + p) * (n_1p / 2.0)
+    executed_flops_per_step = (flops_two_plane + flops_one_plane) / args.steps
     breakdown = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
                  for k, v in timing.items()}
 
@@ -625,6 +647,12 @@ def main():
         "row_split": _hbm("row_split", 22.0 * p * n),
         "transpose": _hbm("transpose", 2.0 * x_bytes * chunk_rows * n),
     }
+    if n_1p:
+        tf1 = flops_one_plane / (ms_1p * 1e-3) / 1e12
+        kernel_rooflines["wupdate_one_plane"] = {
+            "kernel": "gemm_tc_kernel<1,STORE> (W-update products of the late iterations: one fp16 plane)",
+            "bound": "tensor", "achieved": tf1, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+            "frac": tf1 / peaks["bf16_sustained"], "launches": n_1p, "avg_launch_ms": ms_1p / n_1p}
     ms_h, n_h = timing["hessian_product"]
     if n_h:
         planes = 1 if spec.x_dtype == "bf16" else 3
@@ -641,14 +669,16 @@ def main():
     line = {
         "metric": METRIC, "value": ms_step / 1e3, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f16x2-split (fp32 accumulate)", "data": "synthetic",
+        "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
         "config": layer_config(spec, world),
         "layers_per_s": world / (ms_step / 1e3),
         "w_update_useful_tflops": 4.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
-        "w_update_executed_tflops": 12.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
+        "w_update_executed_tflops": executed_flops_per_step / (w_update_ms * 1e-3) / 1e12,
+        "one_plane_iterations": int(n_1p / (2 * args.steps)), "w_update_route": "explicit operator" if explicit_route else "two products",
         "err_before_local_search": rep.err_before, "err_after_local_search": rep.err_after,
         "local_search_moves": rep.moves, "pair_swap_after_local_search": pair_swap, "admm_with_grid_refresh": grid_refresh,
         "admm_with_mse_clip_search": mse_clip, "admm_with_fused_epilogue": fused_variant,
+        "admm_operand_planes": planes_variant,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "kernel_rooflines": kernel_rooflines, "cpu_baseline": cpu_baseline,
         "breakdown": breakdown,

@@ -116,7 +116,8 @@ admmq_status admmq_hessian_set(admmq_ctx* ctx, const float* d_H);
 admmq_status admmq_hessian_export(admmq_ctx* ctx, float* d_Hraw_out, long long* h_tokens);
 admmq_status admmq_hessian_import(admmq_ctx* ctx, const float* d_Hraw, long long n_tokens);
 
-/* ---- Step 2: damping, diagonal scaling, factorisation. ---------------------------------------------
+/* ---- Step 2: damping, diagonal scaling, factorisation.  Synchronises (it reads three scalars of the
+ * factorisation back: the mean and two bounds of the spectrum of H~). --------------------------------
  * H = H_raw / N + damp_frac * mean(diag(H_raw / N)) I                         (App. D, damping)
  * s_i = sqrt(H_ii),  H~ = diag(1/s) H diag(1/s)                   (Sec. 3.2; Algorithm 1 lines 1-2)
  * then the one-time factorisation of H~ (Algorithm 1 line 3) and the per-penalty factors for
@@ -167,6 +168,19 @@ typedef struct {
                            split of the next right-hand side (the faster of the two as measured on B200).
                            1: inside the second product's epilogue, W never leaves the SM.  Same arithmetic per
                            element, so both settings give the same codes. */
+  int wupdate_route;    /* how the W-update of Eq. 7 is evaluated.  1: two products per iteration through the basis
+                           of the factorisation, R Q -> row solve -> Q^T (2 p n^2 multiply-adds).  2: the n x n operator
+                           (H~/rho + I)^{-1} is formed each iteration (a row solve of n rows and one n^3 product) and
+                           applied in one product (n^3 + p n^2): fewer operations when d_out > d_in; needs a context
+                           created with d_out_max >= 1.25 d_in, otherwise ADMMQ_ERR_UNSUPPORTED.  0: route 2 when
+                           d_out >= 1.5 d_in and the context allows it, else route 1.  Both evaluate the same
+                           operator; their results differ by rounding only. */
+  int product_planes;   /* operand precision of the W-update products.  The products carry only the part of the
+                           W-update that is not c R (c = rho / (mu + rho), mu the mean of the spectrum of H~), whose
+                           relative size gamma(rho) = max |mu - lambda| / (lambda + rho) over the spectrum shrinks as the
+                           penalty grows.  0: two fp16 planes per operand (about 22 bits) while gamma > 2^-13, one
+                           plane (11 bits, a third of the tensor-core work) afterwards, where the rounding of one
+                           plane is below the fp32 resolution of the W-update.  2: two planes in every iteration. */
 } admmq_quant_cfg;
 typedef struct {
   double err_before;    /* Tr(E^T H E), E = W_q - W_hat, at entry (local search) / of the ADMM result */
@@ -176,6 +190,7 @@ typedef struct {
   int capped_columns;   /* columns that hit max_moves_per_col */
   float ms;             /* device time of the call, CUDA events */
   int refreshed_iter;   /* quantize_layer: iteration of the accepted grid refresh, -1: none */
+  int one_plane_iters;  /* quantize_layer: iterations whose products ran on one fp16 plane per operand */
 } admmq_report;
 admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out,
                                   const admmq_quant_cfg* cfg, unsigned char* d_codes, float* d_scale,
@@ -265,7 +280,8 @@ typedef enum {
   ADMMQ_T_LOCAL_SEARCH = 7,     /* move loop kernel                                       (step 4) */
   ADMMQ_T_ROW_SPLIT = 8,        /* row pass: projection, dual update, residuals (unless fused into product 2) and
                                    next right-hand side -> scaled fp16 operand planes     (step 3) */
-  ADMMQ_T_KINDS = 9
+  ADMMQ_T_WUPDATE_ONE_PLANE = 9, /* either W-update product when it runs on one fp16 plane per operand (step 3) */
+  ADMMQ_T_KINDS = 10
 } admmq_timing_kind;
 admmq_status admmq_set_timing(admmq_ctx* ctx, int on);
 admmq_status admmq_reset_timing(admmq_ctx* ctx);

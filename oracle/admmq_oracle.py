@@ -460,9 +460,10 @@ class LayerResult:
 def quantize_layer(H: np.ndarray, W_hat: np.ndarray, bits: int, group_size: int,
                    symmetric: bool, rho: np.ndarray, do_local_search: bool = True,
                    precond: bool = True, max_moves: int = 0, tau: float = 1e-6,
-                   probe=None) -> LayerResult:
-    """Algorithm 1 on a damped Hessian H: ADMM loop, then local search (line 12)."""
-    a = admm(H, W_hat, bits, group_size, symmetric, rho, precond=precond, probe=probe)
+                   probe=None, grid: Optional[tuple] = None) -> LayerResult:
+    """Algorithm 1 on a damped Hessian H: ADMM loop, then local search (line 12).
+    `grid` = (Delta, z0), each [p, n/gs]: run on this grid instead of fitting one (passed on to `admm`)."""
+    a = admm(H, W_hat, bits, group_size, symmetric, rho, precond=precond, probe=probe, grid=grid)
     e0 = objective(H, W_hat, a.Wq)
     ls = None
     e1 = e0

@@ -31,9 +31,9 @@ EXPORTS = [
     "admmq_hessian_export", "admmq_hessian_import",
 ]
 T_HESSIAN_PRODUCT, T_TRANSPOSE, T_FACTOR, T_WUPDATE_PRODUCT1, T_TRIDIAG_SOLVE, T_WUPDATE_PRODUCT2, \
-    T_GRADIENT_PRODUCT, T_LOCAL_SEARCH, T_ROW_SPLIT = range(9)
+    T_GRADIENT_PRODUCT, T_LOCAL_SEARCH, T_ROW_SPLIT, T_WUPDATE_ONE_PLANE = range(10)
 TIMING_NAMES = ["hessian_product", "transpose", "factor", "wupdate_product1", "tridiag_solve",
-                "wupdate_product2", "gradient_product", "local_search", "row_split"]
+                "wupdate_product2", "gradient_product", "local_search", "row_split", "wupdate_one_plane"]
 
 
 class FactorCfg(C.Structure):
@@ -46,7 +46,8 @@ class QuantCfg(C.Structure):
     _fields_ = [("struct_size", C.c_size_t), ("bits", C.c_int), ("group_size", C.c_int),
                 ("symmetric", C.c_int), ("use_caller_grid", C.c_int), ("n_refresh", C.c_int),
                 ("h_refresh_iters", C.POINTER(C.c_int)), ("clip_points", C.c_int),
-                ("clip_min_ratio", C.c_double), ("fused_epilogue", C.c_int)]
+                ("clip_min_ratio", C.c_double), ("fused_epilogue", C.c_int), ("wupdate_route", C.c_int),
+                ("product_planes", C.c_int)]
 
 
 class LsCfg(C.Structure):
@@ -62,7 +63,7 @@ class PairSwapCfg(C.Structure):
 class Report(C.Structure):
     _fields_ = [("err_before", C.c_double), ("err_after", C.c_double), ("moves", C.c_longlong),
                 ("iters_run", C.c_int), ("capped_columns", C.c_int), ("ms", C.c_float),
-                ("refreshed_iter", C.c_int)]
+                ("refreshed_iter", C.c_int), ("one_plane_iters", C.c_int)]
 
 
 class AdmmqError(RuntimeError):
@@ -226,7 +227,8 @@ class Solver:
     def quantize_layer(self, W0: torch.Tensor, bits: int, group_size: int = 0, symmetric: bool = False,
                        codes=None, scale=None, zero=None, Wq=None, resid=None, use_caller_grid=False,
                        report: bool = True, refresh_at: Sequence[int] = (), clip_points: int = 0,
-                       clip_min_ratio: float = 0.8, fused_epilogue: bool = False):
+                       clip_min_ratio: float = 0.8, fused_epilogue: bool = False, wupdate_route: int = 0,
+                       product_planes: int = 0):
         p, n = W0.shape
         gs = n if group_size in (0, n) else group_size
         dev = W0.device
@@ -236,7 +238,8 @@ class Solver:
         iters = (C.c_int * max(1, len(refresh_at)))(*[int(t) for t in refresh_at])
         cfg = QuantCfg(C.sizeof(QuantCfg), bits, group_size, int(symmetric), int(use_caller_grid),
                        len(refresh_at), C.cast(iters, C.POINTER(C.c_int)) if len(refresh_at) else None,
-                       int(clip_points), float(clip_min_ratio), int(fused_epilogue))
+                       int(clip_points), float(clip_min_ratio), int(fused_epilogue), int(wupdate_route),
+                       int(product_planes))
         rep = Report()
         st = self.lib.admmq_quantize_layer(self.h, _ptr(W0), p, C.byref(cfg), _ptr(codes), _ptr(scale),
                                            _ptr(zero), _ptr(Wq), _ptr(resid),

@@ -60,6 +60,10 @@ struct Carver {
   }
 };
 
+// The explicit-operator route of the W-update needs an n x n fp32 copy of Q (mu I - T) and pays off only for
+// layers with clearly more output than input channels.
+bool explicit_operator_possible(int n, int p_max) { return (long long)4 * p_max >= (long long)5 * n; }
+
 int slots_cap_for(int n, int p) {
   const int simt = ((p + 63) / 64) * ((n + 63) / 64);
   return simt > 256 ? simt : 256;
@@ -92,6 +96,8 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   c.pvec = cv.take<double>(n);
   c.stage_l = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
   c.stage_invd = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
+  c.shift_c = cv.take<float>((size_t)T + 1);
+  c.Qs32 = explicit_operator_possible(n, p) ? cv.take<float>(nn) : nullptr;
   c.ps_totals = cv.take<double>(PAIR_BATCH_MAX);
   c.ps_chosen = cv.take<int>(16);
   c.ps_d = cv.take<float>((size_t)2 * p);
@@ -103,7 +109,6 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   c.QT_lo = cv.take<bf16>(nn);
   c.H_hi = cv.take<bf16>(nn);
   c.H_lo = cv.take<bf16>(nn);
-  c.Whs = cv.take<float>(pn);
   c.V = cv.take<float>(pn);
   c.Y = cv.take<float>(pn);
   c.R_hi = cv.take<bf16>(pn);
@@ -175,7 +180,8 @@ int group_of(int d_in, int gs) { return (gs == 0 || gs == d_in) ? d_in : gs; }
 // Operand descriptors: Q, Q^T and H are stored once per factorisation as fp16 planes with a common
 // power-of-two scale; R, Y' and E carry one scale per row (output channel).
 Planes op_Q(Ctx* c) { return planes_f16(c->Q_hi, c->Q_lo, c->n, nullptr, c->fscal + 0); }
-Planes op_QT(Ctx* c) { return planes_f16(c->QT_hi, c->QT_lo, c->n, nullptr, c->fscal + 0); }
+// operand of the first product: planes of [Q (mu I - T)]^T with their own scale (shifted operator, elem.cu)
+Planes op_QT(Ctx* c) { return planes_f16(c->QT_hi, c->QT_lo, c->n, nullptr, c->fscal + 3); }
 Planes op_H(Ctx* c) { return planes_f16(c->H_hi, c->H_lo, c->n, nullptr, c->fscal + 1); }
 Planes op_R(Ctx* c) { return planes_f16(c->R_hi, c->R_lo, c->n, c->rs_R, nullptr); }
 Planes op_Y(Ctx* c) { return planes_f16(c->Y_hi, c->Y_lo, c->n, c->rs_Y, nullptr); }
@@ -379,12 +385,28 @@ admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg) {
   launch_split_f32(c, c->H, (long long)n * n, c->H_hi, c->H_lo);
   if (tridiag_reduce(c) != cudaSuccess) return ADMMQ_ERR_CUDA;
   if (tridiag_form_qt(c) != cudaSuccess) return ADMMQ_ERR_CUDA;
-  launch_split_f64(c, c->P64, n, c->QT_hi, c->QT_lo, c->Q_hi, c->Q_lo);
+  launch_split_f64(c, c->P64, n, nullptr, nullptr, c->Q_hi, c->Q_lo);   // planes of Q (second product)
+  launch_shifted_qt(c);                                    // planes of [Q (mu I - T)]^T (first product)
   if (cudaMemcpyAsync(ctx->rho_dev, c->rho_host, sizeof(double) * c->T, cudaMemcpyHostToDevice,
                       c->stream) != cudaSuccess)
     return ADMMQ_ERR_CUDA;
   launch_stage_factors(c, ctx->rho_dev, 0, c->T);
   if (cudaGetLastError() != cudaSuccess) return ADMMQ_ERR_CUDA;
+  // Operand precision per iteration.  The products carry only the part of the W-update that is not c R, of
+  // relative size gamma(rho) = max over the spectrum of |mu - lambda| / (lambda + rho).  Rounding the four
+  // operands to one fp16 plane costs about 2^-11.8 of that part; once gamma <= 2^-13 this is below 2^-24 of the
+  // W-update itself, under the rounding of its fp32 storage, and one plane per operand (one MMA per K step
+  // instead of three) loses nothing.  The bounds come back from the device here: this call synchronises.
+  double spec[3] = {1.0, 0.0, 0.0};
+  if (cudaMemcpy(spec, c->scal + 8, sizeof(spec), cudaMemcpyDeviceToHost) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  c->mu_host = spec[0];
+  c->lam_lo = spec[1] > 0.0 ? spec[1] : 0.0;                // H~ is positive semidefinite
+  c->lam_hi = spec[2];
+  for (int t = 0; t < c->T; ++t) {
+    const double r = c->rho_host[t];
+    const double g = fmax(fabs(c->mu_host - c->lam_lo) / (c->lam_lo + r), fabs(c->mu_host - c->lam_hi) / (c->lam_hi + r));
+    c->planes_host[t] = (isfinite(g) && g <= 1.0 / 8192.0) ? 1 : 2;
+  }
   c->state = 2;
   return ADMMQ_OK;
 }
@@ -406,9 +428,47 @@ static admmq_status check_layer_args(admmq_ctx* ctx, const float* d_W0, int d_ou
 
 // One W-update in the error form of Eq. 7:  W - W_hat' = Q (T/rho + I)^{-1} Q^T R,
 // R = D - V/rho - W_hat'.  Product 1 -> solve -> product 2 (whose epilogue is `epi`).
-static cudaError_t w_update_products(admmq_ctx* a, int p, int stage, const EpiParams& epi) {
+// One plane of an operand pair (the hi plane alone: the value rounded to fp16).
+static Planes hi_only(Planes P) {
+  P.lo = nullptr;
+  return P;
+}
+
+static cudaError_t w_update_products(admmq_ctx* a, int p, int stage, const EpiParams& epi, int planes) {
   Ctx* c = &a->c;
   const int n = c->n;
+  const bool one = planes == 1 && epi.kind == EPI_STORE;   // the fused epilogue exists for two planes only
+  EpiParams e1{};
+  e1.kind = EPI_STORE;
+  e1.C = c->Y;
+  e1.ldc = n;
+  cudaError_t err;
+  {
+    Timed t(a, one ? ADMMQ_T_WUPDATE_ONE_PLANE : ADMMQ_T_WUPDATE_PRODUCT1);
+    err = one ? product(c, hi_only(op_R(c)), hi_only(op_QT(c)), p, n, n, e1) : product(c, op_R(c), op_QT(c), p, n, n, e1);
+  }
+  if (err != cudaSuccess) return err;
+  {
+    Timed t(a, ADMMQ_T_TRIDIAG_SOLVE);
+    launch_tridiag_solve(c, c->Y, p, stage, c->Y_hi, c->Y_lo, c->rs_Y);
+  }
+  Timed t(a, one ? ADMMQ_T_WUPDATE_ONE_PLANE : ADMMQ_T_WUPDATE_PRODUCT2);
+  return one ? product(c, hi_only(op_Y(c)), hi_only(op_Q(c)), p, n, n, epi) : product(c, op_Y(c), op_Q(c), p, n, n, epi);
+}
+
+// The same W-update with the operator formed explicitly, for layers with more output than input channels:
+//   M' = [Q (mu I - T)] (T/rho + I)^{-1} Q^T / (mu + rho)       (n x n: one row solve of n rows + one n^3 product)
+//   W - W_hat' - c R = R M'                                      (one p n^2 product)
+// n^3 + p n^2 multiply-adds per iteration instead of 2 p n^2.  M' is symmetric (a function of H~), so its rows
+// serve as the second product's operand; it takes one power-of-two scale for the whole matrix.
+static cudaError_t w_update_explicit(admmq_ctx* a, int p, int stage, const EpiParams& epi, int planes) {
+  Ctx* c = &a->c;
+  const int n = c->n;
+  const bool one = planes == 1 && epi.kind == EPI_STORE;
+  {
+    Timed t(a, ADMMQ_T_TRIDIAG_SOLVE);
+    launch_tridiag_solve(c, c->Qs32, n, stage, c->Y_hi, c->Y_lo, c->rs_Y);
+  }
   EpiParams e1{};
   e1.kind = EPI_STORE;
   e1.C = c->Y;
@@ -416,15 +476,20 @@ static cudaError_t w_update_products(admmq_ctx* a, int p, int stage, const EpiPa
   cudaError_t err;
   {
     Timed t(a, ADMMQ_T_WUPDATE_PRODUCT1);
-    err = product(c, op_R(c), op_QT(c), p, n, n, e1);
+    err = one ? product(c, hi_only(op_Y(c)), hi_only(op_Q(c)), n, n, n, e1) : product(c, op_Y(c), op_Q(c), n, n, n, e1);
   }
   if (err != cudaSuccess) return err;
   {
-    Timed t(a, ADMMQ_T_TRIDIAG_SOLVE);
-    launch_tridiag_solve(c, p, stage);
+    Timed t(a, ADMMQ_T_ROW_SPLIT);
+    launch_global_split(c, c->Y, (long long)n * n, c->fscal + 6, c->Y_hi, c->Y_lo);
   }
-  Timed t(a, ADMMQ_T_WUPDATE_PRODUCT2);
-  return product(c, op_Y(c), op_Q(c), p, n, n, epi);
+  Timed t(a, one ? ADMMQ_T_WUPDATE_ONE_PLANE : ADMMQ_T_WUPDATE_PRODUCT2);
+  const Planes Mp = planes_f16(c->Y_hi, c->Y_lo, n, nullptr, c->fscal + 6);
+  return one ? product(c, hi_only(op_R(c)), hi_only(Mp), p, n, n, epi) : product(c, op_R(c), Mp, p, n, n, epi);
+}
+
+static cudaError_t w_update_any(admmq_ctx* a, int p, int stage, const EpiParams& epi, bool explicit_op, int planes) {
+  return explicit_op ? w_update_explicit(a, p, stage, epi, planes) : w_update_products(a, p, stage, epi, planes);
 }
 
 // Two events for the device time of a call; destroyed on every exit path.
@@ -448,8 +513,13 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   if (cfg->clip_points < 0 || cfg->clip_points > 4096) return ADMMQ_ERR_INVALID_ARG;
   if (cfg->clip_points > 0 && !(cfg->clip_min_ratio > 0.0 && cfg->clip_min_ratio <= 1.0)) return ADMMQ_ERR_INVALID_ARG;
   if (cfg->n_refresh > 0 && group_of(ctx->c.n, cfg->group_size) < 2) return ADMMQ_ERR_UNSUPPORTED;
+  if (cfg->wupdate_route < 0 || cfg->wupdate_route > 2) return ADMMQ_ERR_INVALID_ARG;
+  if (cfg->product_planes != 0 && cfg->product_planes != 2) return ADMMQ_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
+  if (cfg->wupdate_route == 2 && !c->Qs32) return ADMMQ_ERR_UNSUPPORTED;
   const int n = c->n, p = d_out, gs = group_of(n, cfg->group_size), T = c->T;
+  // explicit operator: asked for, or worth it (n^3 + p n^2 against 2 p n^2, plus three small kernels per iteration)
+  const bool explicit_op = cfg->wupdate_route == 2 || (cfg->wupdate_route == 0 && c->Qs32 && 2 * p >= 3 * n);
   CallEvents ev;
   if (h_report) {
     if (!ev.create()) return ADMMQ_ERR_CUDA;
@@ -462,13 +532,12 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     else
       launch_grid_fit(c, d_W0, p, cfg->bits, gs, cfg->symmetric, d_scale, d_zero);
   }
-  launch_scale_weights(c, d_W0, p);                        // W_hat', V = 0, R = 0 (Algorithm 1 l.2, l.4)
+  launch_scale_weights(c, d_W0, p);                        // V = 0, R = 0 (Algorithm 1 l.4)
   launch_zero(c, c->partials, (size_t)T * c->partial_slots * 2 * sizeof(float));
   int* refresh_flags = c->ps_chosen + 4;                   // [0] this attempt accepted, [1] 1 + accepted iteration
   launch_zero(c, c->ps_chosen, 64);
   EpiParams e{};
   e.kind = EPI_ADMM;
-  e.Whs = c->Whs;
   e.W0 = d_W0;
   e.V = c->V;
   e.codes = d_codes;
@@ -480,6 +549,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.n_groups = n / gs;
   e.kmax = (1 << cfg->bits) - 1;
   e.Rnext = c->Y;                                          // Y is free once its planes exist
+  int one_plane_iters = 0;
   for (int t = 0; t < T; ++t) {
     const double rho = c->rho_host[t];
     const double rho_next = (t + 1 < T) ? c->rho_host[t + 1] : rho;
@@ -488,6 +558,9 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     e.inv_rho = (float)(1.0 / rho);
     e.inv_rho_next = (float)(1.0 / rho_next);
     e.partials = c->partials + (size_t)t * c->partial_slots * 2;
+    e.shift_c = c->shift_c + t;
+    const int planes = (cfg->product_planes == 2 || cfg->fused_epilogue) ? 2 : c->planes_host[t];
+    one_plane_iters += planes == 1;
     bool refresh = false;
     for (int q = 0; q < cfg->n_refresh; ++q) refresh = refresh || (cfg->h_refresh_iters[q] == t);
     if (refresh) {
@@ -496,7 +569,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
       w.kind = EPI_STORE;
       w.C = c->Y;
       w.ldc = n;
-      if (w_update_products(ctx, p, t, w) != cudaSuccess) return ADMMQ_ERR_CUDA;
+      if (w_update_any(ctx, p, t, w, explicit_op, planes) != cudaSuccess) return ADMMQ_ERR_CUDA;
       launch_grid_refresh(c, e, p, cfg->bits, cfg->symmetric, t, d_scale, d_zero, refresh_flags);
       if (t + 1 < T) {
         Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
@@ -505,7 +578,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     } else if (cfg->fused_epilogue) {
       // projection, dual update and residuals inside the second product's epilogue; the next right-hand side
       // leaves it in fp32 and a row pass splits it into planes
-      if (w_update_products(ctx, p, t, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
+      if (w_update_any(ctx, p, t, e, explicit_op, planes) != cudaSuccess) return ADMMQ_ERR_CUDA;
       if (t + 1 < T) {
         Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
         launch_row_split(c, c->Y, p, c->R_hi, c->R_lo, c->rs_R);
@@ -516,7 +589,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
       w.kind = EPI_STORE;
       w.C = c->Y;
       w.ldc = n;
-      if (w_update_products(ctx, p, t, w) != cudaSuccess) return ADMMQ_ERR_CUDA;
+      if (w_update_any(ctx, p, t, w, explicit_op, planes) != cudaSuccess) return ADMMQ_ERR_CUDA;
       Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
       w.kind = EPI_ADMM;
       launch_admm_rows(c, w, p, c->R_hi, c->R_lo, c->rs_R);
@@ -540,6 +613,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   h_report->err_after = err;
   h_report->iters_run = T;
   h_report->refreshed_iter = flags[1] - 1;
+  h_report->one_plane_iters = one_plane_iters;
   return st;
 }
 
@@ -562,11 +636,11 @@ admmq_status admmq_w_update(admmq_ctx* ctx, const float* d_W0, int d_out, int gr
     return ADMMQ_ERR_CUDA;
   launch_stage_factors(c, ctx->rho_dev, stage, 1);
   EpiParams e{};
-  e.kind = EPI_WOUT;
-  e.C = d_W_out;
+  e.kind = EPI_STORE;
+  e.C = c->Y;                                               // free once its planes exist
   e.ldc = n;
-  e.Whs = c->Whs;
-  if (w_update_products(ctx, p, stage, e) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  if (w_update_products(ctx, p, stage, e, 2) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  launch_w_out(c, d_W0, p, gs, d_codes, d_scale, d_zero, d_V, (float)(1.0 / rho), c->shift_c + stage, c->Y, d_W_out);
   return cudaGetLastError() == cudaSuccess ? ADMMQ_OK : ADMMQ_ERR_CUDA;
 }
 

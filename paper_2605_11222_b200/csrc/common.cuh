@@ -75,6 +75,20 @@ __device__ __forceinline__ void dmma_8x8x4(double& d0, double& d1, double a, dou
                : "d"(a), "d"(b));
 }
 
+// Maximum of a double over the block, result in every thread.  `scratch` holds >= 32 doubles.
+__device__ __forceinline__ double block_max_f64(double v, double* scratch) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+  __syncthreads();
+  if (lane == 0) scratch[w] = v;
+  __syncthreads();
+  double t = (lane < nw) ? scratch[lane] : -INFINITY;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t = fmax(t, __shfl_xor_sync(0xffffffffu, t, o));
+  return t;
+}
+
 // Sum over the block, result in every thread.  `scratch` holds >= 32 elements.
 template <typename T>
 __device__ __forceinline__ T block_sum(T v, T* scratch) {

@@ -313,17 +313,15 @@ void launch_grid_fit_mse(Ctx* c, const float* W0, int p, int bits, int gs, int s
   LAUNCH(c);
 }
 
-// W_hat' = Sigma^{-1} W_hat (Algorithm 1 line 2); V^(0) = 0; first right-hand side R = D^(0) - W_hat' = 0
-// (all-zero planes, row scale 1).
-__global__ void scale_weights_kernel(const float* __restrict__ W0, const float* __restrict__ s,
-                                     long long total, int n, float* __restrict__ Whs,
-                                     float* __restrict__ V, bf16* __restrict__ Rhi,
-                                     bf16* __restrict__ Rlo, float* __restrict__ row_inv, int* status) {
+// Start of a layer: V^(0) = 0 and the first right-hand side R = D^(0) - W_hat' = 0 (all-zero planes, row scale 1;
+// Algorithm 1 line 4).  W_hat' = Sigma^{-1} W_hat (line 2) is never stored: every later step works with
+// differences from it.  Also the place where non-finite weights are caught.
+__global__ void init_state_kernel(const float* __restrict__ W0, long long total, int n, float* __restrict__ V,
+                                  bf16* __restrict__ Rhi, bf16* __restrict__ Rlo, float* __restrict__ row_inv,
+                                  int* status) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
-  const float w = W0[i];
-  if (!isfinite(w)) raise_status(status, ST_NONFINITE);
-  Whs[i] = s[i % n] * w;
+  if (!isfinite(W0[i])) raise_status(status, ST_NONFINITE);
   V[i] = 0.f;
   Rhi[i] = __float2bfloat16_rn(0.f);                      // the all-zero pattern is zero in fp16 as well
   Rlo[i] = __float2bfloat16_rn(0.f);
@@ -332,8 +330,8 @@ __global__ void scale_weights_kernel(const float* __restrict__ W0, const float* 
 
 void launch_scale_weights(Ctx* c, const float* W0, int p) {
   const long long total = (long long)p * c->n;
-  scale_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
-      W0, c->s, total, c->n, c->Whs, c->V, c->R_hi, c->R_lo, c->rs_R, c->status);
+  init_state_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(W0, total, c->n, c->V, c->R_hi, c->R_lo,
+                                                                          c->rs_R, c->status);
   LAUNCH(c);
 }
 
@@ -379,7 +377,7 @@ __global__ void split_f64_kernel(const double* __restrict__ src, int n, bf16* __
     float v = 0.f;
     if (r < n && cc < n) {
       v = (float)(src[(long long)r * n + cc] * (double)Q_PLANE_SCALE);
-      store_f16_pair(hi, lo, (long long)r * n + cc, v);
+      if (hi) store_f16_pair(hi, lo, (long long)r * n + cc, v);            // planes of src itself: optional
     }
     tile[i][threadIdx.x] = v;
   }
@@ -396,6 +394,148 @@ void launch_split_f64(Ctx* c, const double* src, int n, bf16* hi, bf16* lo, bf16
   LAUNCH(c);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Shifted form of the W-update operator.  With mu = trace(T) / n (= 1 when H~ has unit diagonal) and
+// c = rho / (mu + rho),
+//     (T/rho + I)^{-1} = c I + (T/rho + I)^{-1} (mu I - T) / (mu + rho),
+// so that  Q (T/rho + I)^{-1} Q^T R = c R + Q (T/rho + I)^{-1} [Q (mu I - T)]^T R / (mu + rho).
+// The first term is exact and stays in each element's own column; only the second goes through the products,
+// whose rounding errors are relative to the whole row of R (a few input channels with a large diagonal scale
+// s_i dominate it) -- and that term is small: of relative size |mu - lambda| / (lambda + rho) for an eigenvalue
+// lambda of H~, and O(1/rho) for the large penalties of the late iterations.  The operand of the first product
+// is therefore row m of  Qs^T = mu P[m] - td[m] P[m] - te[m-1] P[m-1] - te[m] P[m+1]  (P = Q^T), formed in fp64
+// and split into fp16 planes with a power-of-two scale of its own; 1 / (mu + rho) is folded into the inverse
+// pivots of the per-penalty factor, and the element update adds c R.
+// ------------------------------------------------------------------------------------------------
+__global__ void shift_mean_kernel(const double* __restrict__ td, int n, double* __restrict__ mu_out,
+                                  float* __restrict__ fscal) {
+  __shared__ double scratch[32];
+  double acc = 0.0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) acc += td[i];
+  acc = block_sum(acc, scratch);
+  if (threadIdx.x == 0) {
+    mu_out[0] = acc / (double)n;
+    reinterpret_cast<unsigned int*>(fscal)[5] = 0u;        // running maximum of |Qs^T|, as float bits
+  }
+}
+
+// Gershgorin bounds of the spectrum of T (= that of H~): out[0] <= lambda <= out[1].
+__global__ void spectrum_bounds_kernel(const double* __restrict__ td, const double* __restrict__ te, int n,
+                                       double* __restrict__ out) {
+  __shared__ double scratch[32];
+  double lo = INFINITY, hi = -INFINITY;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const double r = fabs(te[i]) + (i > 0 ? fabs(te[i - 1]) : 0.0);
+    lo = fmin(lo, td[i] - r);
+    hi = fmax(hi, td[i] + r);
+  }
+  lo = -block_max_f64(-lo, scratch);
+  hi = block_max_f64(hi, scratch);
+  if (threadIdx.x == 0) {
+    out[0] = lo;
+    out[1] = hi;
+  }
+}
+
+__device__ __forceinline__ double shifted_qt_elem(const double* __restrict__ P, const double* __restrict__ td,
+                                                  const double* __restrict__ te, double mu, int n, int m, int k) {
+  double v = (mu - td[m]) * P[(size_t)m * n + k];
+  if (m > 0) v -= te[m - 1] * P[(size_t)(m - 1) * n + k];
+  if (m + 1 < n) v -= te[m] * P[(size_t)(m + 1) * n + k];
+  return v;
+}
+
+__global__ void shifted_qt_max_kernel(const double* __restrict__ P, const double* __restrict__ td,
+                                      const double* __restrict__ te, const double* __restrict__ mu_p, int n,
+                                      float* __restrict__ fscal) {
+  __shared__ float scratch[32];
+  const double mu = mu_p[0];
+  const int m = blockIdx.x;
+  float mx = 0.0f;
+  for (int k = threadIdx.x; k < n; k += blockDim.x)
+    mx = fmaxf(mx, fabsf((float)shifted_qt_elem(P, td, te, mu, n, m, k)));
+  mx = block_max(mx, scratch);
+  if (threadIdx.x == 0) atomicMax(reinterpret_cast<unsigned int*>(fscal) + 5, __float_as_uint(mx));
+}
+
+__global__ void shifted_qt_scale_kernel(float* __restrict__ fscal) {
+  float inv;
+  const float sc = pow2_scale_for(fscal[5], &inv);
+  fscal[3] = inv;
+  fscal[4] = sc;
+}
+
+__global__ void shifted_qt_split_kernel(const double* __restrict__ P, const double* __restrict__ td,
+                                        const double* __restrict__ te, const double* __restrict__ mu_p, int n,
+                                        const float* __restrict__ fscal, bf16* __restrict__ hi,
+                                        bf16* __restrict__ lo) {
+  const double mu = mu_p[0];
+  const double sc = (double)fscal[4];
+  const int m = blockIdx.x;
+  for (int k = threadIdx.x; k < n; k += blockDim.x)
+    store_f16_pair(hi, lo, (long long)m * n + k, (float)(shifted_qt_elem(P, td, te, mu, n, m, k) * sc));
+}
+
+// Q (mu I - T) itself, [k][m] in fp32 (the transpose of what shifted_qt_split_kernel splits): the input of the
+// row solve that builds the explicit operator.
+__global__ void shifted_q32_kernel(const double* __restrict__ P, const double* __restrict__ td,
+                                   const double* __restrict__ te, const double* __restrict__ mu_p, int n,
+                                   float* __restrict__ out) {
+  __shared__ float tile[32][33];
+  const double mu = mu_p[0];
+  const int m0 = blockIdx.y * 32, k0 = blockIdx.x * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int m = m0 + i, k = k0 + threadIdx.x;
+    tile[i][threadIdx.x] = (m < n && k < n) ? (float)shifted_qt_elem(P, td, te, mu, n, m, k) : 0.0f;
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int k = k0 + i, m = m0 + threadIdx.x;
+    if (k < n && m < n) out[(size_t)k * n + m] = tile[threadIdx.x][i];
+  }
+}
+
+void launch_shifted_qt(Ctx* c) {
+  const int n = c->n;
+  shift_mean_kernel<<<1, 1024, 0, c->stream>>>(c->td, n, c->scal + 8, c->fscal);
+  spectrum_bounds_kernel<<<1, 1024, 0, c->stream>>>(c->td, c->te, n, c->scal + 9);
+  shifted_qt_max_kernel<<<n, 256, 0, c->stream>>>(c->P64, c->td, c->te, c->scal + 8, n, c->fscal);
+  shifted_qt_scale_kernel<<<1, 1, 0, c->stream>>>(c->fscal);
+  shifted_qt_split_kernel<<<n, 256, 0, c->stream>>>(c->P64, c->td, c->te, c->scal + 8, n, c->fscal, c->QT_hi,
+                                                    c->QT_lo);
+  c->launches += 5;
+  if (c->Qs32) {
+    dim3 grid((n + 31) / 32, (n + 31) / 32), block(32, 8);
+    shifted_q32_kernel<<<grid, block, 0, c->stream>>>(c->P64, c->td, c->te, c->scal + 8, n, c->Qs32);
+    LAUNCH(c);
+  }
+}
+
+// W^(t+1) = W_hat' + c R + z for the one-step entry point: R = D - V/rho - W_hat' is rebuilt from the caller's
+// state as init_rhs_kernel built it, z is the product's output.
+__global__ void w_out_kernel(long long total, int n, int gs, int ng, const unsigned char* __restrict__ codes,
+                             const float* __restrict__ delta, const float* __restrict__ zero,
+                             const float* __restrict__ V, float inv_rho, const float* __restrict__ s,
+                             const float* __restrict__ W0, const float* __restrict__ shift_c, const float* __restrict__ z,
+                             float* __restrict__ W_out) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= total) return;
+  const int col = (int)(idx % n);
+  const long long gi = (idx / n) * ng + col / gs;
+  const double e = (double)s[col] * fma((double)delta[gi], (double)codes[idx], (double)zero[gi] - (double)W0[idx]);
+  const float r = fmaf(-V[idx], inv_rho, (float)e);
+  W_out[idx] = fmaf(s[col], W0[idx], fmaf(shift_c[0], r, z[idx]));
+}
+
+void launch_w_out(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes, const float* delta,
+                  const float* zero, const float* V_in, float inv_rho, const float* shift_c, const float* z,
+                  float* W_out) {
+  const long long total = (long long)p * c->n;
+  w_out_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
+      total, c->n, gs, c->n / gs, codes, delta, zero, V_in, inv_rho, c->s, W0, shift_c, z, W_out);
+  LAUNCH(c);
+}
+
 __global__ void split_f32_kernel(const float* __restrict__ src, long long count,
                                  const float* __restrict__ fscal, bf16* __restrict__ hi,
                                  bf16* __restrict__ lo) {
@@ -407,6 +547,51 @@ __global__ void split_f32_kernel(const float* __restrict__ src, long long count,
 void launch_split_f32(Ctx* c, const float* src, long long count, bf16* hi, bf16* lo) {
   split_f32_kernel<<<(unsigned)((count + 255) / 256), 256, 0, c->stream>>>(src, count, c->fscal, hi, lo);
   LAUNCH(c);
+}
+
+// A whole fp32 matrix -> fp16 planes with ONE power-of-two scale (from its largest magnitude): the form an
+// operand needs when its rows are the output columns of a product.  slot: three floats, [0] receives 1 / scale,
+// [1] the scale, [2] is the running maximum (float bits).
+__global__ void absmax_kernel(const float* __restrict__ src, long long count, float* __restrict__ slot) {
+  __shared__ float scratch[32];
+  float m = 0.0f;
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < count;
+       i += (long long)gridDim.x * blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(src + i);       // count is a multiple of 4
+    m = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(m, fmaxf(fabsf(v.z), fabsf(v.w))));
+  }
+  m = block_max(m, scratch);
+  if (threadIdx.x == 0 && isfinite(m)) atomicMax(reinterpret_cast<unsigned int*>(slot) + 2, __float_as_uint(m));
+}
+__global__ void scale_from_max_kernel(float* __restrict__ slot) {
+  float inv;
+  const float sc = pow2_scale_for(slot[2], &inv);
+  slot[0] = inv;
+  slot[1] = sc;
+}
+__global__ void split_scaled_kernel(const float* __restrict__ src, long long count, const float* __restrict__ slot,
+                                    bf16* __restrict__ hi, bf16* __restrict__ lo) {
+  const float sc = slot[1];
+  for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 8; i < count;
+       i += (long long)gridDim.x * blockDim.x * 8) {
+    const float4 a = *reinterpret_cast<const float4*>(src + i), b = *reinterpret_cast<const float4*>(src + i + 4);
+    const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    __align__(16) __half hh[8];
+    __align__(16) __half ll[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) split_f16(v[e] * sc, hh[e], ll[e]);
+    *reinterpret_cast<uint4*>(hi + i) = *reinterpret_cast<const uint4*>(hh);
+    *reinterpret_cast<uint4*>(lo + i) = *reinterpret_cast<const uint4*>(ll);
+  }
+}
+
+void launch_global_split(Ctx* c, const float* src, long long count, float* slot, bf16* hi, bf16* lo) {
+  cudaMemsetAsync(slot + 2, 0, sizeof(float), c->stream);
+  const int blocks = c->num_sms * 8;
+  absmax_kernel<<<blocks, 256, 0, c->stream>>>(src, count, slot);
+  scale_from_max_kernel<<<1, 1, 0, c->stream>>>(slot);
+  split_scaled_kernel<<<blocks, 256, 0, c->stream>>>(src, count, slot, hi, lo);
+  c->launches += 3;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -576,22 +761,36 @@ void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned 
 //           that was kept.  Same arithmetic as the row pass: targets and grid points relative to the weight,
 //           weight-sized differences and the rounding decisions in fp64.
 // ------------------------------------------------------------------------------------------------
+// (W~ - W_hat') / s of one element: the product's output plus its c R part (R rebuilt from the codes and the dual
+// as in the element update), plus V/rho.
+__device__ __forceinline__ float refresh_target(float zp, float w0, float v, int code_old, int first_iter, float s,
+                                                float inv_s, float dl, float z0, float cshift, float inv_rho) {
+  const float e_old = first_iter ? 0.0f
+                                 : (float)((double)s * fma((double)dl, (double)code_old, (double)z0 - (double)w0));
+  const float z = fmaf(cshift, fmaf(-v, inv_rho, e_old), zp);
+  return fmaf(v, inv_rho, z) * inv_s;
+}
+
 __global__ void __launch_bounds__(256)
 refresh_eval_kernel(const float* __restrict__ Zc, const float* __restrict__ W0, const float* __restrict__ V,
+                    const unsigned char* __restrict__ codes, int first_iter, const float* __restrict__ shift_c,
                     const float* __restrict__ s, const float* __restrict__ inv_s, int p, int n, int gs, int kmax,
                     int symmetric, float inv_rho, const float* __restrict__ delta, const float* __restrict__ zero,
                     float* __restrict__ cand_delta, float* __restrict__ cand_zero, double* __restrict__ partial) {
   __shared__ double scratch[32];
   const int ng = n / gs, lane = threadIdx.x & 31;
   const long long groups = (long long)p * ng;
+  const float cs = shift_c[0];
   double e_old = 0.0, e_new = 0.0;
   for (long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; gw < groups;
        gw += ((long long)gridDim.x * blockDim.x) >> 5) {
     const int j = (int)(gw / ng), gq = (int)(gw % ng);
     const size_t base = (size_t)j * n + (size_t)gq * gs;
+    const float d0 = delta[gw], z0 = zero[gw];
     double lo = INFINITY, hi = -INFINITY;
     for (int i = lane; i < gs; i += 32) {
-      const float u = fmaf(V[base + i], inv_rho, Zc[base + i]) * inv_s[gq * gs + i];
+      const float u = refresh_target(Zc[base + i], W0[base + i], V[base + i], first_iter ? 0 : (int)codes[base + i],
+                                     first_iter, s[gq * gs + i], inv_s[gq * gs + i], d0, z0, cs, inv_rho);
       const double y = (double)W0[base + i] + (double)u;
       lo = fmin(lo, y);
       hi = fmax(hi, y);
@@ -612,12 +811,13 @@ refresh_eval_kernel(const float* __restrict__ Zc, const float* __restrict__ W0, 
       cand_delta[gw] = dn;
       cand_zero[gw] = zn;
     }
-    const float d0 = delta[gw], z0 = zero[gw];
     const double id0 = 1.0 / (double)d0, idn = 1.0 / (double)dn;
     double a = 0.0, b = 0.0;
     for (int i = lane; i < gs; i += 32) {
       const double sv = (double)s[gq * gs + i];
-      const double u = (double)(fmaf(V[base + i], inv_rho, Zc[base + i]) * inv_s[gq * gs + i]);
+      const double u = (double)refresh_target(Zc[base + i], W0[base + i], V[base + i],
+                                              first_iter ? 0 : (int)codes[base + i], first_iter, s[gq * gs + i],
+                                              inv_s[gq * gs + i], d0, z0, cs, inv_rho);
       const double w = (double)W0[base + i];
       const double k0 = fmin(fmax(rint(((w - (double)z0) + u) * id0), 0.0), (double)kmax);
       const double kn = fmin(fmax(rint(((w - (double)zn) + u) * idn), 0.0), (double)kmax);
@@ -655,27 +855,37 @@ __global__ void refresh_decide_kernel(const double* __restrict__ partial, int bl
   }
 }
 
+// After this kernel (delta, zero) is the grid in force and (cand_delta, cand_zero) the grid the codes of D^(t)
+// refer to: the two are exchanged when the attempt is accepted, and equal otherwise.
 __global__ void refresh_commit_kernel(long long groups, const int* __restrict__ flags,
-                                      const float* __restrict__ cand_delta, const float* __restrict__ cand_zero,
+                                      float* __restrict__ cand_delta, float* __restrict__ cand_zero,
                                       float* __restrict__ delta, float* __restrict__ zero) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= groups || !flags[0]) return;
-  delta[i] = cand_delta[i];
-  zero[i] = cand_zero[i];
+  if (i >= groups) return;
+  const float d_old = delta[i], z_old = zero[i];
+  if (flags[0]) {
+    delta[i] = cand_delta[i];
+    zero[i] = cand_zero[i];
+  }
+  cand_delta[i] = d_old;
+  cand_zero[i] = z_old;
 }
 
 // The ADMM element update from the stored product z = W^(t+1) - W_hat' (in P.Rnext, overwritten by the next
 // right-hand side).
-__global__ void __launch_bounds__(256) admm_elementwise_kernel(EpiParams P, long long total, int n) {
+__global__ void __launch_bounds__(256) admm_elementwise_kernel(EpiParams P, const float* __restrict__ old_delta,
+                                                               const float* __restrict__ old_zero, long long total,
+                                                               int n) {
   __shared__ float red[32];
   float r2 = 0.f, s2 = 0.f;
+  const float cs = P.shift_c[0];
   for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
     const int col = (int)(idx % n);
     const long long row = idx / n;
     const long long gi = row * P.n_groups + col / P.group_size;
     AdmmElem e = admm_elem(P.Rnext[idx], P.W0[idx], P.V[idx], P.first_iter ? 0 : (int)P.codes[idx], P.s[col],
-                           P.inv_s[col], grid_g(P.delta[gi], P.zero[gi]), P);
+                           P.inv_s[col], grid_g(P.delta[gi], P.zero[gi]), grid_g(old_delta[gi], old_zero[gi]), cs, P);
     P.codes[idx] = e.code;
     P.V[idx] = e.v_new;
     P.Rnext[idx] = e.r_next;
@@ -701,6 +911,7 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
   float r2 = 0.f, s2 = 0.f;
   const int gs = P.group_size;
   const int gsh = (gs & (gs - 1)) == 0 ? 31 - __clz(gs) : -1;      // group index by shift when the size allows
+  const float cs = P.shift_c[0];
   for (int j = blockIdx.x; j < p; j += gridDim.x) {
     const size_t base = (size_t)j * n;
     const float* dlt = P.delta + (size_t)j * P.n_groups;
@@ -717,17 +928,18 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
       const int g0 = gsh >= 0 ? i >> gsh : i / gs;
       const int g3 = gsh >= 0 ? (i + 3) >> gsh : (i + 3) / gs;
       const GridG gg = grid_g(dlt[g0], zr[g0]);
-      AdmmElem e0 = admm_elem(z.x, wh.x, v.x, k.x, sv.x, si.x, gg, P);
+      AdmmElem e0 = admm_elem(z.x, wh.x, v.x, k.x, sv.x, si.x, gg, gg, cs, P);
       AdmmElem e1, e2, e3;
       if (g3 == g0) {
-        e1 = admm_elem(z.y, wh.y, v.y, k.y, sv.y, si.y, gg, P);
-        e2 = admm_elem(z.z, wh.z, v.z, k.z, sv.z, si.z, gg, P);
-        e3 = admm_elem(z.w, wh.w, v.w, k.w, sv.w, si.w, gg, P);
+        e1 = admm_elem(z.y, wh.y, v.y, k.y, sv.y, si.y, gg, gg, cs, P);
+        e2 = admm_elem(z.z, wh.z, v.z, k.z, sv.z, si.z, gg, gg, cs, P);
+        e3 = admm_elem(z.w, wh.w, v.w, k.w, sv.w, si.w, gg, gg, cs, P);
       } else {
         const int g1 = (i + 1) / gs, g2 = (i + 2) / gs;
-        e1 = admm_elem(z.y, wh.y, v.y, k.y, sv.y, si.y, grid_g(dlt[g1], zr[g1]), P);
-        e2 = admm_elem(z.z, wh.z, v.z, k.z, sv.z, si.z, grid_g(dlt[g2], zr[g2]), P);
-        e3 = admm_elem(z.w, wh.w, v.w, k.w, sv.w, si.w, grid_g(dlt[g3], zr[g3]), P);
+        const GridG q1 = grid_g(dlt[g1], zr[g1]), q2 = grid_g(dlt[g2], zr[g2]), q3 = grid_g(dlt[g3], zr[g3]);
+        e1 = admm_elem(z.y, wh.y, v.y, k.y, sv.y, si.y, q1, q1, cs, P);
+        e2 = admm_elem(z.z, wh.z, v.z, k.z, sv.z, si.z, q2, q2, cs, P);
+        e3 = admm_elem(z.w, wh.w, v.w, k.w, sv.w, si.w, q3, q3, cs, P);
       }
       *reinterpret_cast<uchar4*>(P.codes + base + i) = make_uchar4(e0.code, e1.code, e2.code, e3.code);
       *reinterpret_cast<float4*>(P.V + base + i) = make_float4(e0.v_new, e1.v_new, e2.v_new, e3.v_new);
@@ -775,7 +987,8 @@ void launch_grid_refresh(Ctx* c, const EpiParams& P, int p, int bits, int symmet
   float* cand_zero = reinterpret_cast<float*>(c->R_lo);       // and the row pass that rewrites them
   long long want = (groups * 32 + 255) / 256;
   const int blocks = (int)(want < 1184 ? want : 1184);
-  refresh_eval_kernel<<<blocks, 256, 0, c->stream>>>(P.Rnext, P.W0, P.V, P.s, P.inv_s, p, n, gs, (1 << bits) - 1,
+  refresh_eval_kernel<<<blocks, 256, 0, c->stream>>>(P.Rnext, P.W0, P.V, P.codes, P.first_iter, P.shift_c, P.s,
+                                                     P.inv_s, p, n, gs, (1 << bits) - 1,
                                                      symmetric, P.inv_rho, delta, zero, cand_delta, cand_zero,
                                                      c->ps_totals);
   refresh_decide_kernel<<<1, 256, 0, c->stream>>>(c->ps_totals, blocks, iter, flags);
@@ -784,7 +997,7 @@ void launch_grid_refresh(Ctx* c, const EpiParams& P, int p, int bits, int symmet
   const long long total = (long long)p * n;
   int eb = c->partial_slots < 1184 ? c->partial_slots : 1184;
   if ((long long)eb * 256 > total) eb = (int)((total + 255) / 256);
-  admm_elementwise_kernel<<<eb, 256, 0, c->stream>>>(P, total, n);
+  admm_elementwise_kernel<<<eb, 256, 0, c->stream>>>(P, cand_delta, cand_zero, total, n);
   c->launches += 4;
 }
 

@@ -9,17 +9,15 @@ namespace admmq {
 enum EpiKind : int {
   EPI_STORE = 0,   // C = acc
   EPI_ACCUM = 1,   // C += acc                     (Hessian accumulation)
-  EPI_ADMM = 2,    // projection + dual update + residuals + next right-hand side (Eq. 8-10)
-  EPI_WOUT = 3     // C = W_hat' + acc             (W-update of Eq. 7 alone)
+  EPI_ADMM = 2     // projection + dual update + residuals + next right-hand side (Eq. 8-10)
 };
 
 struct EpiParams {
   int kind;
-  float* C;                 // STORE / ACCUM / WOUT: output [M][ldc]
+  float* C;                 // STORE / ACCUM: output [M][ldc]
   long long ldc;
   int lower_only;           // ACCUM: skip elements with col > row (symmetric product)
   // ---- ADMM state, all [p][n] row-major with leading dimension n ----
-  const float* Whs;         // W_hat' = s_i * W_hat  (scaled pre-trained weights; WOUT only)
   const float* W0;          // W_hat, unscaled, as the caller passed it (ADMM element update)
   float* V;                 // dual V (in/out)
   unsigned char* codes;     // codes of D (in: D^(t), out: D^(t+1))
@@ -31,6 +29,8 @@ struct EpiParams {
   int kmax;                 // 2^bits - 1
   int first_iter;           // 1: D^(0) = W_hat' (Algorithm 1 line 4), codes not yet defined
   float rho, inv_rho, inv_rho_next;
+  const float* shift_c;     // device scalar c = rho / (mu + rho) of this iteration: the product's output is the
+                            // W-update correction WITHOUT its c R part, which the element update adds
   float* Rnext;             // next right-hand side D - V/rho_next - W_hat' (fp32; split into planes by a row pass)
   float* partials;          // [slots][2]: per-CTA sums of (W-D)^2 and (D-D_old)^2
   // ---- undoing the operands' power-of-two scales: value = acc * row_inv[row] * a_inv[0] * b_inv[0] ----
@@ -77,16 +77,21 @@ __device__ __forceinline__ GridG grid_g(float dl, float z0) {
   g.inv_dl = 1.0 / (double)dl;
   return g;
 }
-__device__ __forceinline__ AdmmElem admm_elem(float z, float w0, float v, int code_old, float s, float inv_s,
-                                              const GridG& g, const EpiParams& P) {
+// g: the grid the new code is taken on; g_old: the grid code_old refers to (the same one, except in the
+// iteration that accepts a grid refresh).
+__device__ __forceinline__ AdmmElem admm_elem(float zp, float w0, float v, int code_old, float s, float inv_s,
+                                              const GridG& g, const GridG& g_old, float cshift, const EpiParams& P) {
   AdmmElem o;
   const double a = (double)w0 - (double)g.z0;              // w_hat - z0, exact
+  const float e_old = P.first_iter ? 0.0f                                   // D^(0) = W_hat'
+                                   : (float)((double)s * fma((double)g_old.dl, (double)code_old,
+                                                             (double)g_old.z0 - (double)w0));
+  // z = c R + (product output), R = D^(t) - V/rho - W_hat' exactly as the right-hand side was formed
+  const float z = fmaf(cshift, fmaf(-v, P.inv_rho, e_old), zp);
   const float u = fmaf(v, P.inv_rho, z) * inv_s;           // (W~ - W_hat') / s: target minus weight  (Eq. 8)
   double k = rint((a + (double)u) * g.inv_dl);             // nearest level, ties to even    (Eq. 10)
   k = fmin(fmax(k, 0.0), (double)P.kmax);
   const float e_new = (float)((double)s * fma((double)g.dl, k, -a));        // D^(t+1) - W_hat'
-  const float e_old = P.first_iter ? 0.0f                                   // D^(0) = W_hat'
-                                   : (float)((double)s * fma((double)g.dl, (double)code_old, -a));
   const float wd = z - e_new;                              // W^(t+1) - D^(t+1)
   const float dd = e_new - e_old;                          // D^(t+1) - D^(t)
   o.code = (unsigned char)(int)k;
@@ -105,15 +110,14 @@ __device__ __forceinline__ void epi_scalar(const EpiParams& P, int row, int col,
     P.C[(long long)row * P.ldc + col] = acc;
   } else if (P.kind == EPI_ACCUM) {
     if (!P.lower_only || col <= row) P.C[(long long)row * P.ldc + col] += acc;
-  } else if (P.kind == EPI_WOUT) {
-    P.C[(long long)row * P.ldc + col] = P.Whs[(long long)row * n_cols + col] + acc;
   } else {
     const long long idx = (long long)row * n_cols + col;
     const int g = col / P.group_size;
     const float dl = P.delta[(long long)row * P.n_groups + g];
     const float z0 = P.zero[(long long)row * P.n_groups + g];
+    const GridG gg = grid_g(dl, z0);
     AdmmElem e = admm_elem(acc, P.W0[idx], P.V[idx], P.first_iter ? 0 : (int)P.codes[idx], P.s[col],
-                           P.inv_s[col], grid_g(dl, z0), P);
+                           P.inv_s[col], gg, gg, P.shift_c[0], P);
     P.codes[idx] = e.code;
     P.V[idx] = e.v_new;
     P.Rnext[idx] = e.r_next;

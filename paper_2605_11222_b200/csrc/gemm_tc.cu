@@ -245,6 +245,7 @@ __device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, 
     const float ss[4] = {s.x, s.y, s.z, s.w};
     const float si[4] = {is.x, is.y, is.z, is.w};
     const bool one_group = (P.group_size & 3) == 0;        // then the 4 columns share (Delta, z0)
+    const float cshift = P.shift_c[0];
     long long gi = (long long)row * P.n_groups + col / P.group_size;
     GridG gg = grid_g(P.delta[gi], P.zero[gi]);
     float vn[4], rn[4];
@@ -256,7 +257,7 @@ __device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, 
         gg = grid_g(P.delta[gi], P.zero[gi]);
       }
       const int code_old = (int)((codes >> (8 * e)) & 0xffu);
-      AdmmElem r = admm_elem(a[e], wh[e], vv[e], code_old, ss[e], si[e], gg, P);
+      AdmmElem r = admm_elem(a[e], wh[e], vv[e], code_old, ss[e], si[e], gg, gg, cshift, P);
       vn[e] = r.v_new;
       cn |= (uint32_t)r.code << (8 * e);
       rn[e] = r.r_next;
@@ -270,10 +271,6 @@ __device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, 
   }
   float* cp = P.C + (long long)row * P.ldc + col;
   float o[4] = {a[0], a[1], a[2], a[3]};
-  if (EPI == EPI_WOUT) {
-    const float4 c = *reinterpret_cast<const float4*>(P.Whs + (long long)row * N + col);
-    o[0] += c.x; o[1] += c.y; o[2] += c.z; o[3] += c.w;
-  }
   if (EPI == EPI_ACCUM) {
     if (P.lower_only && col + 3 > row) {                   // the tile straddles the diagonal
 #pragma unroll
@@ -300,10 +297,6 @@ __device__ __forceinline__ void epilogue_prefetch(const EpiParams& P, int row, i
     if (!P.first_iter) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.codes + o));
   } else if (EPI == EPI_ACCUM) {
     const float* c = P.C + (long long)row * P.ldc + col0;
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(c));
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(c + 32));
-  } else if (EPI == EPI_WOUT) {
-    const float* c = P.Whs + (long long)row * N + col0;
     asm volatile("prefetch.global.L2 [%0];" ::"l"(c));
     asm volatile("prefetch.global.L2 [%0];" ::"l"(c + 32));
   }
@@ -684,7 +677,6 @@ cudaError_t gemm_tc(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiPa
     case EPI_STORE: return launch_tc<2, EPI_STORE>(c, maps, M, N, K, idesc, epi);
     case EPI_ACCUM: return launch_tc<2, EPI_ACCUM>(c, maps, M, N, K, idesc, epi);
     case EPI_ADMM: return launch_tc<2, EPI_ADMM>(c, maps, M, N, K, idesc, epi);
-    case EPI_WOUT: return launch_tc<2, EPI_WOUT>(c, maps, M, N, K, idesc, epi);
   }
   return cudaErrorInvalidValue;
 }

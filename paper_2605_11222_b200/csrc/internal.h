@@ -36,6 +36,8 @@ struct Ctx {
   int T = 0;
   int precondition = 1;
   double rho_host[4096];
+  unsigned char planes_host[4096];  // per iteration: operand planes the W-update products need (1 or 2)
+  double mu_host = 1.0, lam_lo = 0.0, lam_hi = 0.0;   // mean and Gershgorin bounds of the spectrum of H~ (host copies)
   long long launches = 0;
   long long wait_limit_cycles = 2000000000LL;   // bound of every device-side wait, about a second
   int hold_loads = 0;           // failure-handling tests only: the product kernel's producer issues no loads
@@ -55,7 +57,9 @@ struct Ctx {
   double* beta = nullptr;       // [n] reflector scalars
   double* pvec = nullptr;       // [n] matrix-vector scratch of the reduction
   float* stage_l = nullptr;     // [T_max+1][stage_factor_stride(n)] LDL^T multipliers per penalty
-  float* stage_invd = nullptr;  // [T_max+1][stage_factor_stride(n)] LDL^T inverse pivots per penalty
+  float* stage_invd = nullptr;  // [T_max+1][stage_factor_stride(n)] LDL^T inverse pivots per penalty, times 1 / (mu + rho)
+  float* shift_c = nullptr;     // [T_max+1] c = rho / (mu + rho) per penalty (shifted W-update operator)
+  float* Qs32 = nullptr;        // [n][n] fp32 Q (mu I - T), or nullptr: input of the explicit-operator route (p_max > n only)
   double* ps_totals = nullptr;  // [PAIR_BATCH_MAX] totals of the candidate pairs of a pair-swap round
   int* ps_chosen = nullptr;     // [1] index of the applied pair, -1: none
   float* ps_d = nullptr;        // [2][p] applied perturbations of the two rows
@@ -64,7 +68,6 @@ struct Ctx {
   bf16 *Q_hi = nullptr, *Q_lo = nullptr;    // [n][n] Q   (row i, col m)
   bf16 *QT_hi = nullptr, *QT_lo = nullptr;  // [n][n] Q^T (row m, col k)
   bf16 *H_hi = nullptr, *H_lo = nullptr;    // [n][n] split planes of the damped unscaled H
-  float* Whs = nullptr;         // [p][n] scaled weights
   float* V = nullptr;           // [p][n]
   bf16 *R_hi = nullptr, *R_lo = nullptr;    // [p][n]
   float* Y = nullptr;           // [p][n] (also the local-search gradient g)
@@ -72,7 +75,9 @@ struct Ctx {
   float* partials = nullptr;    // [T_max][slots][2]
   int partial_slots = 0;
   double* scal = nullptr;       // small fp64 scalars (objective, counters)
-  float* fscal = nullptr;       // [0] 1 / scale of the Q planes, [1] 1 / scale of the H planes, [2] scale of the H planes
+  float* fscal = nullptr;       // [0] 1 / scale of the Q planes, [1] 1 / scale of the H planes, [2] scale of the H planes,
+                                // [3] 1 / scale and [4] scale of the shifted Q^T planes, [5] their largest magnitude,
+                                // [6..8] 1 / scale, scale, largest magnitude of the explicit operator's planes
   float* rs_R = nullptr;        // [p] inverse row scales of the R (and E) planes
   float* rs_Y = nullptr;        // [p] inverse row scales of the Y' planes
   bf16 *XT_hi = nullptr, *XT_lo = nullptr;  // [n][XT_ROWS] transposed chunk of X
@@ -97,10 +102,15 @@ void launch_grid_fit(Ctx* c, const float* W0, int p, int bits, int gs, int symme
 void launch_admm_rows(Ctx* c, const EpiParams& P, int p, bf16* hi, bf16* lo, float* row_inv);
 void launch_grid_fit_mse(Ctx* c, const float* W0, int p, int bits, int gs, int symmetric, int points,
                          double min_ratio, float* delta, float* zero);
-void launch_scale_weights(Ctx* c, const float* W0, int p);
+void launch_scale_weights(Ctx* c, const float* W0, int p);   // start of a layer: V = 0, R = 0, finite check of W_hat
 void launch_operand_scales(Ctx* c);   // fscal from diag(H)
 void launch_split_f64(Ctx* c, const double* src, int n, bf16* hi, bf16* lo, bf16* thi, bf16* tlo);
 void launch_split_f32(Ctx* c, const float* src, long long count, bf16* hi, bf16* lo);
+void launch_global_split(Ctx* c, const float* src, long long count, float* slot, bf16* hi, bf16* lo);
+void launch_shifted_qt(Ctx* c);       // mu = mean(td) -> scal[8]; planes of [Q (mu I - T)]^T -> QT_hi / QT_lo, scales -> fscal[3..5]
+void launch_w_out(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes, const float* delta,
+                  const float* zero, const float* V_in, float inv_rho, const float* shift_c, const float* z,
+                  float* W_out);
 void launch_row_split(Ctx* c, const float* src, int p, bf16* hi, bf16* lo, float* row_inv);
 void launch_init_rhs(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes, const float* delta,
                      const float* zero, const float* V_in, float inv_rho, float* R_out);
@@ -126,7 +136,7 @@ size_t tridiag_blocked_scratch_doubles(int n);
 cudaError_t tridiag_form_qt(Ctx* c);                // reflectors -> P64 = Q^T
 size_t stage_factor_stride(int n);                  // floats per penalty in stage_l / stage_invd
 void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count);
-void launch_tridiag_solve(Ctx* c, int p, int stage);
+void launch_tridiag_solve(Ctx* c, const float* Y, int p, int stage, bf16* hi, bf16* lo, float* row_inv);
 
 // ---- local_search.cu ----
 cudaError_t launch_local_search(Ctx* c, const float* W0, int p, int bits, int gs, long long max_moves,

@@ -692,12 +692,16 @@ int solve_ept(int n) { return (((n + SOLVE_THREADS - 1) / SOLVE_THREADS) + 7) & 
 size_t stage_factor_stride(int n) { return (size_t)solve_ept(n) * SOLVE_THREADS; }
 
 __global__ void stage_factors_kernel(const double* __restrict__ td, const double* __restrict__ te, int n,
-                                     const double* __restrict__ rho, int first, int count, int ept,
-                                     float* __restrict__ L, float* __restrict__ invD, int* status) {
+                                     const double* __restrict__ rho, const double* __restrict__ mu_p, int first,
+                                     int count, int ept, float* __restrict__ L, float* __restrict__ invD,
+                                     float* __restrict__ shift_c, int* status) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= count) return;
   const int stage = first + t;
   const double inv_r = 1.0 / rho[stage];
+  // shifted operator: the solve returns (T/rho + I)^{-1} y / (mu + rho); c = rho / (mu + rho) goes to the element update
+  const double wshift = 1.0 / (mu_p[0] + rho[stage]);
+  shift_c[stage] = (float)(rho[stage] * wshift);
   const size_t stride = (size_t)ept * SOLVE_THREADS;
   float* l = L + (size_t)stage * stride;
   float* id = invD + (size_t)stage * stride;
@@ -707,7 +711,7 @@ __global__ void stage_factors_kernel(const double* __restrict__ td, const double
     if (!(piv > 0.0)) bad = true;
     const double ip = 1.0 / piv;
     const size_t q = (size_t)(i % ept) * SOLVE_THREADS + i / ept;
-    id[q] = (float)ip;
+    id[q] = (float)(ip * wshift);
     if (i < n - 1) {
       const double b = te[i] * inv_r;
       const double li = b * ip;
@@ -721,9 +725,9 @@ __global__ void stage_factors_kernel(const double* __restrict__ td, const double
 }
 
 void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count) {
-  stage_factors_kernel<<<(count + 63) / 64, 64, 0, c->stream>>>(c->td, c->te, c->n, rho_dev, first, count,
-                                                               solve_ept(c->n), c->stage_l, c->stage_invd,
-                                                               c->status);
+  stage_factors_kernel<<<(count + 63) / 64, 64, 0, c->stream>>>(c->td, c->te, c->n, rho_dev, c->scal + 8, first,
+                                                               count, solve_ept(c->n), c->stage_l, c->stage_invd,
+                                                               c->shift_c, c->status);
   c->launches++;
 }
 
@@ -1065,42 +1069,42 @@ tridiag_solve_rows_kernel(const float* __restrict__ Y, int p, int n, const float
 }
 
 template <int EPT, int R>
-static void launch_solve_rows_t(Ctx* c, int p, int stage, int ctas_per_sm) {
+static void launch_solve_rows_t(Ctx* c, const float* Y, int p, int stage, int ctas_per_sm, bf16* hi, bf16* lo,
+                                float* row_inv) {
   const size_t fs = stage_factor_stride(c->n);
   const int groups = (p + R - 1) / R;
   int blocks = c->num_sms * ctas_per_sm;
   if (blocks > groups) blocks = groups;
   if (c->n == EPT * SOLVE_THREADS)
     tridiag_solve_rows_kernel<EPT, R, true><<<blocks, SOLVE_THREADS, 0, c->stream>>>(
-        c->Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi, c->Y_lo,
-        c->rs_Y);
+        Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, hi, lo, row_inv);
   else
     tridiag_solve_rows_kernel<EPT, R, false><<<blocks, SOLVE_THREADS, 0, c->stream>>>(
-        c->Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi, c->Y_lo,
-        c->rs_Y);
+        Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, hi, lo, row_inv);
 }
 
 template <int EPT>
-static void launch_solve_t(Ctx* c, int p, int stage, int blocks) {
+static void launch_solve_t(Ctx* c, const float* Y, int p, int stage, int blocks, bf16* hi, bf16* lo,
+                           float* row_inv) {
   const size_t fs = stage_factor_stride(c->n);
   const size_t smem = (size_t)2 * EPT * SOLVE_THREADS * sizeof(float);
   if (ensure_dynamic_smem((const void*)tridiag_solve_kernel<EPT>, (int)smem) != cudaSuccess) return;
   tridiag_solve_kernel<EPT><<<blocks, SOLVE_THREADS, smem, c->stream>>>(
-      c->Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, c->Y_hi, c->Y_lo,
-      c->rs_Y);
+      Y, p, c->n, c->stage_l + (size_t)stage * fs, c->stage_invd + (size_t)stage * fs, hi, lo, row_inv);
 }
 
-void launch_tridiag_solve(Ctx* c, int p, int stage) {
+// rows [0, p) of Y (fp32, [p][n]) -> planes hi / lo with one inverse scale per row
+void launch_tridiag_solve(Ctx* c, const float* Y, int p, int stage, bf16* hi, bf16* lo, float* row_inv) {
   int blocks = c->num_sms * 3;                             // resident CTAs; each loads the factor once
   if (blocks > p) blocks = p;
   switch (solve_ept(c->n)) {
-    case 8: launch_solve_rows_t<8, SOLVE_ROWS>(c, p, stage, 3); break;
-    case 16: launch_solve_rows_t<16, SOLVE_ROWS>(c, p, stage, 3); break;
-    case 24: launch_solve_t<24>(c, p, stage, blocks); break;
-    case 32: launch_solve_t<32>(c, p, stage, blocks); break;
-    case 40: launch_solve_t<40>(c, p, stage, blocks); break;
-    case 48: launch_solve_t<48>(c, p, stage, blocks); break;
-    default: launch_solve_t<56>(c, p, stage, blocks); break;     // n <= 14336
+    case 8: launch_solve_rows_t<8, SOLVE_ROWS>(c, Y, p, stage, 3, hi, lo, row_inv); break;
+    case 16: launch_solve_rows_t<16, SOLVE_ROWS>(c, Y, p, stage, 3, hi, lo, row_inv); break;
+    case 24: launch_solve_t<24>(c, Y, p, stage, blocks, hi, lo, row_inv); break;
+    case 32: launch_solve_t<32>(c, Y, p, stage, blocks, hi, lo, row_inv); break;
+    case 40: launch_solve_t<40>(c, Y, p, stage, blocks, hi, lo, row_inv); break;
+    case 48: launch_solve_t<48>(c, Y, p, stage, blocks, hi, lo, row_inv); break;
+    default: launch_solve_t<56>(c, Y, p, stage, blocks, hi, lo, row_inv); break;     // n <= 14336
   }
   c->launches++;
 }

@@ -151,12 +151,18 @@ __global__ void __launch_bounds__(TB_THREADS, 1) tridiag_blocked_kernel(TrbArgs 
         while (nr * Sf < 32 && Sf < nseg) Sf <<= 1;
         const int sp = (nseg + Sf - 1) / Sf;
         const int items = nr * Sf;
-        for (int it = warp; it < items; it += 32) {
+        // Odd columns sweep the matrix backwards (last row first, last segment first): the end of one sweep is
+        // the start of the next, so whatever part of the trailing matrix the L2 still holds is read from there
+        // before anything is fetched from HBM again.
+        const bool back = (k & 1) != 0;
+        for (int itw = warp; itw < items; itw += 32) {
+          const int it = back ? items - 1 - itw : itw;
           const int rq = it / Sf, part = it - rq * Sf;
           const double* arow = a.A + (size_t)(c + (size_t)(tA + rq) * G) * n;
           double acc = 0.0;
-          const int s_end = (part + 1) * sp < nseg ? (part + 1) * sp : nseg;
-          for (int sg = part * sp; sg < s_end; ++sg) {
+          const int s_beg = part * sp, s_end = (part + 1) * sp < nseg ? (part + 1) * sp : nseg;
+          for (int sq = s_beg; sq < s_end; ++sq) {
+            const int sg = back ? s_beg + s_end - 1 - sq : sq;
             const int i0 = i_lo + (sg << 8) + lane * 2;
             double2 av[4];
 #pragma unroll

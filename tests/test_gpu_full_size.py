@@ -11,8 +11,9 @@ A whole 4096 x 4096 layer is far beyond what the fp64 oracle finishes in seconds
     other d_in = 4096 layers, 16 where d_in = 12288;
   * properties that hold at any size: Q orthogonal and Q T Q^T = H~ for the one-time factorisation,
     grid feasibility, error ordering RTN > ADMM >= local search.
-The oracle receives the GPU's damped fp32 Hessian as its H, so that both sides iterate on bit-identical
-inputs; that Hessian is itself compared with the definition in the same test.
+The oracle receives the GPU's damped fp32 Hessian as its H and the GPU's fp32 grid (Delta, z0), so that
+both sides iterate on bit-identical inputs; that Hessian is itself compared with the definition, and that
+grid with the oracle's own fit, in the same test.
 """
 import numpy as np
 import pytest
@@ -106,6 +107,18 @@ def sampled_input_channels(spec, count=36):
     return sorted(set(out))
 
 
+def checked_grid(Wn, spec, delta_gpu, z0_gpu):
+    """The GPU's grid (Delta, z0 as the fp32 values the call returned), after it has been compared with the
+    oracle's fp64 fit of the same weights: Delta to the two fp32 roundings of (hi - lo) / levels, z0 exactly.
+    The oracle then iterates on this grid, so that both sides solve the same problem: a grid that differs in
+    its 8th digit moves the level k Delta by up to 2^bits times as much, which near a rounding tie is a
+    different code."""
+    d_o, z_o = O.grid_fit(Wn, spec.bits, spec.group_size, spec.symmetric)
+    assert np.allclose(delta_gpu, d_o, rtol=2e-7, atol=0)
+    assert np.array_equal(z0_gpu, z_o)
+    return delta_gpu, z0_gpu
+
+
 def check_hessian_entries(H, xc, cols, n_tokens):
     """H[a, b] for a, b in `cols` against sum_t X_ta X_tb / N + 0.01 mean(diag) [a == b] (Sec. 3.1, App. D),
     to 1e-4 of sqrt(G_aa G_bb).  xc: the columns `cols` of all calibration rows, fp64."""
@@ -193,10 +206,10 @@ def test_cfg2_sampled_channels_against_oracle(cfg2):
     assert len(rows) == 256
     H = np64(cfg2["H"])
     Wn = np64(cfg2["W"])[rows]
-    res = O.quantize_layer(H, Wn, spec.bits, spec.group_size, spec.symmetric, np.array(spec.rho()))
+    grid = checked_grid(Wn, spec, np64(cfg2["scale"])[rows], np64(cfg2["zero"])[rows])
+    res = O.quantize_layer(H, Wn, spec.bits, spec.group_size, spec.symmetric, np.array(spec.rho()), grid=grid)
     ca = cfg2["codes_admm"][rows].cpu().numpy()
     cf = cfg2["codes_final"][rows].cpu().numpy()
-    assert np.allclose(np64(cfg2["scale"])[rows], res.admm.delta, rtol=2e-7, atol=0)
     assert (ca == res.admm.codes).mean() >= CODE_AGREEMENT, (ca == res.admm.codes).mean()
     assert (cf == res.ls.codes).mean() >= CODE_AGREEMENT, (cf == res.ls.codes).mean()
     # no band of 128 channels falls behind the others
@@ -293,10 +306,10 @@ def _solve_and_compare_sampled_channels(spec, rows):
     assert np.array_equal(H, H.T)
     assert check_hessian_entries(H, np.concatenate(xcols), cols, spec.n_tokens) >= 1000
     Wn = np64(W)[rows]
-    res = O.quantize_layer(H, Wn, spec.bits, spec.group_size, spec.symmetric, np.array(spec.rho()))
+    grid = checked_grid(Wn, spec, np64(scale)[rows], np64(zero)[rows])
+    res = O.quantize_layer(H, Wn, spec.bits, spec.group_size, spec.symmetric, np.array(spec.rho()), grid=grid)
     ca = codes_admm[rows].cpu().numpy()
     cf = codes[rows].cpu().numpy()
-    assert np.allclose(np64(scale)[rows], res.admm.delta, rtol=2e-7, atol=0)
     assert (ca == res.admm.codes).mean() >= CODE_AGREEMENT, (ca == res.admm.codes).mean()
     assert (cf == res.ls.codes).mean() >= CODE_AGREEMENT, (cf == res.ls.codes).mean()
     e_a = O.objective(H, Wn, O.dequantize(ca, res.admm.delta, res.admm.z0))

@@ -559,6 +559,62 @@ def test_fused_and_row_pass_element_update_agree():
     assert abs(out[0][4] - out[1][4]) <= 1e-12 * out[0][4]     # the error sum is accumulated atomically
 
 
+@pytest.mark.parametrize("kw", [dict(d_in=256, d_out=640, n_tokens=4096, bits=4, group_size=128),
+                                dict(d_in=264, d_out=400, n_tokens=3000, bits=3, group_size=0)])
+def test_explicit_operator_route_against_oracle_and_two_product_route(kw):
+    """Layers with more output than input channels form the n x n operator of the W-update once per iteration and
+    apply it in one product.  Same operator, other rounding: both routes meet the oracle's bars, and a context
+    too narrow for the explicit route refuses it."""
+    spec = wl.small_case(**kw)
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(spec.d_in, spec.d_out, T_max=spec.T)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=spec.rho())
+    H, Wn, res = _solve_oracle(spec)
+    errs = []
+    for route in (1, 2, 0):
+        resid = torch.zeros(spec.T, 2, device=DEV)
+        codes, scale, zero, rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, resid=resid,
+                                                     wupdate_route=route)
+        assert sol.last_device_status() == B.OK
+        assert (codes.cpu().numpy() == res.admm.codes).mean() >= CODE_AGREEMENT, route
+        assert abs(rep.err_before - res.err_admm) <= ERR_TOL * res.err_admm
+        assert np.allclose(resid.cpu().numpy()[:, 0], res.admm.r, rtol=2e-3, atol=1e-6 * res.admm.r.max())
+        errs.append(rep.err_before)
+    assert abs(errs[0] - errs[1]) <= ERR_TOL * errs[0]
+    narrow = B.Solver(spec.d_in, spec.d_in, T_max=spec.T)           # d_out_max = d_in: no room for the operator
+    narrow.hessian_reset()
+    narrow.hessian_accumulate(wl.gen_x_chunk(spec, 0, DEV))
+    narrow.factor(rho=spec.rho())
+    with pytest.raises(B.AdmmqError) as e:
+        narrow.quantize_layer(W[: spec.d_in].contiguous(), spec.bits, spec.group_size, spec.symmetric, wupdate_route=2)
+    assert e.value.status == B.ERR_UNSUPPORTED
+
+
+def test_one_plane_products_of_the_late_iterations():
+    """Once the penalty is large the products carry a part of the W-update so small that one fp16 plane per
+    operand resolves it below fp32: the default run switches there, a run forced to two planes does not, and
+    both give the oracle's codes."""
+    spec = wl.small_case(d_in=520, d_out=264, n_tokens=4096, bits=4, group_size=0, T=90, gamma=1.25)
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(spec.d_in, spec.d_out, T_max=spec.T)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=spec.rho())
+    H, Wn, res = _solve_oracle(spec)
+    c0, s0, z0, rep0 = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric)
+    c2, s2, z2, rep2 = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, product_planes=2)
+    assert sol.last_device_status() == B.OK
+    assert 10 <= rep0.one_plane_iters < spec.T and rep2.one_plane_iters == 0
+    assert (c0.cpu().numpy() == res.admm.codes).mean() >= CODE_AGREEMENT
+    assert (c2.cpu().numpy() == res.admm.codes).mean() >= CODE_AGREEMENT
+    assert (c0 == c2).float().mean().item() >= 0.9995
+    assert abs(rep0.err_before - res.err_admm) <= ERR_TOL * res.err_admm
+
+
 def test_stacked_layers_share_one_factorisation():
     """Projections that read the same activations share H: stacking their weights into one call gives, channel
     by channel, exactly what separate calls on the same factorisation give (output channels are independent
