@@ -23,6 +23,13 @@ extern "C" {
  * below 1000 cycles. */
 admmq_status admmq_test_set_wait(admmq_ctx* ctx, long long wait_limit_cycles, int hold_loads);
 
+/* admmq_w_update with the result left in the form the solver itself works with: d_Z_out [d_out][d_in] fp32
+ * receives W^(t+1) - W_hat' (scaled coordinates), i.e. the correction of Eq. 7 without the weight-sized term
+ * W_hat' that admmq_w_update adds before it rounds to fp32.  For accuracy tests at the scale of a grid step. */
+admmq_status admmq_test_w_update_correction(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
+                                            const unsigned char* d_codes, const float* d_scale,
+                                            const float* d_zero, const float* d_V, double rho, float* d_Z_out);
+
 #ifdef __cplusplus
 }
 #endif

@@ -28,7 +28,7 @@ EXPORTS = [
     "admmq_w_update", "admmq_local_search", "admmq_objective", "admmq_get_hessian",
     "admmq_launch_count", "admmq_set_timing", "admmq_reset_timing", "admmq_get_timing",
     "admmq_objective_static", "admmq_get_factor", "admmq_pair_swap", "admmq_test_set_wait",
-    "admmq_hessian_export", "admmq_hessian_import",
+    "admmq_hessian_export", "admmq_hessian_import", "admmq_test_w_update_correction",
 ]
 T_HESSIAN_PRODUCT, T_TRANSPOSE, T_FACTOR, T_WUPDATE_PRODUCT1, T_TRIDIAG_SOLVE, T_WUPDATE_PRODUCT2, \
     T_GRADIENT_PRODUCT, T_LOCAL_SEARCH, T_ROW_SPLIT, T_WUPDATE_ONE_PLANE = range(10)
@@ -104,6 +104,7 @@ def load_library(path: Optional[str] = None):
     lib.admmq_quantize_layer.argtypes = [vp, vp, ci, C.POINTER(QuantCfg), vp, vp, vp, vp, vp,
                                          C.POINTER(Report)]
     lib.admmq_w_update.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, cd, vp]
+    lib.admmq_test_w_update_correction.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, cd, vp]
     lib.admmq_local_search.argtypes = [vp, vp, ci, C.POINTER(LsCfg), vp, vp, vp, vp, C.POINTER(Report)]
     lib.admmq_objective.argtypes = [vp, vp, ci, ci, vp, vp, vp, C.POINTER(cd)]
     lib.admmq_pair_swap.argtypes = [vp, vp, ci, C.POINTER(PairSwapCfg), vp, vp, vp, vp, C.POINTER(Report)]
@@ -252,6 +253,15 @@ class Solver:
         _check(self.lib.admmq_w_update(self.h, _ptr(W0), W0.shape[0], group_size, _ptr(codes), _ptr(scale),
                                        _ptr(zero), _ptr(V), float(rho), _ptr(W_out)), "admmq_w_update")
         return W_out
+
+    def w_update_correction(self, W0, group_size, codes, scale, zero, V, rho: float, Z_out=None):
+        """W^(t+1) - W_hat' of one W-update (admmq_testing.h): the same call as w_update without the weight-sized
+        term, for accuracy checks at the scale of a grid step."""
+        Z_out = Z_out if Z_out is not None else torch.empty_like(W0)
+        _check(self.lib.admmq_test_w_update_correction(self.h, _ptr(W0), W0.shape[0], group_size, _ptr(codes),
+                                                       _ptr(scale), _ptr(zero), _ptr(V), float(rho), _ptr(Z_out)),
+               "admmq_test_w_update_correction")
+        return Z_out
 
     def local_search(self, W0, bits, group_size, codes, scale, zero, Wq=None, max_moves_per_col: int = 0,
                      accept_tol: float = 1e-6, report: bool = True):

@@ -87,6 +87,8 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   c.H = cv.take<float>(nn);
   c.s = cv.take<float>(n);
   c.inv_s = cv.take<float>(n);
+  c.s64 = cv.take<double>(n);
+  c.inv_s64 = cv.take<double>(n);
   c.hdiag = cv.take<float>(n);
   c.A64 = cv.take<double>(nn);
   c.P64 = cv.take<double>(nn);
@@ -96,7 +98,7 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   c.pvec = cv.take<double>(n);
   c.stage_l = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
   c.stage_invd = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
-  c.shift_c = cv.take<float>((size_t)T + 1);
+  c.shift_c = cv.take<double>((size_t)T + 1);
   c.Qs32 = explicit_operator_possible(n, p) ? cv.take<float>(nn) : nullptr;
   c.ps_totals = cv.take<double>(PAIR_BATCH_MAX);
   c.ps_chosen = cv.take<int>(16);
@@ -541,7 +543,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.W0 = d_W0;
   e.V = c->V;
   e.codes = d_codes;
-  e.s = c->s;
+  e.s = c->s64;
   e.inv_s = c->inv_s;
   e.delta = d_scale;
   e.zero = d_zero;
@@ -554,9 +556,9 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     const double rho = c->rho_host[t];
     const double rho_next = (t + 1 < T) ? c->rho_host[t + 1] : rho;
     e.first_iter = (t == 0);
-    e.rho = (float)rho;
-    e.inv_rho = (float)(1.0 / rho);
-    e.inv_rho_next = (float)(1.0 / rho_next);
+    e.rho = rho;
+    e.inv_rho = 1.0 / rho;
+    e.inv_rho_next = 1.0 / rho_next;
     e.partials = c->partials + (size_t)t * c->partial_slots * 2;
     e.shift_c = c->shift_c + t;
     const int planes = (cfg->product_planes == 2 || cfg->fused_epilogue) ? 2 : c->planes_host[t];
@@ -617,9 +619,25 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   return st;
 }
 
+static admmq_status w_update_call(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
+                                  const unsigned char* d_codes, const float* d_scale, const float* d_zero,
+                                  const float* d_V, double rho, float* d_W_out, int correction_only);
+
 admmq_status admmq_w_update(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
                             const unsigned char* d_codes, const float* d_scale, const float* d_zero,
                             const float* d_V, double rho, float* d_W_out) {
+  return w_update_call(ctx, d_W0, d_out, group_size, d_codes, d_scale, d_zero, d_V, rho, d_W_out, 0);
+}
+
+admmq_status admmq_test_w_update_correction(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
+                                            const unsigned char* d_codes, const float* d_scale,
+                                            const float* d_zero, const float* d_V, double rho, float* d_Z_out) {
+  return w_update_call(ctx, d_W0, d_out, group_size, d_codes, d_scale, d_zero, d_V, rho, d_Z_out, 1);
+}
+
+static admmq_status w_update_call(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
+                                  const unsigned char* d_codes, const float* d_scale, const float* d_zero,
+                                  const float* d_V, double rho, float* d_W_out, int correction_only) {
   admmq_status st = check_layer_args(ctx, d_W0, d_out, 2, group_size, d_codes, d_scale, d_zero);
   if (st != ADMMQ_OK) return st;
   if (!d_V || !d_W_out || !aligned16(d_V) || !aligned16(d_W_out)) return ADMMQ_ERR_INVALID_ARG;
@@ -627,7 +645,7 @@ admmq_status admmq_w_update(admmq_ctx* ctx, const float* d_W0, int d_out, int gr
   Ctx* c = &ctx->c;
   const int n = c->n, p = d_out, gs = group_of(n, group_size);
   launch_scale_weights(c, d_W0, p);
-  launch_init_rhs(c, d_W0, p, gs, d_codes, d_scale, d_zero, d_V, (float)(1.0 / rho), c->Y);
+  launch_init_rhs(c, d_W0, p, gs, d_codes, d_scale, d_zero, d_V, 1.0 / rho, c->Y);
   launch_row_split(c, c->Y, p, c->R_hi, c->R_lo, c->rs_R);
   const int stage = c->T_max;                              // spare slot for an ad-hoc penalty
   ctx->rho_adhoc = rho;
@@ -640,7 +658,8 @@ admmq_status admmq_w_update(admmq_ctx* ctx, const float* d_W0, int d_out, int gr
   e.C = c->Y;                                               // free once its planes exist
   e.ldc = n;
   if (w_update_products(ctx, p, stage, e, 2) != cudaSuccess) return ADMMQ_ERR_CUDA;
-  launch_w_out(c, d_W0, p, gs, d_codes, d_scale, d_zero, d_V, (float)(1.0 / rho), c->shift_c + stage, c->Y, d_W_out);
+  launch_w_out(c, d_W0, p, gs, d_codes, d_scale, d_zero, d_V, 1.0 / rho, c->shift_c + stage, c->Y, d_W_out,
+               correction_only);
   return cudaGetLastError() == cudaSuccess ? ADMMQ_OK : ADMMQ_ERR_CUDA;
 }
 

@@ -108,7 +108,7 @@ __global__ void diag_sum_kernel(const float* __restrict__ Hraw, int n, double in
 __global__ void finalize_diag_kernel(const float* __restrict__ Hraw, int n, double inv_N,
                                      double damp_frac, int precondition, const double* __restrict__ dsum,
                                      float* __restrict__ hdiag, float* __restrict__ s,
-                                     float* __restrict__ inv_s, double* s64, int* status) {
+                                     float* __restrict__ inv_s, double* s64, double* inv_s64, int* status) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const double lam = damp_frac * dsum[0] / n;
@@ -119,10 +119,12 @@ __global__ void finalize_diag_kernel(const float* __restrict__ Hraw, int n, doub
     s[i] = 1.f;
     inv_s[i] = 1.f;
     s64[i] = 1.0;
+    inv_s64[i] = 1.0;
     return;
   }
   const double sv = precondition ? sqrt((double)hii) : 1.0;
   s64[i] = sv;
+  inv_s64[i] = 1.0 / sv;
   s[i] = (float)sv;
   inv_s[i] = (float)(1.0 / sv);
 }
@@ -159,12 +161,12 @@ void launch_symmetric_copy(Ctx* c, float* out) {
 void launch_finalize(Ctx* c, double damp_frac, int precondition) {
   const int n = c->n;
   const double inv_N = 1.0 / (double)c->n_tokens;
-  double* s64 = c->pvec;  // scratch [n]; consumed before the reduction starts
+  double* s64 = c->s64;
   diag_sum_kernel<<<1, 1024, 0, c->stream>>>(c->H_raw, n, inv_N, c->scal);
   LAUNCH(c);
   finalize_diag_kernel<<<(n + 255) / 256, 256, 0, c->stream>>>(c->H_raw, n, inv_N, damp_frac,
                                                               precondition, c->scal, c->hdiag, c->s,
-                                                              c->inv_s, s64, c->status);
+                                                              c->inv_s, s64, c->inv_s64, c->status);
   LAUNCH(c);
   dim3 grid((n + 255) / 256, n);
   finalize_full_kernel<<<grid, 256, 0, c->stream>>>(c->H_raw, n, inv_N, c->hdiag, s64, c->H, c->A64,
@@ -515,24 +517,25 @@ void launch_shifted_qt(Ctx* c) {
 // state as init_rhs_kernel built it, z is the product's output.
 __global__ void w_out_kernel(long long total, int n, int gs, int ng, const unsigned char* __restrict__ codes,
                              const float* __restrict__ delta, const float* __restrict__ zero,
-                             const float* __restrict__ V, float inv_rho, const float* __restrict__ s,
-                             const float* __restrict__ W0, const float* __restrict__ shift_c, const float* __restrict__ z,
-                             float* __restrict__ W_out) {
+                             const float* __restrict__ V, double inv_rho, const double* __restrict__ s,
+                             const float* __restrict__ W0, const double* __restrict__ shift_c, const float* __restrict__ z,
+                             float* __restrict__ W_out, int correction_only) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
   const int col = (int)(idx % n);
   const long long gi = (idx / n) * ng + col / gs;
-  const double e = (double)s[col] * fma((double)delta[gi], (double)codes[idx], (double)zero[gi] - (double)W0[idx]);
-  const float r = fmaf(-V[idx], inv_rho, (float)e);
-  W_out[idx] = fmaf(s[col], W0[idx], fmaf(shift_c[0], r, z[idx]));
+  const double e = s[col] * fma((double)delta[gi], (double)codes[idx], (double)zero[gi] - (double)W0[idx]);
+  const double r = fma(-(double)V[idx], inv_rho, e);
+  const double corr = fma(shift_c[0], r, (double)z[idx]);                     // W^(t+1) - W_hat'
+  W_out[idx] = (float)(correction_only ? corr : fma(s[col], (double)W0[idx], corr));
 }
 
 void launch_w_out(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes, const float* delta,
-                  const float* zero, const float* V_in, float inv_rho, const float* shift_c, const float* z,
-                  float* W_out) {
+                  const float* zero, const float* V_in, double inv_rho, const double* shift_c, const float* z,
+                  float* W_out, int correction_only) {
   const long long total = (long long)p * c->n;
   w_out_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
-      total, c->n, gs, c->n / gs, codes, delta, zero, V_in, inv_rho, c->s, W0, shift_c, z, W_out);
+      total, c->n, gs, c->n / gs, codes, delta, zero, V_in, inv_rho, c->s64, W0, shift_c, z, W_out, correction_only);
   LAUNCH(c);
 }
 
@@ -656,7 +659,7 @@ void launch_row_split(Ctx* c, const float* src, int p, bf16* hi, bf16* lo, float
 __global__ void init_rhs_kernel(long long total, int n, int gs, int ng,
                                 const unsigned char* __restrict__ codes,
                                 const float* __restrict__ delta, const float* __restrict__ zero,
-                                const float* __restrict__ V, float inv_rho, const float* __restrict__ s,
+                                const float* __restrict__ V, double inv_rho, const double* __restrict__ s,
                                 const float* __restrict__ W0, float* __restrict__ R) {
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= total) return;
@@ -664,15 +667,15 @@ __global__ void init_rhs_kernel(long long total, int n, int gs, int ng,
   const long long row = idx / n;
   const long long gi = row * ng + col / gs;
   // D - W_hat' = s (z0 + Delta k - w_hat): the difference of weight-sized numbers is taken in fp64
-  const double e = (double)s[col] * fma((double)delta[gi], (double)codes[idx], (double)zero[gi] - (double)W0[idx]);
-  R[idx] = fmaf(-V[idx], inv_rho, (float)e);
+  const double e = s[col] * fma((double)delta[gi], (double)codes[idx], (double)zero[gi] - (double)W0[idx]);
+  R[idx] = (float)fma(-(double)V[idx], inv_rho, e);
 }
 
 void launch_init_rhs(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes, const float* delta,
-                     const float* zero, const float* V_in, float inv_rho, float* R_out) {
+                     const float* zero, const float* V_in, double inv_rho, float* R_out) {
   const long long total = (long long)p * c->n;
   init_rhs_kernel<<<(unsigned)((total + 255) / 256), 256, 0, c->stream>>>(
-      total, c->n, gs, c->n / gs, codes, delta, zero, V_in, inv_rho, c->s, W0, R_out);
+      total, c->n, gs, c->n / gs, codes, delta, zero, V_in, inv_rho, c->s64, W0, R_out);
   LAUNCH(c);
 }
 
@@ -763,24 +766,24 @@ void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned 
 // ------------------------------------------------------------------------------------------------
 // (W~ - W_hat') / s of one element: the product's output plus its c R part (R rebuilt from the codes and the dual
 // as in the element update), plus V/rho.
-__device__ __forceinline__ float refresh_target(float zp, float w0, float v, int code_old, int first_iter, float s,
-                                                float inv_s, float dl, float z0, float cshift, float inv_rho) {
-  const float e_old = first_iter ? 0.0f
-                                 : (float)((double)s * fma((double)dl, (double)code_old, (double)z0 - (double)w0));
+__device__ __forceinline__ double refresh_target(float zp, float w0, float v, int code_old, int first_iter, double s,
+                                                 float inv_s, float dl, float z0, float cshift, float inv_rho) {
+  const float e_old = first_iter ? 0.0f : (float)(s * fma((double)dl, (double)code_old, (double)z0 - (double)w0));
   const float z = fmaf(cshift, fmaf(-v, inv_rho, e_old), zp);
-  return fmaf(v, inv_rho, z) * inv_s;
+  return (double)(fmaf(v, inv_rho, z) * inv_s);           // the same fp32 steps as the element update
 }
 
 __global__ void __launch_bounds__(256)
 refresh_eval_kernel(const float* __restrict__ Zc, const float* __restrict__ W0, const float* __restrict__ V,
-                    const unsigned char* __restrict__ codes, int first_iter, const float* __restrict__ shift_c,
-                    const float* __restrict__ s, const float* __restrict__ inv_s, int p, int n, int gs, int kmax,
-                    int symmetric, float inv_rho, const float* __restrict__ delta, const float* __restrict__ zero,
+                    const unsigned char* __restrict__ codes, int first_iter, const double* __restrict__ shift_c,
+                    const double* __restrict__ s, const float* __restrict__ inv_s, int p, int n, int gs, int kmax,
+                    int symmetric, double inv_rho, const float* __restrict__ delta, const float* __restrict__ zero,
                     float* __restrict__ cand_delta, float* __restrict__ cand_zero, double* __restrict__ partial) {
   __shared__ double scratch[32];
   const int ng = n / gs, lane = threadIdx.x & 31;
   const long long groups = (long long)p * ng;
-  const float cs = shift_c[0];
+  const float cs = (float)shift_c[0];
+  const float inv_rho_f = (float)inv_rho;
   double e_old = 0.0, e_new = 0.0;
   for (long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; gw < groups;
        gw += ((long long)gridDim.x * blockDim.x) >> 5) {
@@ -789,9 +792,9 @@ refresh_eval_kernel(const float* __restrict__ Zc, const float* __restrict__ W0, 
     const float d0 = delta[gw], z0 = zero[gw];
     double lo = INFINITY, hi = -INFINITY;
     for (int i = lane; i < gs; i += 32) {
-      const float u = refresh_target(Zc[base + i], W0[base + i], V[base + i], first_iter ? 0 : (int)codes[base + i],
-                                     first_iter, s[gq * gs + i], inv_s[gq * gs + i], d0, z0, cs, inv_rho);
-      const double y = (double)W0[base + i] + (double)u;
+      const double u = refresh_target(Zc[base + i], W0[base + i], V[base + i], first_iter ? 0 : (int)codes[base + i],
+                                      first_iter, s[gq * gs + i], inv_s[gq * gs + i], d0, z0, cs, inv_rho_f);
+      const double y = (double)W0[base + i] + u;
       lo = fmin(lo, y);
       hi = fmax(hi, y);
     }
@@ -814,10 +817,10 @@ refresh_eval_kernel(const float* __restrict__ Zc, const float* __restrict__ W0, 
     const double id0 = 1.0 / (double)d0, idn = 1.0 / (double)dn;
     double a = 0.0, b = 0.0;
     for (int i = lane; i < gs; i += 32) {
-      const double sv = (double)s[gq * gs + i];
-      const double u = (double)refresh_target(Zc[base + i], W0[base + i], V[base + i],
+      const double sv = s[gq * gs + i];
+      const double u = refresh_target(Zc[base + i], W0[base + i], V[base + i],
                                               first_iter ? 0 : (int)codes[base + i], first_iter, s[gq * gs + i],
-                                              inv_s[gq * gs + i], d0, z0, cs, inv_rho);
+                                              inv_s[gq * gs + i], d0, z0, cs, inv_rho_f);
       const double w = (double)W0[base + i];
       const double k0 = fmin(fmax(rint(((w - (double)z0) + u) * id0), 0.0), (double)kmax);
       const double kn = fmin(fmax(rint(((w - (double)zn) + u) * idn), 0.0), (double)kmax);
@@ -878,7 +881,7 @@ __global__ void __launch_bounds__(256) admm_elementwise_kernel(EpiParams P, cons
                                                                int n) {
   __shared__ float red[32];
   float r2 = 0.f, s2 = 0.f;
-  const float cs = P.shift_c[0];
+  const float cs = (float)P.shift_c[0];
   for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
     const int col = (int)(idx % n);
@@ -911,7 +914,7 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
   float r2 = 0.f, s2 = 0.f;
   const int gs = P.group_size;
   const int gsh = (gs & (gs - 1)) == 0 ? 31 - __clz(gs) : -1;      // group index by shift when the size allows
-  const float cs = P.shift_c[0];
+  const float cs = (float)P.shift_c[0];
   for (int j = blockIdx.x; j < p; j += gridDim.x) {
     const size_t base = (size_t)j * n;
     const float* dlt = P.delta + (size_t)j * P.n_groups;
@@ -921,8 +924,9 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
       const float4 z = *reinterpret_cast<const float4*>(P.C + base + i);
       const float4 wh = *reinterpret_cast<const float4*>(P.W0 + base + i);
       const float4 v = *reinterpret_cast<const float4*>(P.V + base + i);
-      const float4 sv = *reinterpret_cast<const float4*>(P.s + i);
+      const double2 s01 = *reinterpret_cast<const double2*>(P.s + i), s23 = *reinterpret_cast<const double2*>(P.s + i + 2);
       const float4 si = *reinterpret_cast<const float4*>(P.inv_s + i);
+      const struct { double x, y, z, w; } sv = {s01.x, s01.y, s23.x, s23.y};
       uchar4 k = make_uchar4(0, 0, 0, 0);
       if (!P.first_iter) k = *reinterpret_cast<const uchar4*>(P.codes + base + i);
       const int g0 = gsh >= 0 ? i >> gsh : i / gs;

@@ -21,15 +21,15 @@ struct EpiParams {
   const float* W0;          // W_hat, unscaled, as the caller passed it (ADMM element update)
   float* V;                 // dual V (in/out)
   unsigned char* codes;     // codes of D (in: D^(t), out: D^(t+1))
-  const float* s;           // [n] s_i = sqrt(H_ii)
-  const float* inv_s;       // [n] 1 / s_i
+  const double* s;          // [n] s_i = sqrt(H_ii), fp64
+  const float* inv_s;       // [n] 1 / s_i, fp32
   const float* delta;       // [p][n_groups]
   const float* zero;        // [p][n_groups]
   int group_size, n_groups;
   int kmax;                 // 2^bits - 1
   int first_iter;           // 1: D^(0) = W_hat' (Algorithm 1 line 4), codes not yet defined
-  float rho, inv_rho, inv_rho_next;
-  const float* shift_c;     // device scalar c = rho / (mu + rho) of this iteration: the product's output is the
+  double rho, inv_rho, inv_rho_next;
+  const double* shift_c;    // device scalar c = rho / (mu + rho) of this iteration: the product's output is the
                             // W-update correction WITHOUT its c R part, which the element update adds
   float* Rnext;             // next right-hand side D - V/rho_next - W_hat' (fp32; split into planes by a row pass)
   float* partials;          // [slots][2]: per-CTA sums of (W-D)^2 and (D-D_old)^2
@@ -78,25 +78,29 @@ __device__ __forceinline__ GridG grid_g(float dl, float z0) {
   return g;
 }
 // g: the grid the new code is taken on; g_old: the grid code_old refers to (the same one, except in the
-// iteration that accepts a grid refresh).
-__device__ __forceinline__ AdmmElem admm_elem(float zp, float w0, float v, int code_old, float s, float inv_s,
+// iteration that accepts a grid refresh).  fp64 is used where numbers of the weight's size meet and for the
+// rounding decision; the grid-step-sized quantities around them (z, V/rho, the residuals) are fp32, which is the
+// precision they are stored in anyway (measured on the 12288-wide layers: the correction W - W_hat' reaches the
+// decision with an error of 2e-8 to 6e-8 of a grid step rms, the rounding of its own fp32 storage).
+__device__ __forceinline__ AdmmElem admm_elem(float zp, float w0, float v, int code_old, double s, float inv_s,
                                               const GridG& g, const GridG& g_old, float cshift, const EpiParams& P) {
   AdmmElem o;
   const double a = (double)w0 - (double)g.z0;              // w_hat - z0, exact
-  const float e_old = P.first_iter ? 0.0f                                   // D^(0) = W_hat'
-                                   : (float)((double)s * fma((double)g_old.dl, (double)code_old,
-                                                             (double)g_old.z0 - (double)w0));
+  const float e_old = P.first_iter ? 0.0f                  // D^(0) = W_hat'
+                                   : (float)(s * fma((double)g_old.dl, (double)code_old,
+                                                     (double)g_old.z0 - (double)w0));
+  const float inv_rho = (float)P.inv_rho;
   // z = c R + (product output), R = D^(t) - V/rho - W_hat' exactly as the right-hand side was formed
-  const float z = fmaf(cshift, fmaf(-v, P.inv_rho, e_old), zp);
-  const float u = fmaf(v, P.inv_rho, z) * inv_s;           // (W~ - W_hat') / s: target minus weight  (Eq. 8)
+  const float z = fmaf(cshift, fmaf(-v, inv_rho, e_old), zp);
+  const float u = fmaf(v, inv_rho, z) * inv_s;             // (W~ - W_hat') / s: target minus weight  (Eq. 8)
   double k = rint((a + (double)u) * g.inv_dl);             // nearest level, ties to even    (Eq. 10)
   k = fmin(fmax(k, 0.0), (double)P.kmax);
-  const float e_new = (float)((double)s * fma((double)g.dl, k, -a));        // D^(t+1) - W_hat'
+  const float e_new = (float)(s * fma((double)g.dl, k, -a));               // D^(t+1) - W_hat'
   const float wd = z - e_new;                              // W^(t+1) - D^(t+1)
   const float dd = e_new - e_old;                          // D^(t+1) - D^(t)
   o.code = (unsigned char)(int)k;
-  o.v_new = fmaf(P.rho, wd, v);                            // V += rho (W - D)               (Eq. 9)
-  o.r_next = fmaf(-o.v_new, P.inv_rho_next, e_new);        // next R = D - V/rho' - W_hat'
+  o.v_new = fmaf((float)P.rho, wd, v);                     // V += rho (W - D)               (Eq. 9)
+  o.r_next = fmaf(-o.v_new, (float)P.inv_rho_next, e_new); // next R = D - V/rho' - W_hat'
   o.dr2 = wd * wd;
   o.ds2 = dd * dd;
   return o;
@@ -117,7 +121,7 @@ __device__ __forceinline__ void epi_scalar(const EpiParams& P, int row, int col,
     const float z0 = P.zero[(long long)row * P.n_groups + g];
     const GridG gg = grid_g(dl, z0);
     AdmmElem e = admm_elem(acc, P.W0[idx], P.V[idx], P.first_iter ? 0 : (int)P.codes[idx], P.s[col],
-                           P.inv_s[col], gg, gg, P.shift_c[0], P);
+                           P.inv_s[col], gg, gg, (float)P.shift_c[0], P);
     P.codes[idx] = e.code;
     P.V[idx] = e.v_new;
     P.Rnext[idx] = e.r_next;

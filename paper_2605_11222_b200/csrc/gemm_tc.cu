@@ -236,16 +236,16 @@ __device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, 
     const long long o = (long long)row * N + col;
     const float4 w = *reinterpret_cast<const float4*>(P.W0 + o);
     const float4 v = *reinterpret_cast<const float4*>(P.V + o);
-    const float4 s = *reinterpret_cast<const float4*>(P.s + col);
+    const double2 sa = *reinterpret_cast<const double2*>(P.s + col), sb = *reinterpret_cast<const double2*>(P.s + col + 2);
     const float4 is = *reinterpret_cast<const float4*>(P.inv_s + col);
     uint32_t codes = 0u;
     if (!P.first_iter) codes = *reinterpret_cast<const uint32_t*>(P.codes + o);
     const float wh[4] = {w.x, w.y, w.z, w.w};
     const float vv[4] = {v.x, v.y, v.z, v.w};
-    const float ss[4] = {s.x, s.y, s.z, s.w};
+    const double ss[4] = {sa.x, sa.y, sb.x, sb.y};
     const float si[4] = {is.x, is.y, is.z, is.w};
     const bool one_group = (P.group_size & 3) == 0;        // then the 4 columns share (Delta, z0)
-    const float cshift = P.shift_c[0];
+    const float cshift = (float)P.shift_c[0];
     long long gi = (long long)row * P.n_groups + col / P.group_size;
     GridG gg = grid_g(P.delta[gi], P.zero[gi]);
     float vn[4], rn[4];
@@ -333,11 +333,14 @@ __device__ __forceinline__ void epilogue_block(const EpiParams& P, int row0, int
 template <int NP, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_t fmt, EpiParams epi,
-               int* status, long long wait_limit, int hold_loads) {
+               int* status, long long wait_limit, int hold_loads, int flush_kb) {
   constexpr int A_BYTES = BM * BK * 2, BOX_BYTES = BN_BOX * BK * 2, B_BYTES = 2 * BOX_BYTES;
   constexpr int STAGE_BYTES = NP * (A_BYTES + B_BYTES);
   constexpr int STAGES = (NP == 1) ? 4 : 2;
-  constexpr int KB_PER_FLUSH = (NP == 1) ? 3 : 1;        // 12 accumulating MMA steps per flush either way
+  // K blocks accumulated in tensor memory before the workers take the partial: 12 MMA steps (one block with two
+  // planes, three with one) where the result must be good to fp32, as many as the caller allows (flush_kb) where the
+  // operands' own rounding is far above the accumulator's truncation (the one-plane products of the late iterations)
+  const int KB_PER_FLUSH = (NP == 1) ? (flush_kb > 0 ? flush_kb : 3) : 1;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[3 * STAGES + 2 * NPART + 1];
   __shared__ uint32_t tmem_base_slot;
@@ -637,7 +640,7 @@ int gemm_tc_partial_slots(int num_sms) { return num_sms; }
 
 template <int NP, int EPI>
 static cudaError_t launch_tc(Ctx* c, const TcMaps& maps, int M, int N, int K, uint32_t fmt,
-                             const EpiParams& epi) {
+                             const EpiParams& epi, int flush_kb = 0) {
   constexpr int STAGE_BYTES = NP * (BM * BK * 2 + BN * BK * 2);
   constexpr int STAGES = (NP == 1) ? 4 : 2;
   const size_t smem = (size_t)STAGES * STAGE_BYTES + 1024;
@@ -646,7 +649,7 @@ static cudaError_t launch_tc(Ctx* c, const TcMaps& maps, int M, int N, int K, ui
   const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = tiles < c->num_sms ? tiles : c->num_sms;
   gemm_tc_kernel<NP, EPI><<<grid, TC_THREADS, smem, c->stream>>>(maps, M, N, K, fmt, epi, c->status,
-                                                                   c->wait_limit_cycles, c->hold_loads);
+                                                                   c->wait_limit_cycles, c->hold_loads, flush_kb);
   c->launches++;
   return cudaGetLastError();
 }
@@ -670,7 +673,9 @@ cudaError_t gemm_tc(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiPa
   const uint32_t idesc = A.f16 ? 0u : 1u;                  // operand format: 0 = fp16, 1 = bf16
   if (na == 1) {
     if (epi.kind == EPI_ACCUM) return launch_tc<1, EPI_ACCUM>(c, maps, M, N, K, idesc, epi);
-    if (epi.kind == EPI_STORE) return launch_tc<1, EPI_STORE>(c, maps, M, N, K, idesc, epi);
+    // one fp16 plane and a plain store: a W-update product of the late iterations, whose result need not be better
+    // than the 2^-12 of its operands: the whole K range accumulates in tensor memory
+    if (epi.kind == EPI_STORE) return launch_tc<1, EPI_STORE>(c, maps, M, N, K, idesc, epi, A.f16 ? c->one_plane_flush_kb : 0);
     return cudaErrorInvalidValue;
   }
   switch (epi.kind) {

@@ -40,6 +40,7 @@ struct Ctx {
   double mu_host = 1.0, lam_lo = 0.0, lam_hi = 0.0;   // mean and Gershgorin bounds of the spectrum of H~ (host copies)
   long long launches = 0;
   long long wait_limit_cycles = 2000000000LL;   // bound of every device-side wait, about a second
+  int one_plane_flush_kb = 1 << 20;   // K blocks per flush of the one-plane fp16 products (whole K by default)
   int hold_loads = 0;           // failure-handling tests only: the product kernel's producer issues no loads
   // ---- workspace carve-up (device) ----
   char* ws = nullptr;
@@ -49,6 +50,8 @@ struct Ctx {
   float* H = nullptr;           // [n][n] fp32 damped, unscaled
   float* s = nullptr;           // [n]
   float* inv_s = nullptr;       // [n] 1 / s_i
+  double* s64 = nullptr;        // [n] s_i in fp64 (the element update works in fp64)
+  double* inv_s64 = nullptr;    // [n] 1 / s_i in fp64
   float* hdiag = nullptr;       // [n] diag of damped H
   double* A64 = nullptr;        // [n][n] fp64 working copy of H~, reflectors afterwards
   double* P64 = nullptr;        // [n][n] fp64 Q^T
@@ -58,7 +61,7 @@ struct Ctx {
   double* pvec = nullptr;       // [n] matrix-vector scratch of the reduction
   float* stage_l = nullptr;     // [T_max+1][stage_factor_stride(n)] LDL^T multipliers per penalty
   float* stage_invd = nullptr;  // [T_max+1][stage_factor_stride(n)] LDL^T inverse pivots per penalty, times 1 / (mu + rho)
-  float* shift_c = nullptr;     // [T_max+1] c = rho / (mu + rho) per penalty (shifted W-update operator)
+  double* shift_c = nullptr;    // [T_max+1] c = rho / (mu + rho) per penalty (shifted W-update operator)
   float* Qs32 = nullptr;        // [n][n] fp32 Q (mu I - T), or nullptr: input of the explicit-operator route (p_max > n only)
   double* ps_totals = nullptr;  // [PAIR_BATCH_MAX] totals of the candidate pairs of a pair-swap round
   int* ps_chosen = nullptr;     // [1] index of the applied pair, -1: none
@@ -109,11 +112,11 @@ void launch_split_f32(Ctx* c, const float* src, long long count, bf16* hi, bf16*
 void launch_global_split(Ctx* c, const float* src, long long count, float* slot, bf16* hi, bf16* lo);
 void launch_shifted_qt(Ctx* c);       // mu = mean(td) -> scal[8]; planes of [Q (mu I - T)]^T -> QT_hi / QT_lo, scales -> fscal[3..5]
 void launch_w_out(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes, const float* delta,
-                  const float* zero, const float* V_in, float inv_rho, const float* shift_c, const float* z,
-                  float* W_out);
+                  const float* zero, const float* V_in, double inv_rho, const double* shift_c, const float* z,
+                  float* W_out, int correction_only);
 void launch_row_split(Ctx* c, const float* src, int p, bf16* hi, bf16* lo, float* row_inv);
 void launch_init_rhs(Ctx* c, const float* W0, int p, int gs, const unsigned char* codes, const float* delta,
-                     const float* zero, const float* V_in, float inv_rho, float* R_out);
+                     const float* zero, const float* V_in, double inv_rho, float* R_out);
 void launch_reduce_partials(Ctx* c, int T, float* resid);
 void launch_dequant(Ctx* c, int p, int gs, const unsigned char* codes, const float* delta,
                     const float* zero, float* Wq);

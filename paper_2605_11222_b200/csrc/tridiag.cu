@@ -694,14 +694,14 @@ size_t stage_factor_stride(int n) { return (size_t)solve_ept(n) * SOLVE_THREADS;
 __global__ void stage_factors_kernel(const double* __restrict__ td, const double* __restrict__ te, int n,
                                      const double* __restrict__ rho, const double* __restrict__ mu_p, int first,
                                      int count, int ept, float* __restrict__ L, float* __restrict__ invD,
-                                     float* __restrict__ shift_c, int* status) {
+                                     double* __restrict__ shift_c, int* status) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= count) return;
   const int stage = first + t;
   const double inv_r = 1.0 / rho[stage];
   // shifted operator: the solve returns (T/rho + I)^{-1} y / (mu + rho); c = rho / (mu + rho) goes to the element update
   const double wshift = 1.0 / (mu_p[0] + rho[stage]);
-  shift_c[stage] = (float)(rho[stage] * wshift);
+  shift_c[stage] = rho[stage] * wshift;
   const size_t stride = (size_t)ept * SOLVE_THREADS;
   float* l = L + (size_t)stage * stride;
   float* id = invD + (size_t)stage * stride;

@@ -8,7 +8,13 @@ A whole 4096 x 4096 layer is far beyond what the fp64 oracle finishes in seconds
   * because output channels are independent problems given H, the complete ADMM + local-search run of
     sampled output channels: 256 of config 2's 4096 (eight in every band of 128 channels, so that every
     row tile of the product kernel and all four quarters of its tensor-memory lanes are hit), 64 for the
-    other d_in = 4096 layers, 16 where d_in = 12288;
+    other d_in = 4096 layers, 128 where d_in = 12288.  (Why so many there: the iterates are stored in fp32,
+    which puts the correction W - W_hat' that reaches a rounding decision 2e-8 to 6e-8 of a grid step away
+    from the fp64 value.  Over 12288 entries and the ~50 iterations in which codes still move, about one
+    channel in thirty meets a decision closer to a tie than that, takes the other level, and from there
+    runs to a different, equally good end point that differs in ~1-2 % of that channel's codes.  The
+    layer-wide agreement this gives, ~99.95 %, is estimated to +-0.02 % from 128 channels, and to no
+    better than the bar's own margin from 16.)
   * properties that hold at any size: Q orthogonal and Q T Q^T = H~ for the one-time factorisation,
     grid feasibility, error ordering RTN > ADMM >= local search.
 The oracle receives the GPU's damped fp32 Hessian as its H and the GPU's fp32 grid (Delta, z0), so that
@@ -312,6 +318,11 @@ def _solve_and_compare_sampled_channels(spec, rows):
     cf = codes[rows].cpu().numpy()
     assert (ca == res.admm.codes).mean() >= CODE_AGREEMENT, (ca == res.admm.codes).mean()
     assert (cf == res.ls.codes).mean() >= CODE_AGREEMENT, (cf == res.ls.codes).mean()
+    # the differences sit in a few channels that took another branch at a near-tie; most channels agree entirely
+    assert (cf == res.ls.codes).all(axis=1).mean() >= 0.85
+    # the local search by itself: the oracle's search started from the GPU's ADMM codes ends where the GPU's did
+    ls_from_gpu = O.local_search(H, Wn, ca, grid[0], grid[1], spec.bits)
+    assert (cf == ls_from_gpu.codes).mean() >= 0.9999, (cf == ls_from_gpu.codes).mean()
     e_a = O.objective(H, Wn, O.dequantize(ca, res.admm.delta, res.admm.z0))
     e_f = O.objective(H, Wn, O.dequantize(cf, res.admm.delta, res.admm.z0))
     assert abs(e_a - res.err_admm) <= ERR_TOL * res.err_admm
@@ -370,10 +381,10 @@ def test_cfg5_down_proj_sampled_channels_against_oracle():
     eigendecomposition of the 12288 x 12288 matrix takes a few minutes of host time)."""
     spec = wl.config5(n_blocks=18)[7 * 17 + 6]
     assert spec.name == "cfg5_b17_down"
-    _solve_and_compare_sampled_channels(spec, spread_channels(spec.d_out, 16))
+    _solve_and_compare_sampled_channels(spec, spread_channels(spec.d_out, 128))
 
 
 def test_cfg3_down_proj_sampled_channels_against_oracle():
     """Config 3, down_proj: d_in = 12288, post-SiLU-like activations, W3 g128, T = 300."""
     spec = wl.config3()[2]
-    _solve_and_compare_sampled_channels(spec, spread_channels(spec.d_out, 16))
+    _solve_and_compare_sampled_channels(spec, spread_channels(spec.d_out, 128))
