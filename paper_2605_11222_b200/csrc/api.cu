@@ -543,7 +543,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.W0 = d_W0;
   e.V = c->V;
   e.codes = d_codes;
-  e.s = c->s64;
+  e.s = c->s;
   e.inv_s = c->inv_s;
   e.delta = d_scale;
   e.zero = d_zero;

@@ -766,9 +766,11 @@ void launch_error_planes(Ctx* c, const float* W0, int p, int gs, const unsigned 
 // ------------------------------------------------------------------------------------------------
 // (W~ - W_hat') / s of one element: the product's output plus its c R part (R rebuilt from the codes and the dual
 // as in the element update), plus V/rho.
-__device__ __forceinline__ double refresh_target(float zp, float w0, float v, int code_old, int first_iter, double s,
+__device__ __forceinline__ double refresh_target(float zp, float w0, float v, int code_old, int first_iter, float s,
                                                  float inv_s, float dl, float z0, float cshift, float inv_rho) {
-  const float e_old = first_iter ? 0.0f : (float)(s * fma((double)dl, (double)code_old, (double)z0 - (double)w0));
+  float a_hi, a_lo;
+  diff_exact(w0, z0, a_hi, a_lo);
+  const float e_old = first_iter ? 0.0f : grid_offset(s, dl, (float)code_old, a_hi, a_lo);
   const float z = fmaf(cshift, fmaf(-v, inv_rho, e_old), zp);
   return (double)(fmaf(v, inv_rho, z) * inv_s);           // the same fp32 steps as the element update
 }
@@ -776,7 +778,7 @@ __device__ __forceinline__ double refresh_target(float zp, float w0, float v, in
 __global__ void __launch_bounds__(256)
 refresh_eval_kernel(const float* __restrict__ Zc, const float* __restrict__ W0, const float* __restrict__ V,
                     const unsigned char* __restrict__ codes, int first_iter, const double* __restrict__ shift_c,
-                    const double* __restrict__ s, const float* __restrict__ inv_s, int p, int n, int gs, int kmax,
+                    const float* __restrict__ s, const float* __restrict__ inv_s, int p, int n, int gs, int kmax,
                     int symmetric, double inv_rho, const float* __restrict__ delta, const float* __restrict__ zero,
                     float* __restrict__ cand_delta, float* __restrict__ cand_zero, double* __restrict__ partial) {
   __shared__ double scratch[32];
@@ -817,7 +819,7 @@ refresh_eval_kernel(const float* __restrict__ Zc, const float* __restrict__ W0, 
     const double id0 = 1.0 / (double)d0, idn = 1.0 / (double)dn;
     double a = 0.0, b = 0.0;
     for (int i = lane; i < gs; i += 32) {
-      const double sv = s[gq * gs + i];
+      const double sv = (double)s[gq * gs + i];
       const double u = refresh_target(Zc[base + i], W0[base + i], V[base + i],
                                               first_iter ? 0 : (int)codes[base + i], first_iter, s[gq * gs + i],
                                               inv_s[gq * gs + i], d0, z0, cs, inv_rho_f);
@@ -924,9 +926,8 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
       const float4 z = *reinterpret_cast<const float4*>(P.C + base + i);
       const float4 wh = *reinterpret_cast<const float4*>(P.W0 + base + i);
       const float4 v = *reinterpret_cast<const float4*>(P.V + base + i);
-      const double2 s01 = *reinterpret_cast<const double2*>(P.s + i), s23 = *reinterpret_cast<const double2*>(P.s + i + 2);
+      const float4 sv = *reinterpret_cast<const float4*>(P.s + i);
       const float4 si = *reinterpret_cast<const float4*>(P.inv_s + i);
-      const struct { double x, y, z, w; } sv = {s01.x, s01.y, s23.x, s23.y};
       uchar4 k = make_uchar4(0, 0, 0, 0);
       if (!P.first_iter) k = *reinterpret_cast<const uchar4*>(P.codes + base + i);
       const int g0 = gsh >= 0 ? i >> gsh : i / gs;

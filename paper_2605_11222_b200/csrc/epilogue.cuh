@@ -21,7 +21,7 @@ struct EpiParams {
   const float* W0;          // W_hat, unscaled, as the caller passed it (ADMM element update)
   float* V;                 // dual V (in/out)
   unsigned char* codes;     // codes of D (in: D^(t), out: D^(t+1))
-  const double* s;          // [n] s_i = sqrt(H_ii), fp64
+  const float* s;           // [n] s_i = sqrt(H_ii)
   const float* inv_s;       // [n] 1 / s_i, fp32
   const float* delta;       // [p][n_groups]
   const float* zero;        // [p][n_groups]
@@ -48,54 +48,79 @@ __device__ __forceinline__ float epi_row_factor(const EpiParams& P, int row) {
   return f;
 }
 
-// One element of the ADMM update (Eq. 8-10).  z = [Q (T/rho + I)^{-1} Q^T R]_{ji} is the product's output, so
-// that W = W_hat' + z is the W-update of Eq. 7 written for the error W - W_hat'.
+// One element of the ADMM update (Eq. 8-10).  zp is the product's output, z = zp + c R the W-update of Eq. 7
+// written for the error W - W_hat'.
 //
 // Every quantity here is kept RELATIVE to the pre-trained weight, i.e. at the size of a grid step, never at
 // the size of the weight itself: in unscaled coordinates the projection target is
 //     Sigma W~ = w_hat + (z + V/rho) / s,
 // so the code is k = rint(((w_hat - z0) + (z + V/rho)/s) / Delta), and the grid point enters only through its
-// distance from the weight, D - W_hat' = s (z0 + Delta k - w_hat).  The two places where numbers of the
-// weight's size meet -- (w_hat - z0) and (Delta k - (w_hat - z0)) -- are evaluated in fp64, where both are
-// exact; the rounding decision of Eq. 10 is taken in fp64 like the oracle's.  (In plain fp32 the sums
-// W_hat' + z, s (z0 + Delta k) and y - z0 each round at the weight's magnitude, up to 2^(bits-1) grid steps:
-// ~1e-6 of a step per iteration at 4 bits, which is what decided most of the codes that differed from an
-// fp64 run.)
+// distance from the weight, D - W_hat' = s (z0 + Delta k - w_hat).  (In plain fp32 the sums W_hat' + z,
+// s (z0 + Delta k) and y - z0 each round at the weight's magnitude, up to 2^(bits-1) grid steps: ~1e-6 of a
+// step per iteration at 4 bits, which decided most of the codes that differed from an fp64 run.)
+//
+// The two places where numbers of the weight's size meet are evaluated without rounding, in fp32:
+//   a = w_hat - z0 as the unevaluated sum a_hi + a_lo of an error-free subtraction;
+//   Delta k as p + pe with p = fl(Delta k) and pe = fma(Delta, k, -p), so that Delta k - a comes out with the
+//   relative accuracy of a grid-step-sized number.
+// The rounding decision itself is first taken on the fp32 value of (a + u) / Delta, which is good to ~1e-6 of a
+// step; only when that lands within ROUND_MARGIN of a half-integer is it retaken in fp64 from the same fp32
+// inputs, like the oracle's.  (An all-fp64 element update was measured: row pass 113 us instead of 72 us, the
+// conversions between the two formats being the cost, and no fewer differing codes.)
 struct AdmmElem {
   unsigned char code;
   float v_new, r_next, dr2, ds2;
 };
-// Constants of one (channel, group): Delta, z0 and 1 / Delta in fp64.
+// Constants of one (channel, group): Delta, z0 and 1 / Delta.
 struct GridG {
-  float dl, z0;
-  double inv_dl;
+  float dl, z0, inv_dl;
 };
 __device__ __forceinline__ GridG grid_g(float dl, float z0) {
   GridG g;
   g.dl = dl;
   g.z0 = z0;
-  g.inv_dl = 1.0 / (double)dl;
+  g.inv_dl = __frcp_rn(dl);
   return g;
 }
+constexpr float ROUND_MARGIN = 1e-4f;
+
+// w_hat - z0 = hi + lo exactly (branch-free two-sum).  The intrinsics keep the compiler from contracting or
+// reordering the steps: each must round exactly once, as written.
+__device__ __forceinline__ void diff_exact(float w0, float z0, float& hi, float& lo) {
+  hi = __fsub_rn(w0, z0);
+  const float bb = __fsub_rn(hi, w0);
+  lo = __fsub_rn(__fsub_rn(w0, __fsub_rn(hi, bb)), __fadd_rn(z0, bb));
+}
+// s (Delta k - a) for a = a_hi + a_lo: the distance of grid point k from the weight, scaled coordinates.
+__device__ __forceinline__ float grid_offset(float s, float dl, float k, float a_hi, float a_lo) {
+  const float p = __fmul_rn(dl, k);
+  const float pe = __fmaf_rn(dl, k, -p);                  // Delta k = p + pe exactly
+  return s * __fsub_rn(__fadd_rn(__fsub_rn(p, a_hi), pe), a_lo);
+}
+
 // g: the grid the new code is taken on; g_old: the grid code_old refers to (the same one, except in the
-// iteration that accepts a grid refresh).  fp64 is used where numbers of the weight's size meet and for the
-// rounding decision; the grid-step-sized quantities around them (z, V/rho, the residuals) are fp32, which is the
-// precision they are stored in anyway (measured on the 12288-wide layers: the correction W - W_hat' reaches the
-// decision with an error of 2e-8 to 6e-8 of a grid step rms, the rounding of its own fp32 storage).
-__device__ __forceinline__ AdmmElem admm_elem(float zp, float w0, float v, int code_old, double s, float inv_s,
+// iteration that accepts a grid refresh).
+__device__ __forceinline__ AdmmElem admm_elem(float zp, float w0, float v, int code_old, float s, float inv_s,
                                               const GridG& g, const GridG& g_old, float cshift, const EpiParams& P) {
   AdmmElem o;
-  const double a = (double)w0 - (double)g.z0;              // w_hat - z0, exact
-  const float e_old = P.first_iter ? 0.0f                  // D^(0) = W_hat'
-                                   : (float)(s * fma((double)g_old.dl, (double)code_old,
-                                                     (double)g_old.z0 - (double)w0));
+  float a_hi, a_lo;
+  diff_exact(w0, g.z0, a_hi, a_lo);
+  float e_old = 0.0f;                                      // D^(0) = W_hat'
+  if (!P.first_iter) {
+    float b_hi = a_hi, b_lo = a_lo;
+    if (g_old.z0 != g.z0) diff_exact(w0, g_old.z0, b_hi, b_lo);
+    e_old = grid_offset(s, g_old.dl, (float)code_old, b_hi, b_lo);
+  }
   const float inv_rho = (float)P.inv_rho;
   // z = c R + (product output), R = D^(t) - V/rho - W_hat' exactly as the right-hand side was formed
   const float z = fmaf(cshift, fmaf(-v, inv_rho, e_old), zp);
   const float u = fmaf(v, inv_rho, z) * inv_s;             // (W~ - W_hat') / s: target minus weight  (Eq. 8)
-  double k = rint((a + (double)u) * g.inv_dl);             // nearest level, ties to even    (Eq. 10)
-  k = fmin(fmax(k, 0.0), (double)P.kmax);
-  const float e_new = (float)(s * fma((double)g.dl, k, -a));               // D^(t+1) - W_hat'
+  const float x = __fadd_rn(__fadd_rn(a_hi, u), a_lo) * g.inv_dl;   // (Sigma W~ - z0) / Delta, good to ~1e-6
+  float k = rintf(x);                                      // nearest level, ties to even    (Eq. 10)
+  if (fabsf(fabsf(x - k) - 0.5f) < ROUND_MARGIN)           // too close to a tie for fp32: decide in fp64
+    k = (float)rint((((double)w0 - (double)g.z0) + (double)u) / (double)g.dl);
+  k = fminf(fmaxf(k, 0.0f), (float)P.kmax);
+  const float e_new = grid_offset(s, g.dl, k, a_hi, a_lo); // D^(t+1) - W_hat'
   const float wd = z - e_new;                              // W^(t+1) - D^(t+1)
   const float dd = e_new - e_old;                          // D^(t+1) - D^(t)
   o.code = (unsigned char)(int)k;

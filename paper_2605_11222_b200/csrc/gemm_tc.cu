@@ -236,13 +236,13 @@ __device__ __forceinline__ void epi_elem4(const EpiParams& P, int row, int col, 
     const long long o = (long long)row * N + col;
     const float4 w = *reinterpret_cast<const float4*>(P.W0 + o);
     const float4 v = *reinterpret_cast<const float4*>(P.V + o);
-    const double2 sa = *reinterpret_cast<const double2*>(P.s + col), sb = *reinterpret_cast<const double2*>(P.s + col + 2);
+    const float4 s = *reinterpret_cast<const float4*>(P.s + col);
     const float4 is = *reinterpret_cast<const float4*>(P.inv_s + col);
     uint32_t codes = 0u;
     if (!P.first_iter) codes = *reinterpret_cast<const uint32_t*>(P.codes + o);
     const float wh[4] = {w.x, w.y, w.z, w.w};
     const float vv[4] = {v.x, v.y, v.z, v.w};
-    const double ss[4] = {sa.x, sa.y, sb.x, sb.y};
+    const float ss[4] = {s.x, s.y, s.z, s.w};
     const float si[4] = {is.x, is.y, is.z, is.w};
     const bool one_group = (P.group_size & 3) == 0;        // then the 4 columns share (Delta, z0)
     const float cshift = (float)P.shift_c[0];
