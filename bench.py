@@ -400,6 +400,9 @@ def main():
     ap.add_argument("--workload", default="cfg2", help="cfg1 | cfg2 | cfg3_gate | cfg3_up | cfg3_down | "
                     "cfg4_k | cfg4_v | cfg4_o | cfg5_<q|k|v|o|gate|up|down>  (default: the metric's own, cfg2)")
     ap.add_argument("--iters", type=int, default=0, help="ADMM iterations T (0: the workload's own, 300)")
+    ap.add_argument("--rho0", type=float, default=0.0,
+                    help="first penalty of the geometric schedule (0: the workload's own, 0.1); a large value makes "
+                         "a short run consist of late iterations, e.g. to profile their one-plane products")
     ap.add_argument("--stack-blocks", type=int, default=0,
                     help="instead of one layer: quantize the first B decoder blocks of config 5 (7 layers each, "
                          "36 = the whole stack), every layer once, and report the wall time")
@@ -429,6 +432,8 @@ def main():
         base = dataclasses.replace(base, n_tokens=args.tokens)
     if args.iters > 0:
         base = dataclasses.replace(base, T=args.iters)
+    if args.rho0 > 0:
+        base = dataclasses.replace(base, rho0=args.rho0)
 
     if args.impl == "reference":
         return run_reference(args, base, wl)

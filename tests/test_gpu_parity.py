@@ -395,6 +395,18 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable():
     assert (codes.cpu().numpy() == res.ls.codes).mean() >= CODE_AGREEMENT
     with pytest.raises(B.AdmmqError):
         sol.test_set_wait(10)                                     # bounds below 1000 cycles are refused
+    # the same for the one-plane products of large penalties (another instantiation of the kernel)
+    sol.factor(rho=[1e7, 2e7, 4e7])
+    sol.test_set_wait(2_000_000, hold_loads=True)
+    with pytest.raises(B.AdmmqError) as e:
+        sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric)
+    assert e.value.status == B.ERR_TIMEOUT
+    torch.cuda.synchronize()
+    sol.test_set_wait()
+    c3, _, _, rep3 = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric)
+    assert sol.last_device_status() == B.OK and rep3.one_plane_iters >= 2
+    ref3 = O.admm(H, Wn, spec.bits, spec.group_size, spec.symmetric, np.array([1e7, 2e7, 4e7]))
+    assert (c3.cpu().numpy() == ref3.codes).mean() >= CODE_AGREEMENT
 
 
 # ------------------------------------------------------------------ pair-swap refinement (Sec. 3.5, Eq. 11 in full)
