@@ -602,6 +602,283 @@ gemm_tc_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_
   }
 }
 
+// ------------------------------------------------------------------ one-plane products on CTA pairs
+// The W-update products of the late iterations run on one fp16 plane per operand: one MMA per K step, so a
+// 128 x 256 tile asks its SM for 48 KB of operands per 512 tensor-core cycles, more than the shared memory of one
+// SM can keep in flight against the latency of L2 (measured: 57-60 % of the tensor peak).  Here two SMs work as a
+// pair (a cluster of two CTAs, tcgen05.mma.cta_group::2) on a 256 x 256 tile: each CTA stages its own 128 rows of
+// A and 128 of the 256 rows of B, 32 KB per K block, and the tensor cores of both read B from both shared
+// memories.  The result of such a product need not be better than the 2^-12 of its operands, so the whole K range
+// accumulates in tensor memory (one of two 256-column buffers per tile) and the workers take it once per tile,
+// while the issuer already works on the next tile in the other buffer.
+//   warp 0       TMA producer in both CTAs; the bytes of both are counted by the leader's (rank 0) mbarriers, which
+//                the leader's producer alone arms;
+//   warp 1       MMA issuer in the leader only: tcgen05.mma M = 256 and tcgen05.commit, which arrives on the
+//                barriers of both CTAs;
+//   warps 2-17   workers in both CTAs, each CTA on its own 128 rows: tensor memory -> registers -> staging buffer ->
+//                coalesced stores, then an arrival on the leader's "buffer free" barrier.
+// No multicast load anywhere: every CTA fetches its own tiles.  Waits are bounded as in the single-CTA kernel;
+// both CTAs always reach the cluster barrier at the end, so an expired wait in one cannot strand the other.
+constexpr int PAIR_M = 2 * BM;
+constexpr int PAIR_BOX = 64;             // rows of B per TMA box (a CTA takes two per tile, one per half tile)
+constexpr int PAIR_STAGES = 6;
+constexpr int PAIR_A_BYTES = BM * BK * 2, PAIR_B_BYTES = (BN / 2) * BK * 2;
+constexpr int PAIR_STAGE_BYTES = PAIR_A_BYTES + PAIR_B_BYTES;   // 32 KB
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster (shared::cluster window).
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrivals on a barrier that may live in the other CTA of the pair (cluster addresses).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+// Tile load of one CTA of a pair into its own shared memory; the completion bytes go to `cluster_bar`, the
+// leader's barrier.  (A plain load: no multicast.)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar,
+                                                 int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(x), "r"(y)
+      : "memory");
+}
+// Arrives, once the MMAs issued so far are complete, on the barrier at this offset in both CTAs of the pair.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile(
+      "{\n.reg .b16 m;\nmov.b16 m, 3;\n"
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n}"
+      ::"r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__host__ __device__ constexpr uint32_t idesc_m256(uint32_t fmt, uint32_t n_cols) {
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((n_cols >> 3) << 17) | ((uint32_t)(PAIR_M >> 4) << 24);
+}
+
+// Work units of a pair: whole 256 x 256 tiles, except that the tiles of a last wave that would fill at most half
+// of the pairs are cut into two 256 x 128 units.
+__device__ __forceinline__ Schedule make_pair_schedule(int M, int N, int pairs) {
+  Schedule s;
+  s.tiles_m = (M + PAIR_M - 1) / PAIR_M;
+  s.tiles_n = (N + BN - 1) / BN;
+  const int tiles = s.tiles_m * s.tiles_n;
+  const int waves = tiles / pairs, rem = tiles - waves * pairs;
+  const bool split = rem > 0 && 2 * rem <= pairs;
+  s.full_units = split ? waves * pairs : tiles;
+  s.num_units = split ? waves * pairs + 2 * rem : tiles;
+  return s;
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc_pair_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_t fmt, EpiParams epi,
+                    int* status, long long wait_limit, int hold_loads) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * PAIR_STAGES + 2 * NPART + 1];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  __shared__ uint32_t fill_state[2];       // producer's record for the abort path: armed stages / their parities
+  __shared__ __align__(16) float stage_all[WORKER_WARPS * STAGE_FLOATS];
+
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &abort_flag_s;
+  const uint32_t rank = cluster_ctarank();                 // 0: leader of the pair
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+
+  const uint32_t full0 = smem_u32(&bars[0]);
+  const uint32_t empty0 = smem_u32(&bars[PAIR_STAGES]);
+  const uint32_t pfull0 = smem_u32(&bars[2 * PAIR_STAGES]);
+  const uint32_t pempty0 = smem_u32(&bars[2 * PAIR_STAGES + NPART]);
+  const uint32_t drain_bar = smem_u32(&bars[2 * PAIR_STAGES + 2 * NPART]);
+
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    fill_state[0] = fill_state[1] = 0u;
+    mbar_init(drain_bar, 1);
+    for (int s = 0; s < PAIR_STAGES; ++s) {
+      mbar_init(full0 + 8 * s, 1);                         // the leader's producer arrives, expecting the bytes of both
+      mbar_init(empty0 + 8 * s, 1);
+    }
+    for (int a = 0; a < NPART; ++a) {
+      mbar_init(pfull0 + 8 * a, 1);
+      mbar_init(pempty0 + 8 * a, 2 * WORKER_WARPS);        // the workers of both CTAs (the leader's is used)
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(
+                     smem_u32(&tmem_base_slot))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                      // the peer's barriers exist before any remote arrival
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  const Schedule sched = make_pair_schedule(M, N, num_pairs);
+  const int num_kb = (K + BK - 1) / BK;
+
+  if (warp == 0) {
+    // ===================== TMA producer (both CTAs) =====================
+    if (lane == 0 && !hold_loads) {
+      int stage = 0;
+      uint32_t phase = 0, armed = 0u, par = 0u;
+      bool ok = true;
+      for (int u = pair; u < sched.num_units && ok; u += num_pairs) {
+        const Unit un = unit_of(sched, u);
+        const int half_cols = un.ncols / 2;                // B rows staged by this CTA
+        const int boxes = half_cols / PAIR_BOX;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          ok = mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag, status, wait_limit);
+          if (!ok) break;
+          const uint32_t sbase = tiles_base + stage * PAIR_STAGE_BYTES;
+          const uint32_t fb = map_to_cta(full0 + 8 * stage, 0);           // the leader's barrier
+          // The leader expects the bytes of both CTAs (each loads the same amount) with a local arrival; the peer
+          // only issues its loads, whose completion bytes go to the leader's barrier.  (An arrival of the peer on
+          // the leader's barrier for every stage, with cluster-scope release, was measured: it held the producer
+          // ~1500 cycles per K block and the tensor pipe at 28 %.)
+          if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * (PAIR_A_BYTES + boxes * PAIR_BOX * BK * 2));
+          armed |= 1u << stage;
+          par = (par & ~(1u << stage)) | (phase << stage);
+          tma_load_2d_pair(sbase, &maps.a[0], fb, kb * BK, un.tm * PAIR_M + (int)rank * BM);
+          for (int bx = 0; bx < boxes; ++bx)
+            tma_load_2d_pair(sbase + PAIR_A_BYTES + bx * PAIR_BOX * BK * 2, &maps.b[0], fb, kb * BK,
+                             un.col0 + (int)rank * half_cols + bx * PAIR_BOX);
+          if (++stage == PAIR_STAGES) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+      }
+      fill_state[0] = armed;
+      fill_state[1] = par;
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer (leader CTA) =====================
+    if (lane == 0 && rank == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t g = 0;                        // unit counter, shared sequence with the workers
+      bool ok = true;
+      for (int u = pair; u < sched.num_units && ok; u += num_pairs) {
+        const Unit un = unit_of(sched, u);
+        const uint32_t idesc = idesc_m256(fmt, (uint32_t)un.ncols);
+        const int pb = (int)(g % NPART);
+        ok = mbar_wait(pempty0 + 8 * pb, ((g / NPART) & 1u) ^ 1u, abort_flag, status, wait_limit);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)pb * BN;
+        uint32_t accumulate = 0;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          ok = mbar_wait(full0 + 8 * stage, phase, abort_flag, status, wait_limit);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sbase = tiles_base + stage * PAIR_STAGE_BYTES;
+          const uint64_t a_desc = make_kmajor_sw128_desc(sbase);
+          const uint64_t b_desc = make_kmajor_sw128_desc(sbase + PAIR_A_BYTES);
+#pragma unroll
+          for (int k16 = 0; k16 < BK / 16; ++k16) {
+            const uint64_t koff = (uint64_t)((k16 * 32) >> 4);   // 16 elements = 32 bytes along K
+            tc_mma_f16_pair(d_tmem, a_desc + koff, b_desc + koff, idesc, accumulate);
+            accumulate = 1;
+          }
+          tc_commit_pair(empty0 + 8 * stage);   // stage reusable in both CTAs once these MMAs have read it
+          if (++stage == PAIR_STAGES) {
+            stage = 0;
+            phase ^= 1u;
+          }
+        }
+        if (!ok) break;
+        tc_commit_pair(pfull0 + 8 * pb);        // the tile is complete in both CTAs
+        ++g;
+      }
+    }
+  } else {
+    // ===================== workers (both CTAs) =====================
+    const int q = warp & 3;                                // tensor-memory lane quarter this warp may read
+    const int cq = (warp - 2) >> 2;                        // which 64 of the 256 columns
+    float r2 = 0.f, s2 = 0.f;
+    uint32_t g = 0;
+    bool ok = true;
+    const uint32_t pempty_leader = map_to_cta(pempty0, 0);
+    for (int u = pair; u < sched.num_units && ok; u += num_pairs) {
+      const Unit un = unit_of(sched, u);
+      const bool mine = cq * COLS_PER_THREAD < un.ncols;   // a half unit has columns for cq = 0, 1 only
+      const int row0 = un.tm * PAIR_M + (int)rank * BM + q * 32, col0 = un.col0 + cq * COLS_PER_THREAD;
+      const int pb = (int)(g % NPART);
+      ok = mbar_wait_warp(pfull0 + 8 * pb, (g / NPART) & 1u, abort_flag, status, wait_limit);
+      if (!ok) break;
+      tc_fence_after();
+      float sums[COLS_PER_THREAD];
+      if (mine) {
+        const uint32_t taddr = tmem_base + (uint32_t)pb * BN + (uint32_t)(cq * COLS_PER_THREAD) +
+                               ((uint32_t)(q * 32) << 16);
+#pragma unroll
+        for (int h = 0; h < COLS_PER_THREAD / 8; ++h) {
+          uint32_t v[8];
+          tc_ld8_issue(taddr + 8 * h, v);
+          tc_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 8; ++e) sums[8 * h + e] = __uint_as_float(v[e]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(pempty_leader + 8 * pb);   // in registers: the buffer is free
+      ++g;
+      if (mine)
+        epilogue_block<EPI_STORE>(epi, row0, col0, M, N, sums, stage_all + (warp - 2) * STAGE_FLOATS, lane, r2, s2);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag_s) {
+    // as in the single-CTA kernel: the fills this CTA armed must have landed (they are counted on the leader's
+    // barriers, which the leader waits for, the peer being held at the cluster barrier below meanwhile), and the
+    // MMAs issued must have completed, before shared and tensor memory are given back
+    if (threadIdx.x == 0 && rank == 0) {
+      const uint32_t armed = fill_state[0], par = fill_state[1];
+      for (int s = 0; s < PAIR_STAGES; ++s)
+        if (armed >> s & 1u) mbar_wait_quiet(full0 + 8 * s, par >> s & 1u);
+    }
+    if (threadIdx.x == 32 && rank == 0) {
+      tc_commit_pair(drain_bar);             // (every tcgen05 instruction of a kernel names the same CTA group)
+      mbar_wait_quiet(drain_bar, 0u);
+    }
+    if (threadIdx.x == 64) {                 // loads of this CTA that the leader never armed a barrier for: let them land
+      const long long t0 = clock64();
+      while (clock64() - t0 < 100000LL) {
+      }
+    }
+    __syncthreads();
+  }
+  cluster_sync_all();                        // both CTAs are done with tensor memory and with remote arrivals
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+  }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -654,6 +931,54 @@ static cudaError_t launch_tc(Ctx* c, const TcMaps& maps, int M, int N, int K, ui
   return cudaGetLastError();
 }
 
+// Row-major 16-bit plane -> tensor map with the given box height (defined below).
+static bool encode_plane(CUtensorMap* map, const bf16* ptr, long long rows, long long cols, long long ld,
+                         int box_rows, int f16);
+
+static cudaError_t launch_tc_pair(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiParams& epi) {
+  TcMaps maps;
+  if (!encode_plane(&maps.a[0], A.hi, M, K, A.ld, BM, A.f16) ||
+      !encode_plane(&maps.b[0], B.hi, N, K, B.ld, PAIR_BOX, B.f16))
+    return cudaErrorInvalidValue;
+  maps.a[1] = maps.a[0];
+  maps.b[1] = maps.b[0];
+  const size_t smem = (size_t)PAIR_STAGES * PAIR_STAGE_BYTES + 1024;
+  const cudaError_t ea = ensure_dynamic_smem((const void*)gemm_tc_pair_kernel, (int)smem);
+  if (ea != cudaSuccess) return ea;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * (c->num_sms / 2));
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  // pairs that can be resident at once: a persistent kernel must not launch more, or the surplus would run after
+  // the others (asked once per context, which belongs to one device)
+  if (c->pair_clusters == 0) {
+    int nc = 0;
+    if (cudaOccupancyMaxActiveClusters(&nc, gemm_tc_pair_kernel, &cfg) != cudaSuccess || nc < 1) {
+      c->pair_clusters = -1;
+      cudaGetLastError();
+    } else {
+      c->pair_clusters = nc < c->num_sms / 2 ? nc : c->num_sms / 2;
+    }
+  }
+  if (c->pair_clusters < 1) return cudaErrorNotSupported;
+  const int tiles = ((M + PAIR_M - 1) / PAIR_M) * ((N + BN - 1) / BN);
+  const int pairs = tiles < c->pair_clusters ? tiles : c->pair_clusters;
+  cfg.gridDim = dim3(2 * pairs);
+  const uint32_t fmt = A.f16 ? 0u : 1u;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel, maps, M, N, K, fmt, epi, c->status,
+                                     c->wait_limit_cycles, c->hold_loads);
+  c->launches++;
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 cudaError_t gemm_tc(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiParams& epi_in) {
   const int na = A.lo ? 2 : 1, nb = B.lo ? 2 : 1;
   if (na != nb || A.f16 != B.f16) return cudaErrorInvalidValue;   // one MMA takes A and B of one type
@@ -671,6 +996,11 @@ cudaError_t gemm_tc(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiPa
   epi.a_inv = A.all_inv;
   epi.b_inv = B.all_inv;
   const uint32_t idesc = A.f16 ? 0u : 1u;                  // operand format: 0 = fp16, 1 = bf16
+  // one fp16 plane and a plain store, large enough for 256 x 256 tiles: the CTA-pair kernel
+  if (na == 1 && A.f16 && epi.kind == EPI_STORE && c->use_pair_kernel && M >= PAIR_M && N >= BN && c->num_sms >= 2) {
+    const cudaError_t ep = launch_tc_pair(c, A, B, M, N, K, epi);
+    if (ep != cudaErrorNotSupported) return ep;           // no room for a pair on this device: single-CTA kernel
+  }
   if (na == 1) {
     if (epi.kind == EPI_ACCUM) return launch_tc<1, EPI_ACCUM>(c, maps, M, N, K, idesc, epi);
     // one fp16 plane and a plain store: a W-update product of the late iterations, whose result need not be better

@@ -40,6 +40,8 @@ struct Ctx {
   double mu_host = 1.0, lam_lo = 0.0, lam_hi = 0.0;   // mean and Gershgorin bounds of the spectrum of H~ (host copies)
   long long launches = 0;
   long long wait_limit_cycles = 2000000000LL;   // bound of every device-side wait, about a second
+  int pair_clusters = 0;
+  int use_pair_kernel = 1;
   int one_plane_flush_kb = 1 << 20;   // K blocks per flush of the one-plane fp16 products (whole K by default)
   int hold_loads = 0;           // failure-handling tests only: the product kernel's producer issues no loads
   // ---- workspace carve-up (device) ----
