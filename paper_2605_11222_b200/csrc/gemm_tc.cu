@@ -761,9 +761,9 @@ gemm_tc_pair_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, ui
           armed |= 1u << stage;
           par = (par & ~(1u << stage)) | (phase << stage);
           tma_load_2d_pair(sbase, &maps.a[0], fb, kb * BK, un.tm * PAIR_M + (int)rank * BM);
-          for (int bx = 0; bx < boxes; ++bx)
-            tma_load_2d_pair(sbase + PAIR_A_BYTES + bx * PAIR_BOX * BK * 2, &maps.b[0], fb, kb * BK,
-                             un.col0 + (int)rank * half_cols + bx * PAIR_BOX);
+          // this CTA's half of B: one box of 128 rows for a whole tile (map b[1]), one of 64 for a half tile (b[0])
+          tma_load_2d_pair(sbase + PAIR_A_BYTES, boxes == 2 ? &maps.b[1] : &maps.b[0], fb, kb * BK,
+                           un.col0 + (int)rank * half_cols);
           if (++stage == PAIR_STAGES) {
             stage = 0;
             phase ^= 1u;
@@ -938,10 +938,10 @@ static bool encode_plane(CUtensorMap* map, const bf16* ptr, long long rows, long
 static cudaError_t launch_tc_pair(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiParams& epi) {
   TcMaps maps;
   if (!encode_plane(&maps.a[0], A.hi, M, K, A.ld, BM, A.f16) ||
-      !encode_plane(&maps.b[0], B.hi, N, K, B.ld, PAIR_BOX, B.f16))
+      !encode_plane(&maps.b[0], B.hi, N, K, B.ld, PAIR_BOX, B.f16) ||
+      !encode_plane(&maps.b[1], B.hi, N, K, B.ld, 2 * PAIR_BOX, B.f16))
     return cudaErrorInvalidValue;
   maps.a[1] = maps.a[0];
-  maps.b[1] = maps.b[0];
   const size_t smem = (size_t)PAIR_STAGES * PAIR_STAGE_BYTES + 1024;
   const cudaError_t ea = ensure_dynamic_smem((const void*)gemm_tc_pair_kernel, (int)smem);
   if (ea != cudaSuccess) return ea;
