@@ -646,16 +646,20 @@ def main():
         return {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": gbs / peaks["hbm_gbs"], "launches": cnt, "avg_launch_ms": ms / cnt}
 
+    # solve: read Y fp32, write two fp16 planes, for d_out rows (the n rows of the operator on the explicit route).
+    # row pass: reads z 4, w 4, V 4, codes 1; writes V 4, codes 1, two fp16 planes 4 bytes per element; on the
+    # explicit route the same timer also takes the split of the n x n operator (maximum pass 4, split 4 + 4 bytes
+    # per element), so a launch there is the mean of the two.
     kernel_rooflines = {
-        "tridiag_solve": _hbm("tridiag_solve", 8.0 * p * n),          # read Y fp32, write two fp16 planes
-        # row pass: reads z 4, w_hat 4, V 4, codes 1; writes V 4, codes 1, two fp16 planes 4 bytes per element
-        "row_split": _hbm("row_split", 22.0 * p * n),
+        "tridiag_solve": _hbm("tridiag_solve", 8.0 * rows_p1 * n),
+        "row_split": _hbm("row_split", (22.0 * p * n + 12.0 * n * n) / 2 if explicit_route else 22.0 * p * n),
         "transpose": _hbm("transpose", 2.0 * x_bytes * chunk_rows * n),
     }
     if n_1p:
         tf1 = flops_one_plane / (ms_1p * 1e-3) / 1e12
         kernel_rooflines["wupdate_one_plane"] = {
-            "kernel": "gemm_tc_kernel<1,STORE> (W-update products of the late iterations: one fp16 plane)",
+            "kernel": "gemm_tc_pair_kernel (W-update products of the late iterations: one fp16 plane, CTA pairs; "
+                      "gemm_tc_kernel<1,STORE> where a product is narrower than 256)",
             "bound": "tensor", "achieved": tf1, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
             "frac": tf1 / peaks["bf16_sustained"], "launches": n_1p, "avg_launch_ms": ms_1p / n_1p}
     ms_h, n_h = timing["hessian_product"]
