@@ -537,10 +537,20 @@ def main():
     c_two = codes.clone()
     _, _, _, df_rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, codes=codes, scale=scale,
                                          zero=zero, resid=resid)
-    planes_variant = {"two_planes_always_ms": tp_rep.ms, "default_ms": df_rep.ms,
+    c_def = codes.clone()
+    # ... and with the late iterations through the factorisation (one-plane products + solve) instead of the series
+    _, _, _, ns_rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, codes=codes, scale=scale,
+                                         zero=zero, resid=resid, wupdate_series=1)
+    planes_variant = {"two_planes_always_ms": tp_rep.ms, "one_plane_without_series_ms": ns_rep.ms,
+                      "default_ms": df_rep.ms,
                       "default_one_plane_iterations": df_rep.one_plane_iters,
-                      "err_admm_two_planes": tp_rep.err_before, "err_admm_default": df_rep.err_before,
-                      "codes_equal_fraction": float((c_two == codes).float().mean().item())}
+                      "default_series_iterations": df_rep.series_iters,
+                      "err_admm_two_planes": tp_rep.err_before, "err_admm_without_series": ns_rep.err_before,
+                      "err_admm_default": df_rep.err_before,
+                      "codes_equal_fraction": float((c_two == c_def).float().mean().item()),
+                      "codes_equal_fraction_without_series": float((codes == c_def).float().mean().item())}
+    n_series = int(df_rep.series_iters)
+    n_one_plane = int(df_rep.one_plane_iters)
 
     # ---- a run whose grid comes from the MSE search for the clipping ratio, 100 candidates down to 0.8
     #      (another widened row: measured, not part of `value`), followed by the local search ----
@@ -627,8 +637,9 @@ def main():
                 "flops_per_full_launch": flops_launch,
                 "product1_launch_ms": ms_p1 / max(1, n_p1), "product2_launch_ms": ms_p2 / max(1, n_p2)}
     w_update_ms = (ms_p1 + ms_p2 + ms_1p + timing["tridiag_solve"][0] + timing["row_split"][0]) / args.steps
-    # one-plane launches: both products of an iteration, so half of them have rows_p1 rows
-    flops_one_plane = 2.0 * n * n * (rows_p1 + p) * (n_1p / 2.0)
+    # one-plane launches: one product R (mu I - H~) per iteration of the truncated series, else both products of an
+    # iteration, of which the first has rows_p1 rows
+    flops_one_plane = args.steps * 2.0 * n * n * (n_series * p + (n_one_plane - n_series) * (rows_p1 + p))
     executed_flops_per_step = (flops_two_plane + flops_one_plane) / args.steps
     breakdown = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
                  for k, v in timing.items()}
@@ -658,8 +669,9 @@ def main():
     if n_1p:
         tf1 = flops_one_plane / (ms_1p * 1e-3) / 1e12
         kernel_rooflines["wupdate_one_plane"] = {
-            "kernel": "gemm_tc_pair_kernel (W-update products of the late iterations: one fp16 plane, CTA pairs; "
-                      "gemm_tc_kernel<1,STORE> where a product is narrower than 256)",
+            "kernel": "gemm_tc_pair_kernel (W-update products of the late iterations: one fp16 plane, CTA pairs, one "
+                      "product per iteration of the truncated series; gemm_tc_kernel<1,STORE> where a product is "
+                      "narrower than 256)",
             "bound": "tensor", "achieved": tf1, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
             "frac": tf1 / peaks["bf16_sustained"], "launches": n_1p, "avg_launch_ms": ms_1p / n_1p}
     ms_h, n_h = timing["hessian_product"]
@@ -683,7 +695,7 @@ def main():
         "layers_per_s": world / (ms_step / 1e3),
         "w_update_useful_tflops": 4.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
         "w_update_executed_tflops": executed_flops_per_step / (w_update_ms * 1e-3) / 1e12,
-        "one_plane_iterations": int(n_1p / (2 * args.steps)), "w_update_route": "explicit operator" if explicit_route else "two products",
+        "one_plane_iterations": n_one_plane, "series_iterations": n_series, "w_update_route": "explicit operator" if explicit_route else "two products",
         "err_before_local_search": rep.err_before, "err_after_local_search": rep.err_after,
         "local_search_moves": rep.moves, "pair_swap_after_local_search": pair_swap, "admm_with_grid_refresh": grid_refresh,
         "admm_with_mse_clip_search": mse_clip, "admm_with_fused_epilogue": fused_variant,

@@ -1,5 +1,5 @@
 /*
- * admmq_testing.h -- hooks for tests of the library's failure handling.  Not part of the solver's
+ * admmq_testing.h -- hooks for tests of the library's failure handling and accuracy.  Not part of the solver's
  * contract: nothing here is needed to quantize a layer, and the paper has no counterpart.
  */
 #ifndef ADMMQ_TESTING_H_
@@ -29,6 +29,13 @@ admmq_status admmq_test_set_wait(admmq_ctx* ctx, long long wait_limit_cycles, in
 admmq_status admmq_test_w_update_correction(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
                                             const unsigned char* d_codes, const float* d_scale,
                                             const float* d_zero, const float* d_V, double rho, float* d_Z_out);
+
+/* The same correction evaluated as the late iterations do it (admmq_quant_cfg.wupdate_series): c R + c R E with
+ * the fixed one-plane operand mu I - H~, whatever gamma(rho) is.  For a test that compares it with the route
+ * through the factorisation at a penalty where the solver would switch to it. */
+admmq_status admmq_test_w_update_series(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
+                                        const unsigned char* d_codes, const float* d_scale,
+                                        const float* d_zero, const float* d_V, double rho, float* d_Z_out);
 
 #ifdef __cplusplus
 }

@@ -29,6 +29,7 @@ EXPORTS = [
     "admmq_launch_count", "admmq_set_timing", "admmq_reset_timing", "admmq_get_timing",
     "admmq_objective_static", "admmq_get_factor", "admmq_pair_swap", "admmq_test_set_wait",
     "admmq_hessian_export", "admmq_hessian_import", "admmq_test_w_update_correction",
+    "admmq_test_w_update_series",
 ]
 T_HESSIAN_PRODUCT, T_TRANSPOSE, T_FACTOR, T_WUPDATE_PRODUCT1, T_TRIDIAG_SOLVE, T_WUPDATE_PRODUCT2, \
     T_GRADIENT_PRODUCT, T_LOCAL_SEARCH, T_ROW_SPLIT, T_WUPDATE_ONE_PLANE = range(10)
@@ -47,7 +48,7 @@ class QuantCfg(C.Structure):
                 ("symmetric", C.c_int), ("use_caller_grid", C.c_int), ("n_refresh", C.c_int),
                 ("h_refresh_iters", C.POINTER(C.c_int)), ("clip_points", C.c_int),
                 ("clip_min_ratio", C.c_double), ("fused_epilogue", C.c_int), ("wupdate_route", C.c_int),
-                ("product_planes", C.c_int)]
+                ("product_planes", C.c_int), ("wupdate_series", C.c_int)]
 
 
 class LsCfg(C.Structure):
@@ -63,7 +64,7 @@ class PairSwapCfg(C.Structure):
 class Report(C.Structure):
     _fields_ = [("err_before", C.c_double), ("err_after", C.c_double), ("moves", C.c_longlong),
                 ("iters_run", C.c_int), ("capped_columns", C.c_int), ("ms", C.c_float),
-                ("refreshed_iter", C.c_int), ("one_plane_iters", C.c_int)]
+                ("refreshed_iter", C.c_int), ("one_plane_iters", C.c_int), ("series_iters", C.c_int)]
 
 
 class AdmmqError(RuntimeError):
@@ -105,6 +106,7 @@ def load_library(path: Optional[str] = None):
                                          C.POINTER(Report)]
     lib.admmq_w_update.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, cd, vp]
     lib.admmq_test_w_update_correction.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, cd, vp]
+    lib.admmq_test_w_update_series.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, cd, vp]
     lib.admmq_local_search.argtypes = [vp, vp, ci, C.POINTER(LsCfg), vp, vp, vp, vp, C.POINTER(Report)]
     lib.admmq_objective.argtypes = [vp, vp, ci, ci, vp, vp, vp, C.POINTER(cd)]
     lib.admmq_pair_swap.argtypes = [vp, vp, ci, C.POINTER(PairSwapCfg), vp, vp, vp, vp, C.POINTER(Report)]
@@ -229,7 +231,7 @@ class Solver:
                        codes=None, scale=None, zero=None, Wq=None, resid=None, use_caller_grid=False,
                        report: bool = True, refresh_at: Sequence[int] = (), clip_points: int = 0,
                        clip_min_ratio: float = 0.8, fused_epilogue: bool = False, wupdate_route: int = 0,
-                       product_planes: int = 0):
+                       product_planes: int = 0, wupdate_series: int = 0):
         p, n = W0.shape
         gs = n if group_size in (0, n) else group_size
         dev = W0.device
@@ -240,7 +242,7 @@ class Solver:
         cfg = QuantCfg(C.sizeof(QuantCfg), bits, group_size, int(symmetric), int(use_caller_grid),
                        len(refresh_at), C.cast(iters, C.POINTER(C.c_int)) if len(refresh_at) else None,
                        int(clip_points), float(clip_min_ratio), int(fused_epilogue), int(wupdate_route),
-                       int(product_planes))
+                       int(product_planes), int(wupdate_series))
         rep = Report()
         st = self.lib.admmq_quantize_layer(self.h, _ptr(W0), p, C.byref(cfg), _ptr(codes), _ptr(scale),
                                            _ptr(zero), _ptr(Wq), _ptr(resid),
@@ -261,6 +263,14 @@ class Solver:
         _check(self.lib.admmq_test_w_update_correction(self.h, _ptr(W0), W0.shape[0], group_size, _ptr(codes),
                                                        _ptr(scale), _ptr(zero), _ptr(V), float(rho), _ptr(Z_out)),
                "admmq_test_w_update_correction")
+        return Z_out
+
+    def w_update_series(self, W0, group_size, codes, scale, zero, V, rho: float, Z_out=None):
+        """The same correction evaluated as the truncated series of the late iterations (admmq_testing.h)."""
+        Z_out = Z_out if Z_out is not None else torch.empty_like(W0)
+        _check(self.lib.admmq_test_w_update_series(self.h, _ptr(W0), W0.shape[0], group_size, _ptr(codes),
+                                                   _ptr(scale), _ptr(zero), _ptr(V), float(rho), _ptr(Z_out)),
+               "admmq_test_w_update_series")
         return Z_out
 
     def local_search(self, W0, bits, group_size, codes, scale, zero, Wq=None, max_moves_per_col: int = 0,

@@ -100,6 +100,8 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   c.stage_invd = cv.take<float>((size_t)(T + 1) * stage_factor_stride(n));
   c.shift_c = cv.take<double>((size_t)T + 1);
   c.Qs32 = explicit_operator_possible(n, p) ? cv.take<float>(nn) : nullptr;
+  c.N_hi = cv.take<bf16>(nn);
+  c.series_f = cv.take<float>((size_t)T + 1);
   c.ps_totals = cv.take<double>(PAIR_BATCH_MAX);
   c.ps_chosen = cv.take<int>(16);
   c.ps_d = cv.take<float>((size_t)2 * p);
@@ -385,6 +387,7 @@ admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg) {
   launch_finalize(c, cfg->damp_frac, c->precondition);
   launch_operand_scales(c);
   launch_split_f32(c, c->H, (long long)n * n, c->H_hi, c->H_lo);
+  launch_series_operand(c);                                // plane of mu I - H~, before the reduction overwrites H~
   if (tridiag_reduce(c) != cudaSuccess) return ADMMQ_ERR_CUDA;
   if (tridiag_form_qt(c) != cudaSuccess) return ADMMQ_ERR_CUDA;
   launch_split_f64(c, c->P64, n, nullptr, nullptr, c->Q_hi, c->Q_lo);   // planes of Q (second product)
@@ -408,6 +411,9 @@ admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg) {
     const double r = c->rho_host[t];
     const double g = fmax(fabs(c->mu_host - c->lam_lo) / (c->lam_lo + r), fabs(c->mu_host - c->lam_hi) / (c->lam_hi + r));
     c->planes_host[t] = (isfinite(g) && g <= 1.0 / 8192.0) ? 1 : 2;
+    // truncated series c (I + E) R: ||E|| = max |mu - lambda| / (mu + rho); its remainder is below ||E||^2 of R
+    const double e = fmax(fabs(c->mu_host - c->lam_lo), fabs(c->mu_host - c->lam_hi)) / (c->mu_host + r);
+    c->series_host[t] = (c->planes_host[t] == 1 && isfinite(e) && e <= 1.0 / 8192.0) ? 1 : 0;
   }
   c->state = 2;
   return ADMMQ_OK;
@@ -490,7 +496,21 @@ static cudaError_t w_update_explicit(admmq_ctx* a, int p, int stage, const EpiPa
   return one ? product(c, hi_only(op_R(c)), hi_only(Mp), p, n, n, epi) : product(c, op_R(c), Mp, p, n, n, epi);
 }
 
-static cudaError_t w_update_any(admmq_ctx* a, int p, int stage, const EpiParams& epi, bool explicit_op, int planes) {
+// The late iterations' W-update as the series c (I + E + ...) truncated after E = (mu I - H~) / (mu + rho):
+//   W - W_hat' - c R = c R E = [rho / (mu + rho)^2] R (mu I - H~)
+// one p n^2 product of the one-plane right-hand side with the fixed one-plane operand; the dropped terms are
+// below gamma(rho)^2 of R.  mu I - H~ is symmetric, so its rows serve as the operand.
+static cudaError_t w_update_series(admmq_ctx* a, int p, int stage, const EpiParams& epi) {
+  Ctx* c = &a->c;
+  const int n = c->n;
+  Timed t(a, ADMMQ_T_WUPDATE_ONE_PLANE);
+  const Planes Np = planes_f16(c->N_hi, nullptr, n, nullptr, c->series_f + stage);
+  return product(c, hi_only(op_R(c)), Np, p, n, n, epi);
+}
+
+static cudaError_t w_update_any(admmq_ctx* a, int p, int stage, const EpiParams& epi, bool explicit_op, int planes,
+                                bool series = false) {
+  if (series && planes == 1 && epi.kind == EPI_STORE) return w_update_series(a, p, stage, epi);
   return explicit_op ? w_update_explicit(a, p, stage, epi, planes) : w_update_products(a, p, stage, epi, planes);
 }
 
@@ -517,6 +537,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   if (cfg->n_refresh > 0 && group_of(ctx->c.n, cfg->group_size) < 2) return ADMMQ_ERR_UNSUPPORTED;
   if (cfg->wupdate_route < 0 || cfg->wupdate_route > 2) return ADMMQ_ERR_INVALID_ARG;
   if (cfg->product_planes != 0 && cfg->product_planes != 2) return ADMMQ_ERR_INVALID_ARG;
+  if (cfg->wupdate_series != 0 && cfg->wupdate_series != 1) return ADMMQ_ERR_INVALID_ARG;
   Ctx* c = &ctx->c;
   if (cfg->wupdate_route == 2 && !c->Qs32) return ADMMQ_ERR_UNSUPPORTED;
   const int n = c->n, p = d_out, gs = group_of(n, cfg->group_size), T = c->T;
@@ -551,7 +572,8 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.n_groups = n / gs;
   e.kmax = (1 << cfg->bits) - 1;
   e.Rnext = c->Y;                                          // Y is free once its planes exist
-  int one_plane_iters = 0;
+  int one_plane_iters = 0, series_iters = 0;
+  const bool series = cfg->wupdate_series == 0;
   for (int t = 0; t < T; ++t) {
     const double rho = c->rho_host[t];
     const double rho_next = (t + 1 < T) ? c->rho_host[t + 1] : rho;
@@ -563,6 +585,8 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     e.shift_c = c->shift_c + t;
     const int planes = (cfg->product_planes == 2 || cfg->fused_epilogue) ? 2 : c->planes_host[t];
     one_plane_iters += planes == 1;
+    const bool series_t = series && planes == 1 && c->series_host[t];
+    series_iters += series_t;
     bool refresh = false;
     for (int q = 0; q < cfg->n_refresh; ++q) refresh = refresh || (cfg->h_refresh_iters[q] == t);
     if (refresh) {
@@ -571,7 +595,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
       w.kind = EPI_STORE;
       w.C = c->Y;
       w.ldc = n;
-      if (w_update_any(ctx, p, t, w, explicit_op, planes) != cudaSuccess) return ADMMQ_ERR_CUDA;
+      if (w_update_any(ctx, p, t, w, explicit_op, planes, series_t) != cudaSuccess) return ADMMQ_ERR_CUDA;
       launch_grid_refresh(c, e, p, cfg->bits, cfg->symmetric, t, d_scale, d_zero, refresh_flags);
       if (t + 1 < T) {
         Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
@@ -591,10 +615,12 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
       w.kind = EPI_STORE;
       w.C = c->Y;
       w.ldc = n;
-      if (w_update_any(ctx, p, t, w, explicit_op, planes) != cudaSuccess) return ADMMQ_ERR_CUDA;
+      if (w_update_any(ctx, p, t, w, explicit_op, planes, series_t) != cudaSuccess) return ADMMQ_ERR_CUDA;
       Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
       w.kind = EPI_ADMM;
-      launch_admm_rows(c, w, p, c->R_hi, c->R_lo, c->rs_R);
+      // the lo plane of the next right-hand side is written only if the next iteration's products read it
+      const bool next_two = t + 1 >= T || cfg->product_planes == 2 || c->planes_host[t + 1] != 1;
+      launch_admm_rows(c, w, p, c->R_hi, next_two ? c->R_lo : nullptr, c->rs_R);
     }
   }
   if (d_resid) launch_reduce_partials(c, T, d_resid);
@@ -616,6 +642,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   h_report->iters_run = T;
   h_report->refreshed_iter = flags[1] - 1;
   h_report->one_plane_iters = one_plane_iters;
+  h_report->series_iters = series_iters;
   return st;
 }
 
@@ -635,6 +662,13 @@ admmq_status admmq_test_w_update_correction(admmq_ctx* ctx, const float* d_W0, i
   return w_update_call(ctx, d_W0, d_out, group_size, d_codes, d_scale, d_zero, d_V, rho, d_Z_out, 1);
 }
 
+admmq_status admmq_test_w_update_series(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
+                                        const unsigned char* d_codes, const float* d_scale,
+                                        const float* d_zero, const float* d_V, double rho, float* d_Z_out) {
+  return w_update_call(ctx, d_W0, d_out, group_size, d_codes, d_scale, d_zero, d_V, rho, d_Z_out, 2);
+}
+
+// correction_only: 0 the whole W-update, 1 the correction W - W_hat', 2 the correction by the truncated series
 static admmq_status w_update_call(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
                                   const unsigned char* d_codes, const float* d_scale, const float* d_zero,
                                   const float* d_V, double rho, float* d_W_out, int correction_only) {
@@ -657,9 +691,10 @@ static admmq_status w_update_call(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.kind = EPI_STORE;
   e.C = c->Y;                                               // free once its planes exist
   e.ldc = n;
-  if (w_update_products(ctx, p, stage, e, 2) != cudaSuccess) return ADMMQ_ERR_CUDA;
+  if ((correction_only == 2 ? w_update_series(ctx, p, stage, e) : w_update_products(ctx, p, stage, e, 2)) != cudaSuccess)
+    return ADMMQ_ERR_CUDA;
   launch_w_out(c, d_W0, p, gs, d_codes, d_scale, d_zero, d_V, 1.0 / rho, c->shift_c + stage, c->Y, d_W_out,
-               correction_only);
+               correction_only != 0);
   return cudaGetLastError() == cudaSuccess ? ADMMQ_OK : ADMMQ_ERR_CUDA;
 }
 

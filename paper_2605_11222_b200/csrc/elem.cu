@@ -588,6 +588,55 @@ __global__ void split_scaled_kernel(const float* __restrict__ src, long long cou
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Operand of the truncated-series W-update: N = mu0 I - H~ as ONE fp16 plane with a power-of-two scale for the
+// whole matrix, mu0 the mean of the diagonal of H~ (1 up to rounding when H~ has been scaled to unit diagonal).
+// H~ + rho I = (mu0 + rho) (I - N / (mu0 + rho)), so rho (H~ + rho I)^{-1} = c (I + E + E^2 + ...) with
+// E = N / (mu0 + rho); the late iterations keep the terms c R + c R E.  Read from the fp64 copy of H~ before
+// the reduction overwrites it.
+// ------------------------------------------------------------------------------------------------
+__global__ void series_mean_kernel(const double* __restrict__ A, int n, double* __restrict__ mu_out) {
+  __shared__ double scratch[32];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) s += A[(size_t)i * n + i];
+  s = block_sum(s, scratch);
+  if (threadIdx.x == 0) mu_out[0] = s / (double)n;
+}
+__global__ void series_max_kernel(const double* __restrict__ A, int n, const double* __restrict__ mu,
+                                  float* __restrict__ slot) {
+  __shared__ float scratch[32];
+  const int a = blockIdx.x;
+  const double m0 = mu[0];
+  float m = 0.0f;
+  for (int b = threadIdx.x; b < n; b += blockDim.x) {
+    const double v = (a == b ? m0 : 0.0) - A[(size_t)a * n + b];
+    m = fmaxf(m, fabsf((float)v));
+  }
+  m = block_max(m, scratch);
+  if (threadIdx.x == 0 && isfinite(m)) atomicMax(reinterpret_cast<unsigned int*>(slot) + 2, __float_as_uint(m));
+}
+__global__ void series_split_kernel(const double* __restrict__ A, int n, const double* __restrict__ mu,
+                                    const float* __restrict__ slot, bf16* __restrict__ hi) {
+  const int a = blockIdx.x;
+  const double m0 = mu[0], sc = (double)slot[1];
+  __half* out = reinterpret_cast<__half*>(hi) + (size_t)a * n;
+  for (int b = threadIdx.x; b < n; b += blockDim.x) {
+    const double v = ((a == b ? m0 : 0.0) - A[(size_t)a * n + b]) * sc;
+    out[b] = __float2half_rn(fminf(fmaxf((float)v, -60000.0f), 60000.0f));
+  }
+}
+
+void launch_series_operand(Ctx* c) {
+  const int n = c->n;
+  float* slot = c->fscal + 9;
+  cudaMemsetAsync(slot + 2, 0, sizeof(float), c->stream);
+  series_mean_kernel<<<1, 1024, 0, c->stream>>>(c->A64, n, c->scal + 11);
+  series_max_kernel<<<n, 256, 0, c->stream>>>(c->A64, n, c->scal + 11, slot);
+  scale_from_max_kernel<<<1, 1, 0, c->stream>>>(slot);
+  series_split_kernel<<<n, 256, 0, c->stream>>>(c->A64, n, c->scal + 11, slot, c->N_hi);
+  c->launches += 4;
+}
+
 void launch_global_split(Ctx* c, const float* src, long long count, float* slot, bf16* hi, bf16* lo) {
   cudaMemsetAsync(slot + 2, 0, sizeof(float), c->stream);
   const int blocks = c->num_sms * 8;
@@ -963,7 +1012,7 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
 #pragma unroll
       for (int e = 0; e < 8; ++e) split_f16(rowbuf[i + e] * sc, hh[e], ll[e]);
       *reinterpret_cast<uint4*>(hi + base + i) = *reinterpret_cast<const uint4*>(hh);
-      *reinterpret_cast<uint4*>(lo + base + i) = *reinterpret_cast<const uint4*>(ll);
+      if (lo) *reinterpret_cast<uint4*>(lo + base + i) = *reinterpret_cast<const uint4*>(ll);   // nullptr: one plane
     }
     __syncthreads();
   }

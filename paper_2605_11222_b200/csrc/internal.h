@@ -37,6 +37,7 @@ struct Ctx {
   int precondition = 1;
   double rho_host[4096];
   unsigned char planes_host[4096];  // per iteration: operand planes the W-update products need (1 or 2)
+  unsigned char series_host[4096];  // per iteration: 1 when the truncated series c (I + E) R is accurate to fp32
   double mu_host = 1.0, lam_lo = 0.0, lam_hi = 0.0;   // mean and Gershgorin bounds of the spectrum of H~ (host copies)
   long long launches = 0;
   long long wait_limit_cycles = 2000000000LL;   // bound of every device-side wait, about a second
@@ -64,11 +65,13 @@ struct Ctx {
   float* stage_l = nullptr;     // [T_max+1][stage_factor_stride(n)] LDL^T multipliers per penalty
   float* stage_invd = nullptr;  // [T_max+1][stage_factor_stride(n)] LDL^T inverse pivots per penalty, times 1 / (mu + rho)
   double* shift_c = nullptr;    // [T_max+1] c = rho / (mu + rho) per penalty (shifted W-update operator)
+  bf16* N_hi = nullptr;         // [n][n] one fp16 plane of mu I - H~ (operand of the truncated-series W-update), scale in fscal[9..11]
+  float* series_f = nullptr;    // [T_max+1] per penalty: rho / (mu + rho)^2 times the inverse scale of N_hi
   float* Qs32 = nullptr;        // [n][n] fp32 Q (mu I - T), or nullptr: input of the explicit-operator route (p_max > n only)
   double* ps_totals = nullptr;  // [PAIR_BATCH_MAX] totals of the candidate pairs of a pair-swap round
   int* ps_chosen = nullptr;     // [1] index of the applied pair, -1: none
   float* ps_d = nullptr;        // [2][p] applied perturbations of the two rows
-  double* trd_ws = nullptr;     // scratch of the blocked reduction: 66 n + 67 * 256 doubles
+  double* trd_ws = nullptr;     // scratch of the blocked reduction (tridiag_blocked_scratch_doubles)
   double* wy_s = nullptr;       // [ceil(n/32)][32][32] triangular factors of the reflector blocks
   bf16 *Q_hi = nullptr, *Q_lo = nullptr;    // [n][n] Q   (row i, col m)
   bf16 *QT_hi = nullptr, *QT_lo = nullptr;  // [n][n] Q^T (row m, col k)
@@ -82,7 +85,7 @@ struct Ctx {
   double* scal = nullptr;       // small fp64 scalars (objective, counters)
   float* fscal = nullptr;       // [0] 1 / scale of the Q planes, [1] 1 / scale of the H planes, [2] scale of the H planes,
                                 // [3] 1 / scale and [4] scale of the shifted Q^T planes, [5] their largest magnitude,
-                                // [6..8] 1 / scale, scale, largest magnitude of the explicit operator's planes
+                                // [6..8] 1 / scale, scale, largest magnitude of the explicit operator's planes; [9..11] the same of N_hi
   float* rs_R = nullptr;        // [p] inverse row scales of the R (and E) planes
   float* rs_Y = nullptr;        // [p] inverse row scales of the Y' planes
   bf16 *XT_hi = nullptr, *XT_lo = nullptr;  // [n][XT_ROWS] transposed chunk of X
@@ -141,6 +144,7 @@ size_t tridiag_blocked_scratch_doubles(int n);
 cudaError_t tridiag_form_qt(Ctx* c);                // reflectors -> P64 = Q^T
 size_t stage_factor_stride(int n);                  // floats per penalty in stage_l / stage_invd
 void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count);
+void launch_series_operand(Ctx* c);   // A64 = H~ (before the reduction overwrites it) -> N_hi, fscal[9..11]; mean of its diagonal -> scal[11]
 void launch_tridiag_solve(Ctx* c, const float* Y, int p, int stage, bf16* hi, bf16* lo, float* row_inv);
 
 // ---- local_search.cu ----

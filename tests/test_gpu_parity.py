@@ -135,6 +135,49 @@ def test_w_update_parity(n, p, gs, kind):
     assert sol.last_device_status() == B.OK
 
 
+@pytest.mark.parametrize("n,p", [(520, 264), (1024, 512)])
+def test_w_update_as_truncated_series_at_large_penalties(n, p):
+    """rho (H~ + rho I)^{-1} = c (I + E + E^2 + ...), E = (mu I - H~) / (mu + rho) (Eq. 7 rearranged).  The late
+    iterations keep c R + c R E; what they drop is bounded by gamma^2 ||R|| with gamma = max |mu - lambda| / (mu +
+    rho).  Checked against the fp64 W-update of the oracle at penalties on both sides of the solver's switch
+    (gamma <= 2^-13): the error follows gamma^2 where the truncation dominates and sits at the level of the route
+    through the factorisation where it does not."""
+    spec = wl.small_case(n, p, 4096, group_size=0, T=2)
+    W = wl.gen_weight(spec, DEV)
+    sol = B.Solver(n, p, T_max=2)
+    sol.hessian_reset()
+    for c in range(spec.n_chunks):
+        sol.hessian_accumulate(wl.gen_x_chunk(spec, c, DEV))
+    sol.factor(rho=[0.1, 0.2])
+    Ho = oracle_hessian(spec, DEV)
+    Wn = np64(W)
+    delta, z0 = O.grid_fit(Wn, spec.bits, 0, False)
+    s, Ht, Ws = O.precondition(Ho, Wn)
+    lam, U = O.eig_factor(Ht)
+    mu = float(np.trace(Ht)) / n
+    rng = np.random.default_rng(11)
+    codes = rng.integers(0, 1 << spec.bits, size=Wn.shape).astype(np.uint8)
+    V = (0.01 * np.abs(Ws).mean() * rng.standard_normal(Wn.shape)).astype(np.float32)
+    D = s[None, :] * O.dequantize(codes, delta, z0)
+    args = (W, 0, to_dev(codes, torch.uint8, DEV), to_dev(delta, torch.float32, DEV),
+            to_dev(z0, torch.float32, DEV), to_dev(V, torch.float32, DEV))
+    spread = max(abs(mu - lam.min()), abs(mu - lam.max()))
+    for gamma in (2.0 ** -6, 2.0 ** -10, 2.0 ** -13, 2.0 ** -16):
+        rho = spread / gamma - mu
+        Zo = O.w_update(lam, U, Ws @ Ht, D, V.astype(np.float64), rho) - Ws      # W - W_hat' in fp64
+        R = D - V.astype(np.float64) / rho - Ws
+        Zs = np64(sol.w_update_series(*args, rho))
+        Ze = np64(sol.w_update_correction(*args, rho))
+        err_series = np.linalg.norm(Zs - Zo) / np.linalg.norm(R)
+        err_exact = np.linalg.norm(Ze - Zo) / np.linalg.norm(R)
+        assert err_exact <= 4e-7, (gamma, err_exact)
+        # truncation (<= gamma^2 / (1 - gamma)) plus the rounding of a one-plane product of relative size gamma
+        assert err_series <= gamma * gamma / (1 - gamma) + gamma * 2.0 ** -11 + 4e-7, (gamma, err_series)
+        if gamma <= 2.0 ** -13:                                  # where the solver uses it: fp32 resolution
+            assert err_series <= 2.0 ** -22, (gamma, err_series)
+    assert sol.last_device_status() == B.OK
+
+
 # ------------------------------------------------------------------ whole layer, mid size
 @pytest.mark.parametrize("kw", [
     dict(d_in=512, d_out=384, n_tokens=6144),                                   # g128, asym, 3 bit
@@ -620,10 +663,17 @@ def test_one_plane_products_of_the_late_iterations():
     c0, s0, z0, rep0 = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric)
     c2, s2, z2, rep2 = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, product_planes=2)
     assert sol.last_device_status() == B.OK
+    c1, s1, z1, rep1 = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, wupdate_series=1)
     assert 10 <= rep0.one_plane_iters < spec.T and rep2.one_plane_iters == 0
+    # by default those iterations are evaluated as the truncated series; wupdate_series = 1 keeps them on the
+    # factorisation (one-plane products and the row solve)
+    assert rep0.one_plane_iters - 1 <= rep0.series_iters <= rep0.one_plane_iters and rep2.series_iters == 0
+    assert rep1.one_plane_iters == rep0.one_plane_iters and rep1.series_iters == 0
     assert (c0.cpu().numpy() == res.admm.codes).mean() >= CODE_AGREEMENT
+    assert (c1.cpu().numpy() == res.admm.codes).mean() >= CODE_AGREEMENT
     assert (c2.cpu().numpy() == res.admm.codes).mean() >= CODE_AGREEMENT
     assert (c0 == c2).float().mean().item() >= 0.9995
+    assert (c1 == c2).float().mean().item() >= 0.9995
     assert abs(rep0.err_before - res.err_admm) <= ERR_TOL * res.err_admm
 
 
