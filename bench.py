@@ -545,11 +545,13 @@ def main():
                       "default_ms": df_rep.ms,
                       "default_one_plane_iterations": df_rep.one_plane_iters,
                       "default_series_iterations": df_rep.series_iters,
+                      "default_two_term_series_iterations": df_rep.series2_iters,
                       "err_admm_two_planes": tp_rep.err_before, "err_admm_without_series": ns_rep.err_before,
                       "err_admm_default": df_rep.err_before,
                       "codes_equal_fraction": float((c_two == c_def).float().mean().item()),
                       "codes_equal_fraction_without_series": float((codes == c_def).float().mean().item())}
     n_series = int(df_rep.series_iters)
+    n_series2 = int(df_rep.series2_iters)
     n_one_plane = int(df_rep.one_plane_iters)
 
     # ---- a run whose grid comes from the MSE search for the clipping ratio, 100 candidates down to 0.8
@@ -639,7 +641,9 @@ def main():
     w_update_ms = (ms_p1 + ms_p2 + ms_1p + timing["tridiag_solve"][0] + timing["row_split"][0]) / args.steps
     # one-plane launches: one product R (mu I - H~) per iteration of the truncated series, else both products of an
     # iteration, of which the first has rows_p1 rows
-    flops_one_plane = args.steps * 2.0 * n * n * (n_series * p + (n_one_plane - n_series) * (rows_p1 + p))
+    # (the two-term series adds one p-row one-plane product per iteration; its two-plane product is timed as
+    # a second product, p rows)
+    flops_one_plane = args.steps * 2.0 * n * n * ((n_series + n_series2) * p + (n_one_plane - n_series) * (rows_p1 + p))
     executed_flops_per_step = (flops_two_plane + flops_one_plane) / args.steps
     breakdown = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
                  for k, v in timing.items()}
@@ -661,9 +665,22 @@ def main():
     # row pass: reads z 4, w 4, V 4, codes 1; writes V 4, codes 1, two fp16 planes 4 bytes per element; on the
     # explicit route the same timer also takes the split of the n x n operator (maximum pass 4, split 4 + 4 bytes
     # per element), so a launch there is the mean of the two.
+    def _row_pass_roofline():
+        # all launches under the row-pass timer: T row passes (22 p n bytes), the splits of the two-term series'
+        # intermediate (8 p n) and, on the explicit route, of the n x n operator (12 n^2) in the other iterations
+        ms, cnt = timing["row_split"]
+        if cnt == 0 or ms <= 0:
+            return None
+        n_fact = T - n_series - n_series2
+        total = args.steps * (22.0 * p * n * T + 8.0 * p * n * n_series2 +
+                              (12.0 * n * n * n_fact if explicit_route else 0.0))
+        gbs = total / (ms * 1e-3) / 1e9
+        return {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / peaks["hbm_gbs"], "launches": cnt, "avg_launch_ms": ms / cnt}
+
     kernel_rooflines = {
         "tridiag_solve": _hbm("tridiag_solve", 8.0 * rows_p1 * n),
-        "row_split": _hbm("row_split", (22.0 * p * n + 12.0 * n * n) / 2 if explicit_route else 22.0 * p * n),
+        "row_split": _row_pass_roofline(),
         "transpose": _hbm("transpose", 2.0 * x_bytes * chunk_rows * n),
     }
     if n_1p:
@@ -695,7 +712,7 @@ def main():
         "layers_per_s": world / (ms_step / 1e3),
         "w_update_useful_tflops": 4.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
         "w_update_executed_tflops": executed_flops_per_step / (w_update_ms * 1e-3) / 1e12,
-        "one_plane_iterations": n_one_plane, "series_iterations": n_series, "w_update_route": "explicit operator" if explicit_route else "two products",
+        "one_plane_iterations": n_one_plane, "series_iterations": n_series, "two_term_series_iterations": n_series2, "w_update_route": "explicit operator" if explicit_route else "two products",
         "err_before_local_search": rep.err_before, "err_after_local_search": rep.err_after,
         "local_search_moves": rep.moves, "pair_swap_after_local_search": pair_swap, "admm_with_grid_refresh": grid_refresh,
         "admm_with_mse_clip_search": mse_clip, "admm_with_fused_epilogue": fused_variant,

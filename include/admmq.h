@@ -181,14 +181,17 @@ typedef struct {
                            penalty grows.  0: two fp16 planes per operand (about 22 bits) while gamma > 2^-13, one
                            plane (11 bits, a third of the tensor-core work) afterwards, where the rounding of one
                            plane is below the fp32 resolution of the W-update.  2: two planes in every iteration. */
-  int wupdate_series;   /* the late iterations' W-update as a truncated series.  With E = (mu I - H~) / (mu + rho) the
+  int wupdate_series;   /* the later iterations' W-update as a truncated series.  With E = (mu I - H~) / (mu + rho) the
                            operator of Eq. 7 is rho (H~ + rho I)^{-1} = c (I - E)^{-1} = c (I + E + E^2 + ...), and
-                           ||E|| = max |mu - lambda| / (mu + rho).  0: once ||E|| <= 2^-13 (in effect the iterations that run on
-                           one plane) the update is evaluated as c R + c R E -- ONE product with the fixed operand mu I - H~
-                           instead of two products and a row solve; the dropped terms are below ||E||^2 <= 2^-26 of
-                           the right-hand side, under the fp32 resolution of the stored iterate.  1: never (every
+                           ||E|| = max |mu - lambda| / (mu + rho) shrinks as the penalty grows.  0: once ||E|| <= 2^-13
+                           (in effect the iterations that run on one plane) the update is evaluated as c R + c R E --
+                           ONE product with the fixed operand mu I - H~ instead of two products and a row solve; for
+                           2^-13 < ||E|| <= 2^-9 as c R + c R E + c R E^2 -- the first product on two planes, the
+                           second (of relative size ||E||^2) on one.  The dropped terms are below 2^-26 of the
+                           right-hand side, under the fp32 resolution of the stored iterate.  1: never (every
                            iteration goes through the factorisation).  Ignored with product_planes = 2 or
-                           fused_epilogue = 1, which keep every iteration on the two-plane route. */
+                           fused_epilogue = 1, which keep every iteration on the two-plane route through the
+                           factorisation. */
 } admmq_quant_cfg;
 typedef struct {
   double err_before;    /* Tr(E^T H E), E = W_q - W_hat, at entry (local search) / of the ADMM result */
@@ -199,7 +202,8 @@ typedef struct {
   float ms;             /* device time of the call, CUDA events */
   int refreshed_iter;   /* quantize_layer: iteration of the accepted grid refresh, -1: none */
   int one_plane_iters;  /* quantize_layer: iterations whose products ran on one fp16 plane per operand */
-  int series_iters;     /* quantize_layer: of those, iterations evaluated as the truncated series (one product) */
+  int series_iters;     /* quantize_layer: iterations evaluated as the series with one term of E (one product) */
+  int series2_iters;    /* quantize_layer: iterations evaluated as the series with two terms of E (two products) */
 } admmq_report;
 admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out,
                                   const admmq_quant_cfg* cfg, unsigned char* d_codes, float* d_scale,

@@ -30,12 +30,14 @@ admmq_status admmq_test_w_update_correction(admmq_ctx* ctx, const float* d_W0, i
                                             const unsigned char* d_codes, const float* d_scale,
                                             const float* d_zero, const float* d_V, double rho, float* d_Z_out);
 
-/* The same correction evaluated as the late iterations do it (admmq_quant_cfg.wupdate_series): c R + c R E with
- * the fixed one-plane operand mu I - H~, whatever gamma(rho) is.  For a test that compares it with the route
- * through the factorisation at a penalty where the solver would switch to it. */
+/* The same correction evaluated as the later iterations do it (admmq_quant_cfg.wupdate_series): the series
+ * c (I + E + E^2 + ...) R with `terms` = 1 or 2 terms of E kept, on the fixed operand mu I - H~, whatever ||E|| is
+ * at this penalty.  For a test that compares it with the route through the factorisation on both sides of the
+ * penalties where the solver would switch to it.  ADMMQ_ERR_INVALID_ARG for any other `terms`. */
 admmq_status admmq_test_w_update_series(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
                                         const unsigned char* d_codes, const float* d_scale,
-                                        const float* d_zero, const float* d_V, double rho, float* d_Z_out);
+                                        const float* d_zero, const float* d_V, double rho, int terms,
+                                        float* d_Z_out);
 
 #ifdef __cplusplus
 }

@@ -64,7 +64,8 @@ class PairSwapCfg(C.Structure):
 class Report(C.Structure):
     _fields_ = [("err_before", C.c_double), ("err_after", C.c_double), ("moves", C.c_longlong),
                 ("iters_run", C.c_int), ("capped_columns", C.c_int), ("ms", C.c_float),
-                ("refreshed_iter", C.c_int), ("one_plane_iters", C.c_int), ("series_iters", C.c_int)]
+                ("refreshed_iter", C.c_int), ("one_plane_iters", C.c_int), ("series_iters", C.c_int),
+                ("series2_iters", C.c_int)]
 
 
 class AdmmqError(RuntimeError):
@@ -106,7 +107,7 @@ def load_library(path: Optional[str] = None):
                                          C.POINTER(Report)]
     lib.admmq_w_update.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, cd, vp]
     lib.admmq_test_w_update_correction.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, cd, vp]
-    lib.admmq_test_w_update_series.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, cd, vp]
+    lib.admmq_test_w_update_series.argtypes = [vp, vp, ci, ci, vp, vp, vp, vp, cd, ci, vp]
     lib.admmq_local_search.argtypes = [vp, vp, ci, C.POINTER(LsCfg), vp, vp, vp, vp, C.POINTER(Report)]
     lib.admmq_objective.argtypes = [vp, vp, ci, ci, vp, vp, vp, C.POINTER(cd)]
     lib.admmq_pair_swap.argtypes = [vp, vp, ci, C.POINTER(PairSwapCfg), vp, vp, vp, vp, C.POINTER(Report)]
@@ -265,11 +266,13 @@ class Solver:
                "admmq_test_w_update_correction")
         return Z_out
 
-    def w_update_series(self, W0, group_size, codes, scale, zero, V, rho: float, Z_out=None):
-        """The same correction evaluated as the truncated series of the late iterations (admmq_testing.h)."""
+    def w_update_series(self, W0, group_size, codes, scale, zero, V, rho: float, terms: int = 1, Z_out=None):
+        """The same correction evaluated as the truncated series of the later iterations, `terms` terms of E kept
+        (admmq_testing.h)."""
         Z_out = Z_out if Z_out is not None else torch.empty_like(W0)
         _check(self.lib.admmq_test_w_update_series(self.h, _ptr(W0), W0.shape[0], group_size, _ptr(codes),
-                                                   _ptr(scale), _ptr(zero), _ptr(V), float(rho), _ptr(Z_out)),
+                                                   _ptr(scale), _ptr(zero), _ptr(V), float(rho), int(terms),
+                                                   _ptr(Z_out)),
                "admmq_test_w_update_series")
         return Z_out
 

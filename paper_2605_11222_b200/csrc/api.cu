@@ -101,6 +101,8 @@ size_t carve(admmq_ctx* a, char* base, int n, int p, int T) {
   c.shift_c = cv.take<double>((size_t)T + 1);
   c.Qs32 = explicit_operator_possible(n, p) ? cv.take<float>(nn) : nullptr;
   c.N_hi = cv.take<bf16>(nn);
+  c.N_lo = cv.take<bf16>(nn);
+  c.series_g = cv.take<float>((size_t)T + 1);
   c.series_f = cv.take<float>((size_t)T + 1);
   c.ps_totals = cv.take<double>(PAIR_BATCH_MAX);
   c.ps_chosen = cv.take<int>(16);
@@ -413,7 +415,9 @@ admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg) {
     c->planes_host[t] = (isfinite(g) && g <= 1.0 / 8192.0) ? 1 : 2;
     // truncated series c (I + E) R: ||E|| = max |mu - lambda| / (mu + rho); its remainder is below ||E||^2 of R
     const double e = fmax(fabs(c->mu_host - c->lam_lo), fabs(c->mu_host - c->lam_hi)) / (c->mu_host + r);
-    c->series_host[t] = (c->planes_host[t] == 1 && isfinite(e) && e <= 1.0 / 8192.0) ? 1 : 0;
+    // one term of E (one plane) once ||E|| <= 2^-13; two terms -- the first on two planes, the second, of relative
+    // size ||E||^2, on one -- once ||E|| <= 2^-9 (remainder below ||E||^3 <= 2^-27)
+    c->series_host[t] = !isfinite(e) ? 0 : (c->planes_host[t] == 1 && e <= 1.0 / 8192.0) ? 1 : (e <= 1.0 / 512.0 ? 2 : 0);
   }
   c->state = 2;
   return ADMMQ_OK;
@@ -508,9 +512,35 @@ static cudaError_t w_update_series(admmq_ctx* a, int p, int stage, const EpiPara
   return product(c, hi_only(op_R(c)), Np, p, n, n, epi);
 }
 
+// Two terms, c R E + c R E^2, for the iterations just before: the first term is the product above on two planes per
+// operand (its rounding must stay below 2^-24 / ||E|| of itself), the second -- of relative size ||E||^2 <= 2^-18 --
+// a one-plane product of the first with the same operand, added into the stored result.
+static cudaError_t w_update_series2(admmq_ctx* a, int p, int stage, const EpiParams& epi) {
+  Ctx* c = &a->c;
+  const int n = c->n;
+  cudaError_t err;
+  {
+    Timed t(a, ADMMQ_T_WUPDATE_PRODUCT2);
+    const Planes Np = planes_f16(c->N_hi, c->N_lo, n, nullptr, c->series_f + stage);
+    err = product(c, op_R(c), Np, p, n, n, epi);            // epi.C = c R E
+  }
+  if (err != cudaSuccess) return err;
+  {
+    Timed t(a, ADMMQ_T_ROW_SPLIT);
+    launch_row_split(c, epi.C, p, c->Y_hi, c->Y_lo, c->rs_Y);
+  }
+  EpiParams e2 = epi;
+  e2.kind = EPI_ACCUM;
+  e2.lower_only = 0;
+  Timed t(a, ADMMQ_T_WUPDATE_ONE_PLANE);
+  const Planes Ng = planes_f16(c->N_hi, nullptr, n, nullptr, c->series_g + stage);
+  return product(c, hi_only(op_Y(c)), Ng, p, n, n, e2);     // epi.C += (c R E) E
+}
+
 static cudaError_t w_update_any(admmq_ctx* a, int p, int stage, const EpiParams& epi, bool explicit_op, int planes,
-                                bool series = false) {
-  if (series && planes == 1 && epi.kind == EPI_STORE) return w_update_series(a, p, stage, epi);
+                                int series = 0) {
+  if (series == 1 && planes == 1 && epi.kind == EPI_STORE) return w_update_series(a, p, stage, epi);
+  if (series == 2 && epi.kind == EPI_STORE && epi.ldc == a->c.n) return w_update_series2(a, p, stage, epi);
   return explicit_op ? w_update_explicit(a, p, stage, epi, planes) : w_update_products(a, p, stage, epi, planes);
 }
 
@@ -572,8 +602,9 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.n_groups = n / gs;
   e.kmax = (1 << cfg->bits) - 1;
   e.Rnext = c->Y;                                          // Y is free once its planes exist
-  int one_plane_iters = 0, series_iters = 0;
-  const bool series = cfg->wupdate_series == 0;
+  int one_plane_iters = 0, series_iters = 0, series2_iters = 0;
+  const bool series = cfg->wupdate_series == 0 && !cfg->fused_epilogue && cfg->product_planes != 2;
+  auto series_of = [&](int t) { return series ? (int)c->series_host[t] : 0; };
   for (int t = 0; t < T; ++t) {
     const double rho = c->rho_host[t];
     const double rho_next = (t + 1 < T) ? c->rho_host[t + 1] : rho;
@@ -585,8 +616,10 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     e.shift_c = c->shift_c + t;
     const int planes = (cfg->product_planes == 2 || cfg->fused_epilogue) ? 2 : c->planes_host[t];
     one_plane_iters += planes == 1;
-    const bool series_t = series && planes == 1 && c->series_host[t];
-    series_iters += series_t;
+    // terms of E this iteration's W-update keeps (0: through the factorisation)
+    const int series_t = series_of(t);
+    series_iters += series_t == 1;
+    series2_iters += series_t == 2;
     bool refresh = false;
     for (int q = 0; q < cfg->n_refresh; ++q) refresh = refresh || (cfg->h_refresh_iters[q] == t);
     if (refresh) {
@@ -619,7 +652,8 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
       Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
       w.kind = EPI_ADMM;
       // the lo plane of the next right-hand side is written only if the next iteration's products read it
-      const bool next_two = t + 1 >= T || cfg->product_planes == 2 || c->planes_host[t + 1] != 1;
+      const bool next_two = t + 1 >= T || cfg->product_planes == 2 || series_of(t + 1) == 2 ||
+                            (series_of(t + 1) == 0 && c->planes_host[t + 1] != 1);
       launch_admm_rows(c, w, p, c->R_hi, next_two ? c->R_lo : nullptr, c->rs_R);
     }
   }
@@ -643,6 +677,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   h_report->refreshed_iter = flags[1] - 1;
   h_report->one_plane_iters = one_plane_iters;
   h_report->series_iters = series_iters;
+  h_report->series2_iters = series2_iters;
   return st;
 }
 
@@ -664,11 +699,13 @@ admmq_status admmq_test_w_update_correction(admmq_ctx* ctx, const float* d_W0, i
 
 admmq_status admmq_test_w_update_series(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
                                         const unsigned char* d_codes, const float* d_scale,
-                                        const float* d_zero, const float* d_V, double rho, float* d_Z_out) {
-  return w_update_call(ctx, d_W0, d_out, group_size, d_codes, d_scale, d_zero, d_V, rho, d_Z_out, 2);
+                                        const float* d_zero, const float* d_V, double rho, int terms,
+                                        float* d_Z_out) {
+  if (terms != 1 && terms != 2) return ADMMQ_ERR_INVALID_ARG;
+  return w_update_call(ctx, d_W0, d_out, group_size, d_codes, d_scale, d_zero, d_V, rho, d_Z_out, 1 + terms);
 }
 
-// correction_only: 0 the whole W-update, 1 the correction W - W_hat', 2 the correction by the truncated series
+// correction_only: 0 the whole W-update, 1 the correction W - W_hat', 2 / 3 the correction by the series with one / two terms of E
 static admmq_status w_update_call(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
                                   const unsigned char* d_codes, const float* d_scale, const float* d_zero,
                                   const float* d_V, double rho, float* d_W_out, int correction_only) {
@@ -691,8 +728,10 @@ static admmq_status w_update_call(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.kind = EPI_STORE;
   e.C = c->Y;                                               // free once its planes exist
   e.ldc = n;
-  if ((correction_only == 2 ? w_update_series(ctx, p, stage, e) : w_update_products(ctx, p, stage, e, 2)) != cudaSuccess)
-    return ADMMQ_ERR_CUDA;
+  const cudaError_t err = correction_only == 2   ? w_update_series(ctx, p, stage, e)
+                          : correction_only == 3 ? w_update_series2(ctx, p, stage, e)
+                                                 : w_update_products(ctx, p, stage, e, 2);
+  if (err != cudaSuccess) return ADMMQ_ERR_CUDA;
   launch_w_out(c, d_W0, p, gs, d_codes, d_scale, d_zero, d_V, 1.0 / rho, c->shift_c + stage, c->Y, d_W_out,
                correction_only != 0);
   return cudaGetLastError() == cudaSuccess ? ADMMQ_OK : ADMMQ_ERR_CUDA;

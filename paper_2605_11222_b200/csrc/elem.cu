@@ -589,10 +589,10 @@ __global__ void split_scaled_kernel(const float* __restrict__ src, long long cou
 }
 
 // ------------------------------------------------------------------------------------------------
-// Operand of the truncated-series W-update: N = mu0 I - H~ as ONE fp16 plane with a power-of-two scale for the
-// whole matrix, mu0 the mean of the diagonal of H~ (1 up to rounding when H~ has been scaled to unit diagonal).
+// Operand of the truncated-series W-update: N = mu0 I - H~ as fp16 planes (hi, lo) with a power-of-two scale for
+// the whole matrix, mu0 the mean of the diagonal of H~ (1 up to rounding when H~ has been scaled to unit diagonal).
 // H~ + rho I = (mu0 + rho) (I - N / (mu0 + rho)), so rho (H~ + rho I)^{-1} = c (I + E + E^2 + ...) with
-// E = N / (mu0 + rho); the late iterations keep the terms c R + c R E.  Read from the fp64 copy of H~ before
+// E = N / (mu0 + rho); the later iterations keep c R + c R E (+ c R E^2 somewhat earlier).  Read from the fp64 copy of H~ before
 // the reduction overwrites it.
 // ------------------------------------------------------------------------------------------------
 __global__ void series_mean_kernel(const double* __restrict__ A, int n, double* __restrict__ mu_out) {
@@ -616,13 +616,15 @@ __global__ void series_max_kernel(const double* __restrict__ A, int n, const dou
   if (threadIdx.x == 0 && isfinite(m)) atomicMax(reinterpret_cast<unsigned int*>(slot) + 2, __float_as_uint(m));
 }
 __global__ void series_split_kernel(const double* __restrict__ A, int n, const double* __restrict__ mu,
-                                    const float* __restrict__ slot, bf16* __restrict__ hi) {
+                                    const float* __restrict__ slot, bf16* __restrict__ hi,
+                                    bf16* __restrict__ lo) {
   const int a = blockIdx.x;
   const double m0 = mu[0], sc = (double)slot[1];
-  __half* out = reinterpret_cast<__half*>(hi) + (size_t)a * n;
+  __half* oh = reinterpret_cast<__half*>(hi) + (size_t)a * n;
+  __half* ol = reinterpret_cast<__half*>(lo) + (size_t)a * n;
   for (int b = threadIdx.x; b < n; b += blockDim.x) {
     const double v = ((a == b ? m0 : 0.0) - A[(size_t)a * n + b]) * sc;
-    out[b] = __float2half_rn(fminf(fmaxf((float)v, -60000.0f), 60000.0f));
+    split_f16((float)v, oh[b], ol[b]);
   }
 }
 
@@ -633,7 +635,7 @@ void launch_series_operand(Ctx* c) {
   series_mean_kernel<<<1, 1024, 0, c->stream>>>(c->A64, n, c->scal + 11);
   series_max_kernel<<<n, 256, 0, c->stream>>>(c->A64, n, c->scal + 11, slot);
   scale_from_max_kernel<<<1, 1, 0, c->stream>>>(slot);
-  series_split_kernel<<<n, 256, 0, c->stream>>>(c->A64, n, c->scal + 11, slot, c->N_hi);
+  series_split_kernel<<<n, 256, 0, c->stream>>>(c->A64, n, c->scal + 11, slot, c->N_hi, c->N_lo);
   c->launches += 4;
 }
 

@@ -687,6 +687,7 @@ __device__ __forceinline__ Schedule make_pair_schedule(int M, int N, int pairs) 
   return s;
 }
 
+template <int EPI>                          // EPI_STORE, or EPI_ACCUM (C += the product, whole tiles)
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, uint32_t fmt, EpiParams epi,
                     int* status, long long wait_limit, int hold_loads) {
@@ -847,7 +848,7 @@ gemm_tc_pair_kernel(const __grid_constant__ TcMaps maps, int M, int N, int K, ui
       if (lane == 0) mbar_arrive_cluster(pempty_leader + 8 * pb);   // in registers: the buffer is free
       ++g;
       if (mine)
-        epilogue_block<EPI_STORE>(epi, row0, col0, M, N, sums, stage_all + (warp - 2) * STAGE_FLOATS, lane, r2, s2);
+        epilogue_block<EPI>(epi, row0, col0, M, N, sums, stage_all + (warp - 2) * STAGE_FLOATS, lane, r2, s2);
     }
   }
   tc_fence_before();
@@ -943,7 +944,9 @@ static cudaError_t launch_tc_pair(Ctx* c, Planes A, Planes B, int M, int N, int 
     return cudaErrorInvalidValue;
   maps.a[1] = maps.a[0];
   const size_t smem = (size_t)PAIR_STAGES * PAIR_STAGE_BYTES + 1024;
-  const cudaError_t ea = ensure_dynamic_smem((const void*)gemm_tc_pair_kernel, (int)smem);
+  const bool accum = epi.kind == EPI_ACCUM;
+  auto kernel = accum ? gemm_tc_pair_kernel<EPI_ACCUM> : gemm_tc_pair_kernel<EPI_STORE>;
+  const cudaError_t ea = ensure_dynamic_smem((const void*)kernel, (int)smem);
   if (ea != cudaSuccess) return ea;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * (c->num_sms / 2));
@@ -961,7 +964,7 @@ static cudaError_t launch_tc_pair(Ctx* c, Planes A, Planes B, int M, int N, int 
   // the others (asked once per context, which belongs to one device)
   if (c->pair_clusters == 0) {
     int nc = 0;
-    if (cudaOccupancyMaxActiveClusters(&nc, gemm_tc_pair_kernel, &cfg) != cudaSuccess || nc < 1) {
+    if (cudaOccupancyMaxActiveClusters(&nc, kernel, &cfg) != cudaSuccess || nc < 1) {
       c->pair_clusters = -1;
       cudaGetLastError();
     } else {
@@ -973,7 +976,7 @@ static cudaError_t launch_tc_pair(Ctx* c, Planes A, Planes B, int M, int N, int 
   const int pairs = tiles < c->pair_clusters ? tiles : c->pair_clusters;
   cfg.gridDim = dim3(2 * pairs);
   const uint32_t fmt = A.f16 ? 0u : 1u;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_tc_pair_kernel, maps, M, N, K, fmt, epi, c->status,
+  cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, maps, M, N, K, fmt, epi, c->status,
                                      c->wait_limit_cycles, c->hold_loads);
   c->launches++;
   return e != cudaSuccess ? e : cudaGetLastError();
@@ -996,8 +999,10 @@ cudaError_t gemm_tc(Ctx* c, Planes A, Planes B, int M, int N, int K, const EpiPa
   epi.a_inv = A.all_inv;
   epi.b_inv = B.all_inv;
   const uint32_t idesc = A.f16 ? 0u : 1u;                  // operand format: 0 = fp16, 1 = bf16
-  // one fp16 plane and a plain store, large enough for 256 x 256 tiles: the CTA-pair kernel
-  if (na == 1 && A.f16 && epi.kind == EPI_STORE && c->use_pair_kernel && M >= PAIR_M && N >= BN && c->num_sms >= 2) {
+  // one fp16 plane and a plain store (or a sum into whole tiles of C), large enough for 256 x 256 tiles: the
+  // CTA-pair kernel
+  const bool pair_epi = epi.kind == EPI_STORE || (epi.kind == EPI_ACCUM && !epi.lower_only);
+  if (na == 1 && A.f16 && pair_epi && c->use_pair_kernel && M >= PAIR_M && N >= BN && c->num_sms >= 2) {
     const cudaError_t ep = launch_tc_pair(c, A, B, M, N, K, epi);
     if (ep != cudaErrorNotSupported) return ep;           // no room for a pair on this device: single-CTA kernel
   }

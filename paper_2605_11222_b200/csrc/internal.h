@@ -37,7 +37,7 @@ struct Ctx {
   int precondition = 1;
   double rho_host[4096];
   unsigned char planes_host[4096];  // per iteration: operand planes the W-update products need (1 or 2)
-  unsigned char series_host[4096];  // per iteration: 1 when the truncated series c (I + E) R is accurate to fp32
+  unsigned char series_host[4096];  // per iteration: terms of E the truncated series needs to be accurate to fp32 (1, 2), 0: not usable
   double mu_host = 1.0, lam_lo = 0.0, lam_hi = 0.0;   // mean and Gershgorin bounds of the spectrum of H~ (host copies)
   long long launches = 0;
   long long wait_limit_cycles = 2000000000LL;   // bound of every device-side wait, about a second
@@ -66,6 +66,8 @@ struct Ctx {
   float* stage_invd = nullptr;  // [T_max+1][stage_factor_stride(n)] LDL^T inverse pivots per penalty, times 1 / (mu + rho)
   double* shift_c = nullptr;    // [T_max+1] c = rho / (mu + rho) per penalty (shifted W-update operator)
   bf16* N_hi = nullptr;         // [n][n] one fp16 plane of mu I - H~ (operand of the truncated-series W-update), scale in fscal[9..11]
+  bf16* N_lo = nullptr;         // its lo plane (first-order term of the two-term series, which needs two planes)
+  float* series_g = nullptr;    // [T_max+1] per penalty: 1 / (mu + rho) times the inverse scale of the N planes
   float* series_f = nullptr;    // [T_max+1] per penalty: rho / (mu + rho)^2 times the inverse scale of N_hi
   float* Qs32 = nullptr;        // [n][n] fp32 Q (mu I - T), or nullptr: input of the explicit-operator route (p_max > n only)
   double* ps_totals = nullptr;  // [PAIR_BATCH_MAX] totals of the candidate pairs of a pair-swap round

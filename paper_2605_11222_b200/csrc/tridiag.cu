@@ -695,7 +695,7 @@ __global__ void stage_factors_kernel(const double* __restrict__ td, const double
                                      const double* __restrict__ rho, const double* __restrict__ mu_p, int first,
                                      int count, int ept, float* __restrict__ L, float* __restrict__ invD,
                                      double* __restrict__ shift_c, const float* __restrict__ series_inv,
-                                     float* __restrict__ series_f, int* status) {
+                                     float* __restrict__ series_f, float* __restrict__ series_g, int* status) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= count) return;
   const int stage = first + t;
@@ -706,6 +706,7 @@ __global__ void stage_factors_kernel(const double* __restrict__ td, const double
   // truncated series c (I + E), E = (mu I - H~) / (mu + rho): factor of the product R (mu I - H~), with the inverse
   // of the operand plane's scale folded in
   series_f[stage] = (float)(rho[stage] * wshift * wshift * (double)series_inv[0]);
+  series_g[stage] = (float)(wshift * (double)series_inv[0]);   // one more factor E: (c R E) (mu I - H~) / (mu + rho)
   const size_t stride = (size_t)ept * SOLVE_THREADS;
   float* l = L + (size_t)stage * stride;
   float* id = invD + (size_t)stage * stride;
@@ -731,7 +732,7 @@ __global__ void stage_factors_kernel(const double* __restrict__ td, const double
 void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count) {
   stage_factors_kernel<<<(count + 63) / 64, 64, 0, c->stream>>>(c->td, c->te, c->n, rho_dev, c->scal + 8, first,
                                                                count, solve_ept(c->n), c->stage_l, c->stage_invd,
-                                                               c->shift_c, c->fscal + 9, c->series_f, c->status);
+                                                               c->shift_c, c->fscal + 9, c->series_f, c->series_g, c->status);
   c->launches++;
 }
 

@@ -138,10 +138,10 @@ def test_w_update_parity(n, p, gs, kind):
 @pytest.mark.parametrize("n,p", [(520, 264), (1024, 512)])
 def test_w_update_as_truncated_series_at_large_penalties(n, p):
     """rho (H~ + rho I)^{-1} = c (I + E + E^2 + ...), E = (mu I - H~) / (mu + rho) (Eq. 7 rearranged).  The late
-    iterations keep c R + c R E; what they drop is bounded by gamma^2 ||R|| with gamma = max |mu - lambda| / (mu +
-    rho).  Checked against the fp64 W-update of the oracle at penalties on both sides of the solver's switch
-    (gamma <= 2^-13): the error follows gamma^2 where the truncation dominates and sits at the level of the route
-    through the factorisation where it does not."""
+    iterations keep c R + c R E, those before them one more term; what they drop is bounded by gamma^2 ||R||
+    (gamma^3) with gamma = max |mu - lambda| / (mu + rho).  Checked against the fp64 W-update of the oracle at
+    penalties on both sides of the solver's switches (gamma <= 2^-13, 2^-9): the error follows the bound where the
+    truncation dominates and sits at the level of the route through the factorisation where it does not."""
     spec = wl.small_case(n, p, 4096, group_size=0, T=2)
     W = wl.gen_weight(spec, DEV)
     sol = B.Solver(n, p, T_max=2)
@@ -162,19 +162,25 @@ def test_w_update_as_truncated_series_at_large_penalties(n, p):
     args = (W, 0, to_dev(codes, torch.uint8, DEV), to_dev(delta, torch.float32, DEV),
             to_dev(z0, torch.float32, DEV), to_dev(V, torch.float32, DEV))
     spread = max(abs(mu - lam.min()), abs(mu - lam.max()))
-    for gamma in (2.0 ** -6, 2.0 ** -10, 2.0 ** -13, 2.0 ** -16):
+    for gamma in (2.0 ** -6, 2.0 ** -9, 2.0 ** -10, 2.0 ** -13, 2.0 ** -16):
         rho = spread / gamma - mu
         Zo = O.w_update(lam, U, Ws @ Ht, D, V.astype(np.float64), rho) - Ws      # W - W_hat' in fp64
         R = D - V.astype(np.float64) / rho - Ws
-        Zs = np64(sol.w_update_series(*args, rho))
         Ze = np64(sol.w_update_correction(*args, rho))
-        err_series = np.linalg.norm(Zs - Zo) / np.linalg.norm(R)
         err_exact = np.linalg.norm(Ze - Zo) / np.linalg.norm(R)
         assert err_exact <= 4e-7, (gamma, err_exact)
-        # truncation (<= gamma^2 / (1 - gamma)) plus the rounding of a one-plane product of relative size gamma
-        assert err_series <= gamma * gamma / (1 - gamma) + gamma * 2.0 ** -11 + 4e-7, (gamma, err_series)
-        if gamma <= 2.0 ** -13:                                  # where the solver uses it: fp32 resolution
-            assert err_series <= 2.0 ** -22, (gamma, err_series)
+        Z1 = np64(sol.w_update_series(*args, rho, terms=1))
+        Z2 = np64(sol.w_update_series(*args, rho, terms=2))
+        err1 = np.linalg.norm(Z1 - Zo) / np.linalg.norm(R)
+        err2 = np.linalg.norm(Z2 - Zo) / np.linalg.norm(R)
+        # truncation (<= gamma^(terms+1) / (1 - gamma)) plus the rounding of the products: a one-plane product of
+        # relative size gamma (one term), a two-plane one of size gamma and a one-plane one of size gamma^2 (two)
+        assert err1 <= gamma ** 2 / (1 - gamma) + gamma * 2.0 ** -11 + 4e-7, (gamma, err1)
+        assert err2 <= gamma ** 3 / (1 - gamma) + gamma * 2.0 ** -20 + gamma ** 2 * 2.0 ** -11 + 4e-7, (gamma, err2)
+        if gamma <= 2.0 ** -13:                                  # where the solver uses one term: fp32 resolution
+            assert err1 <= 2.0 ** -22, (gamma, err1)
+        if gamma <= 2.0 ** -9:                                   # ... and two terms
+            assert err2 <= 2.0 ** -22, (gamma, err2)
     assert sol.last_device_status() == B.OK
 
 
@@ -604,8 +610,9 @@ def test_fused_and_row_pass_element_update_agree():
     out = []
     for fused in (False, True):
         resid = torch.zeros(spec.T, 2, device=DEV)
+        # (both runs through the factorisation in every iteration: the fused variant has no series route)
         codes, scale, zero, rep = sol.quantize_layer(W, spec.bits, spec.group_size, spec.symmetric, resid=resid,
-                                                     fused_epilogue=fused)
+                                                     fused_epilogue=fused, wupdate_series=1)
         assert sol.last_device_status() == B.OK
         out.append((codes.clone(), scale.clone(), zero.clone(), resid.cpu().numpy(), rep.err_before))
     assert torch.equal(out[0][0], out[1][0])
@@ -668,6 +675,7 @@ def test_one_plane_products_of_the_late_iterations():
     # by default those iterations are evaluated as the truncated series; wupdate_series = 1 keeps them on the
     # factorisation (one-plane products and the row solve)
     assert rep0.one_plane_iters - 1 <= rep0.series_iters <= rep0.one_plane_iters and rep2.series_iters == 0
+    assert rep0.series2_iters >= 5 and rep1.series2_iters == 0 and rep2.series2_iters == 0
     assert rep1.one_plane_iters == rep0.one_plane_iters and rep1.series_iters == 0
     assert (c0.cpu().numpy() == res.admm.codes).mean() >= CODE_AGREEMENT
     assert (c1.cpu().numpy() == res.admm.codes).mean() >= CODE_AGREEMENT
