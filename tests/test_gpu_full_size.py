@@ -64,11 +64,12 @@ def _check_factor(sol, H, s, tol_orth=1e-10, tol_rec=1e-10):
     assert te[-1].item() == 0.0
 
 
-@pytest.mark.parametrize("n", [8, 72, 264, 1000, 4096, 4104, 6144, 12288, 14336])
+@pytest.mark.parametrize("n", [8, 72, 264, 1000, 4096, 4104, 5120, 6144, 12288, 13312, 14336])
 def test_factorisation_properties(n):
     """The one-time factorisation at sizes that cover every code path: tiny and ragged sizes, the benchmark
-    sizes (4096, 12288), sizes that are no multiple of the panel and segment widths (1000, 4104), and the
-    largest supported size."""
+    sizes (4096, 12288), sizes that are no multiple of the panel and segment widths (1000, 4104), the smallest
+    size whose first panels take the lower-triangle sweep (5120), the largest the blocked kernel's shared memory
+    holds (13312), and the largest supported size."""
     p = 8
     N = 2 * wl.CHUNK_ROWS if n >= 4096 else 3 * n + 40
     spec = wl.small_case(n, p, N, group_size=0, T=2)
