@@ -546,12 +546,14 @@ def main():
                       "default_one_plane_iterations": df_rep.one_plane_iters,
                       "default_series_iterations": df_rep.series_iters,
                       "default_two_term_series_iterations": df_rep.series2_iters,
+                      "default_no_product_iterations": df_rep.series0_iters,
                       "err_admm_two_planes": tp_rep.err_before, "err_admm_without_series": ns_rep.err_before,
                       "err_admm_default": df_rep.err_before,
                       "codes_equal_fraction": float((c_two == c_def).float().mean().item()),
                       "codes_equal_fraction_without_series": float((codes == c_def).float().mean().item())}
     n_series = int(df_rep.series_iters)
     n_series2 = int(df_rep.series2_iters)
+    n_series0 = int(df_rep.series0_iters)
     n_one_plane = int(df_rep.one_plane_iters)
 
     # ---- a run whose grid comes from the MSE search for the clipping ratio, 100 candidates down to 0.8
@@ -643,7 +645,8 @@ def main():
     # iteration, of which the first has rows_p1 rows
     # (the two-term series adds one p-row one-plane product per iteration; its two-plane product is timed as
     # a second product, p rows)
-    flops_one_plane = args.steps * 2.0 * n * n * ((n_series + n_series2) * p + (n_one_plane - n_series) * (rows_p1 + p))
+    flops_one_plane = args.steps * 2.0 * n * n * ((n_series + n_series2) * p +
+                                                    (n_one_plane - n_series - n_series0) * (rows_p1 + p))
     executed_flops_per_step = (flops_two_plane + flops_one_plane) / args.steps
     breakdown = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
                  for k, v in timing.items()}
@@ -671,8 +674,8 @@ def main():
         ms, cnt = timing["row_split"]
         if cnt == 0 or ms <= 0:
             return None
-        n_fact = T - n_series - n_series2
-        total = args.steps * (22.0 * p * n * T + 8.0 * p * n * n_series2 +
+        n_fact = T - n_series - n_series2 - n_series0
+        total = args.steps * (22.0 * p * n * T - 4.0 * p * n * n_series0 + 8.0 * p * n * n_series2 +
                               (12.0 * n * n * n_fact if explicit_route else 0.0))
         gbs = total / (ms * 1e-3) / 1e9
         return {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -712,7 +715,7 @@ def main():
         "layers_per_s": world / (ms_step / 1e3),
         "w_update_useful_tflops": 4.0 * n * n * p * T / (w_update_ms * 1e-3) / 1e12,
         "w_update_executed_tflops": executed_flops_per_step / (w_update_ms * 1e-3) / 1e12,
-        "one_plane_iterations": n_one_plane, "series_iterations": n_series, "two_term_series_iterations": n_series2, "w_update_route": "explicit operator" if explicit_route else "two products",
+        "one_plane_iterations": n_one_plane, "series_iterations": n_series, "two_term_series_iterations": n_series2, "no_product_iterations": n_series0, "w_update_route": "explicit operator" if explicit_route else "two products",
         "err_before_local_search": rep.err_before, "err_after_local_search": rep.err_after,
         "local_search_moves": rep.moves, "pair_swap_after_local_search": pair_swap, "admm_with_grid_refresh": grid_refresh,
         "admm_with_mse_clip_search": mse_clip, "admm_with_fused_epilogue": fused_variant,

@@ -187,7 +187,8 @@ typedef struct {
                            (in effect the iterations that run on one plane) the update is evaluated as c R + c R E --
                            ONE product with the fixed operand mu I - H~ instead of two products and a row solve; for
                            2^-13 < ||E|| <= 2^-9 as c R + c R E + c R E^2 -- the first product on two planes, the
-                           second (of relative size ||E||^2) on one.  The dropped terms are below 2^-26 of the
+                           second (of relative size ||E||^2) on one; and once ||E|| <= 2^-26 as c R alone, without a
+                           product.  The dropped terms are below 2^-26 of the
                            right-hand side, under the fp32 resolution of the stored iterate.  1: never (every
                            iteration goes through the factorisation).  Ignored with product_planes = 2 or
                            fused_epilogue = 1, which keep every iteration on the two-plane route through the
@@ -204,6 +205,7 @@ typedef struct {
   int one_plane_iters;  /* quantize_layer: iterations whose products ran on one fp16 plane per operand */
   int series_iters;     /* quantize_layer: iterations evaluated as the series with one term of E (one product) */
   int series2_iters;    /* quantize_layer: iterations evaluated as the series with two terms of E (two products) */
+  int series0_iters;    /* quantize_layer: iterations evaluated as c R alone (||E|| <= 2^-26: no product) */
 } admmq_report;
 admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out,
                                   const admmq_quant_cfg* cfg, unsigned char* d_codes, float* d_scale,

@@ -31,7 +31,7 @@ admmq_status admmq_test_w_update_correction(admmq_ctx* ctx, const float* d_W0, i
                                             const float* d_zero, const float* d_V, double rho, float* d_Z_out);
 
 /* The same correction evaluated as the later iterations do it (admmq_quant_cfg.wupdate_series): the series
- * c (I + E + E^2 + ...) R with `terms` = 1 or 2 terms of E kept, on the fixed operand mu I - H~, whatever ||E|| is
+ * c (I + E + E^2 + ...) R with `terms` = 0, 1 or 2 terms of E kept, on the fixed operand mu I - H~, whatever ||E|| is
  * at this penalty.  For a test that compares it with the route through the factorisation on both sides of the
  * penalties where the solver would switch to it.  ADMMQ_ERR_INVALID_ARG for any other `terms`. */
 admmq_status admmq_test_w_update_series(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,

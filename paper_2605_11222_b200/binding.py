@@ -65,7 +65,7 @@ class Report(C.Structure):
     _fields_ = [("err_before", C.c_double), ("err_after", C.c_double), ("moves", C.c_longlong),
                 ("iters_run", C.c_int), ("capped_columns", C.c_int), ("ms", C.c_float),
                 ("refreshed_iter", C.c_int), ("one_plane_iters", C.c_int), ("series_iters", C.c_int),
-                ("series2_iters", C.c_int)]
+                ("series2_iters", C.c_int), ("series0_iters", C.c_int)]
 
 
 class AdmmqError(RuntimeError):

@@ -418,6 +418,8 @@ admmq_status admmq_factor(admmq_ctx* ctx, const admmq_factor_cfg* cfg) {
     // one term of E (one plane) once ||E|| <= 2^-13; two terms -- the first on two planes, the second, of relative
     // size ||E||^2, on one -- once ||E|| <= 2^-9 (remainder below ||E||^3 <= 2^-27)
     c->series_host[t] = !isfinite(e) ? 0 : (c->planes_host[t] == 1 && e <= 1.0 / 8192.0) ? 1 : (e <= 1.0 / 512.0 ? 2 : 0);
+    // ... and no term at all once ||E|| itself is below 2^-26: the W-update is c R to the same accuracy
+    if (c->series_host[t] == 1 && e <= 1.0 / 67108864.0) c->series_host[t] = 3;
   }
   c->state = 2;
   return ADMMQ_OK;
@@ -602,7 +604,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.n_groups = n / gs;
   e.kmax = (1 << cfg->bits) - 1;
   e.Rnext = c->Y;                                          // Y is free once its planes exist
-  int one_plane_iters = 0, series_iters = 0, series2_iters = 0;
+  int one_plane_iters = 0, series_iters = 0, series2_iters = 0, series0_iters = 0;
   const bool series = cfg->wupdate_series == 0 && !cfg->fused_epilogue && cfg->product_planes != 2;
   auto series_of = [&](int t) { return series ? (int)c->series_host[t] : 0; };
   for (int t = 0; t < T; ++t) {
@@ -617,11 +619,13 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     const int planes = (cfg->product_planes == 2 || cfg->fused_epilogue) ? 2 : c->planes_host[t];
     one_plane_iters += planes == 1;
     // terms of E this iteration's W-update keeps (0: through the factorisation)
-    const int series_t = series_of(t);
-    series_iters += series_t == 1;
-    series2_iters += series_t == 2;
+    int series_t = series_of(t);
     bool refresh = false;
     for (int q = 0; q < cfg->n_refresh; ++q) refresh = refresh || (cfg->h_refresh_iters[q] == t);
+    if (series_t == 3 && refresh) series_t = 1;             // a refresh attempt wants the product stored
+    series_iters += series_t == 1;
+    series2_iters += series_t == 2;
+    series0_iters += series_t == 3;
     if (refresh) {
       // grid refresh attempt: z = W^(t+1) - W_hat' is stored by the plain epilogue, then evaluated on both grids
       EpiParams w = e;
@@ -648,7 +652,10 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
       w.kind = EPI_STORE;
       w.C = c->Y;
       w.ldc = n;
-      if (w_update_any(ctx, p, t, w, explicit_op, planes, series_t) != cudaSuccess) return ADMMQ_ERR_CUDA;
+      if (series_t == 3)
+        w.C = nullptr;                                       // W^(t+1) - W_hat' = c R: nothing to add in the row pass
+      else if (w_update_any(ctx, p, t, w, explicit_op, planes, series_t) != cudaSuccess)
+        return ADMMQ_ERR_CUDA;
       Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
       w.kind = EPI_ADMM;
       // the lo plane of the next right-hand side is written only if the next iteration's products read it
@@ -678,6 +685,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   h_report->one_plane_iters = one_plane_iters;
   h_report->series_iters = series_iters;
   h_report->series2_iters = series2_iters;
+  h_report->series0_iters = series0_iters;
   return st;
 }
 
@@ -701,11 +709,12 @@ admmq_status admmq_test_w_update_series(admmq_ctx* ctx, const float* d_W0, int d
                                         const unsigned char* d_codes, const float* d_scale,
                                         const float* d_zero, const float* d_V, double rho, int terms,
                                         float* d_Z_out) {
-  if (terms != 1 && terms != 2) return ADMMQ_ERR_INVALID_ARG;
-  return w_update_call(ctx, d_W0, d_out, group_size, d_codes, d_scale, d_zero, d_V, rho, d_Z_out, 1 + terms);
+  if (terms < 0 || terms > 2) return ADMMQ_ERR_INVALID_ARG;
+  return w_update_call(ctx, d_W0, d_out, group_size, d_codes, d_scale, d_zero, d_V, rho, d_Z_out, terms == 0 ? 4 : 1 + terms);
 }
 
-// correction_only: 0 the whole W-update, 1 the correction W - W_hat', 2 / 3 the correction by the series with one / two terms of E
+// correction_only: 0 the whole W-update, 1 the correction W - W_hat', 2 / 3 / 4 the correction by the series with
+// one / two / no terms of E
 static admmq_status w_update_call(admmq_ctx* ctx, const float* d_W0, int d_out, int group_size,
                                   const unsigned char* d_codes, const float* d_scale, const float* d_zero,
                                   const float* d_V, double rho, float* d_W_out, int correction_only) {
@@ -728,9 +737,10 @@ static admmq_status w_update_call(admmq_ctx* ctx, const float* d_W0, int d_out, 
   e.kind = EPI_STORE;
   e.C = c->Y;                                               // free once its planes exist
   e.ldc = n;
-  const cudaError_t err = correction_only == 2   ? w_update_series(ctx, p, stage, e)
-                          : correction_only == 3 ? w_update_series2(ctx, p, stage, e)
-                                                 : w_update_products(ctx, p, stage, e, 2);
+  const cudaError_t err = correction_only == 2            ? w_update_series(ctx, p, stage, e)
+                          : correction_only == 3            ? w_update_series2(ctx, p, stage, e)
+                          : correction_only == 4            ? cudaMemsetAsync(c->Y, 0, (size_t)p * n * sizeof(float), c->stream)
+                                                            : w_update_products(ctx, p, stage, e, 2);
   if (err != cudaSuccess) return ADMMQ_ERR_CUDA;
   launch_w_out(c, d_W0, p, gs, d_codes, d_scale, d_zero, d_V, 1.0 / rho, c->shift_c + stage, c->Y, d_W_out,
                correction_only != 0);

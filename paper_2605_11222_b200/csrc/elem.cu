@@ -974,7 +974,8 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
     const float* zr = P.zero + (size_t)j * P.n_groups;
     float m = 0.0f;
     for (int i = threadIdx.x * 4; i < n; i += ROW_THREADS * 4) {          // n is a multiple of 8
-      const float4 z = *reinterpret_cast<const float4*>(P.C + base + i);
+      // P.C == nullptr: the product's part of the W-update is below fp32 resolution and was not formed
+      const float4 z = P.C ? *reinterpret_cast<const float4*>(P.C + base + i) : make_float4(0.f, 0.f, 0.f, 0.f);
       const float4 wh = *reinterpret_cast<const float4*>(P.W0 + base + i);
       const float4 v = *reinterpret_cast<const float4*>(P.V + base + i);
       const float4 sv = *reinterpret_cast<const float4*>(P.s + i);

@@ -162,7 +162,7 @@ def test_w_update_as_truncated_series_at_large_penalties(n, p):
     args = (W, 0, to_dev(codes, torch.uint8, DEV), to_dev(delta, torch.float32, DEV),
             to_dev(z0, torch.float32, DEV), to_dev(V, torch.float32, DEV))
     spread = max(abs(mu - lam.min()), abs(mu - lam.max()))
-    for gamma in (2.0 ** -6, 2.0 ** -9, 2.0 ** -10, 2.0 ** -13, 2.0 ** -16):
+    for gamma in (2.0 ** -6, 2.0 ** -9, 2.0 ** -10, 2.0 ** -13, 2.0 ** -16, 2.0 ** -26, 2.0 ** -29):
         rho = spread / gamma - mu
         Zo = O.w_update(lam, U, Ws @ Ht, D, V.astype(np.float64), rho) - Ws      # W - W_hat' in fp64
         R = D - V.astype(np.float64) / rho - Ws
@@ -177,6 +177,11 @@ def test_w_update_as_truncated_series_at_large_penalties(n, p):
         # relative size gamma (one term), a two-plane one of size gamma and a one-plane one of size gamma^2 (two)
         assert err1 <= gamma ** 2 / (1 - gamma) + gamma * 2.0 ** -11 + 4e-7, (gamma, err1)
         assert err2 <= gamma ** 3 / (1 - gamma) + gamma * 2.0 ** -20 + gamma ** 2 * 2.0 ** -11 + 4e-7, (gamma, err2)
+        Z0 = np64(sol.w_update_series(*args, rho, terms=0))      # c R alone
+        err0 = np.linalg.norm(Z0 - Zo) / np.linalg.norm(R)
+        assert err0 <= gamma / (1 - gamma) + 4e-7, (gamma, err0)
+        if gamma <= 2.0 ** -26:                                  # where the solver drops the product
+            assert err0 <= 2.0 ** -22, (gamma, err0)
         if gamma <= 2.0 ** -13:                                  # where the solver uses one term: fp32 resolution
             assert err1 <= 2.0 ** -22, (gamma, err1)
         if gamma <= 2.0 ** -9:                                   # ... and two terms
@@ -674,7 +679,8 @@ def test_one_plane_products_of_the_late_iterations():
     assert 10 <= rep0.one_plane_iters < spec.T and rep2.one_plane_iters == 0
     # by default those iterations are evaluated as the truncated series; wupdate_series = 1 keeps them on the
     # factorisation (one-plane products and the row solve)
-    assert rep0.one_plane_iters - 1 <= rep0.series_iters <= rep0.one_plane_iters and rep2.series_iters == 0
+    assert rep0.one_plane_iters - 1 <= rep0.series_iters + rep0.series0_iters <= rep0.one_plane_iters
+    assert rep2.series_iters == 0 and rep2.series0_iters == 0 and rep1.series0_iters == 0
     assert rep0.series2_iters >= 5 and rep1.series2_iters == 0 and rep2.series2_iters == 0
     assert rep1.one_plane_iters == rep0.one_plane_iters and rep1.series_iters == 0
     assert (c0.cpu().numpy() == res.admm.codes).mean() >= CODE_AGREEMENT
