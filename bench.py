@@ -675,7 +675,8 @@ def main():
         if cnt == 0 or ms <= 0:
             return None
         n_fact = T - n_series - n_series2 - n_series0
-        total = args.steps * (22.0 * p * n * T - 4.0 * p * n * n_series0 + 8.0 * p * n * n_series2 +
+        # (an iteration without a product reads no z, and its predecessor writes no plane for it: 16 instead of 22)
+        total = args.steps * (22.0 * p * n * T - 6.0 * p * n * n_series0 + 8.0 * p * n * n_series2 +
                               (12.0 * n * n * n_fact if explicit_route else 0.0))
         gbs = total / (ms * 1e-3) / 1e9
         return {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -607,6 +607,11 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
   int one_plane_iters = 0, series_iters = 0, series2_iters = 0, series0_iters = 0;
   const bool series = cfg->wupdate_series == 0 && !cfg->fused_epilogue && cfg->product_planes != 2;
   auto series_of = [&](int t) { return series ? (int)c->series_host[t] : 0; };
+  auto refresh_at = [&](int t) {
+    for (int q = 0; q < cfg->n_refresh; ++q)
+      if (cfg->h_refresh_iters[q] == t) return true;
+    return false;
+  };
   for (int t = 0; t < T; ++t) {
     const double rho = c->rho_host[t];
     const double rho_next = (t + 1 < T) ? c->rho_host[t + 1] : rho;
@@ -620,8 +625,7 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
     one_plane_iters += planes == 1;
     // terms of E this iteration's W-update keeps (0: through the factorisation)
     int series_t = series_of(t);
-    bool refresh = false;
-    for (int q = 0; q < cfg->n_refresh; ++q) refresh = refresh || (cfg->h_refresh_iters[q] == t);
+    const bool refresh = refresh_at(t);
     if (series_t == 3 && refresh) series_t = 1;             // a refresh attempt wants the product stored
     series_iters += series_t == 1;
     series2_iters += series_t == 2;
@@ -661,7 +665,10 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
       // the lo plane of the next right-hand side is written only if the next iteration's products read it
       const bool next_two = t + 1 >= T || cfg->product_planes == 2 || series_of(t + 1) == 2 ||
                             (series_of(t + 1) == 0 && c->planes_host[t + 1] != 1);
-      launch_admm_rows(c, w, p, c->R_hi, next_two ? c->R_lo : nullptr, c->rs_R);
+      // ... and none of its planes when the next iteration forms no product (or there is none): the element update
+      // rebuilds R from the codes and the dual
+      const bool next_none = t + 1 >= T || (series_of(t + 1) == 3 && !refresh_at(t + 1));
+      launch_admm_rows(c, w, p, next_none ? nullptr : c->R_hi, next_two && !next_none ? c->R_lo : nullptr, c->rs_R);
     }
   }
   if (d_resid) launch_reduce_partials(c, T, d_resid);

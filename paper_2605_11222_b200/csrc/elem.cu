@@ -1000,11 +1000,13 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
       }
       *reinterpret_cast<uchar4*>(P.codes + base + i) = make_uchar4(e0.code, e1.code, e2.code, e3.code);
       *reinterpret_cast<float4*>(P.V + base + i) = make_float4(e0.v_new, e1.v_new, e2.v_new, e3.v_new);
-      *reinterpret_cast<float4*>(rowbuf + i) = make_float4(e0.r_next, e1.r_next, e2.r_next, e3.r_next);
-      m = fmaxf(fmaxf(fabsf(e0.r_next), fabsf(e1.r_next)), fmaxf(m, fmaxf(fabsf(e2.r_next), fabsf(e3.r_next))));
       r2 += (e0.dr2 + e1.dr2) + (e2.dr2 + e3.dr2);
       s2 += (e0.ds2 + e1.ds2) + (e2.ds2 + e3.ds2);
+      if (!hi) continue;                                   // no product reads the next right-hand side: no planes
+      *reinterpret_cast<float4*>(rowbuf + i) = make_float4(e0.r_next, e1.r_next, e2.r_next, e3.r_next);
+      m = fmaxf(fmaxf(fabsf(e0.r_next), fabsf(e1.r_next)), fmaxf(m, fmaxf(fabsf(e2.r_next), fabsf(e3.r_next))));
     }
+    if (!hi) continue;                                     // (uniform in the grid)
     m = block_max(m, scratch);
     float inv;
     const float sc = pow2_scale_for(m, &inv);
