@@ -675,9 +675,9 @@ def main():
         if cnt == 0 or ms <= 0:
             return None
         n_fact = T - n_series - n_series2 - n_series0
-        # (an iteration without a product reads no z, and its predecessor writes no plane for it: 16 instead of 22)
-        total = args.steps * (22.0 * p * n * T - 6.0 * p * n * n_series0 + 8.0 * p * n * n_series2 +
-                              (12.0 * n * n * n_fact if explicit_route else 0.0))
+        # (the last iterations, which form no product, are one pass over the state: 18 p n bytes for all of them)
+        total = args.steps * (22.0 * p * n * (T - n_series0) + (18.0 * p * n if n_series0 else 0.0) +
+                              8.0 * p * n * n_series2 + (12.0 * n * n * n_fact if explicit_route else 0.0))
         gbs = total / (ms * 1e-3) / 1e9
         return {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": gbs / peaks["hbm_gbs"], "launches": cnt, "avg_launch_ms": ms / cnt}

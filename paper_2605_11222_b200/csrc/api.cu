@@ -612,7 +612,18 @@ admmq_status admmq_quantize_layer(admmq_ctx* ctx, const float* d_W0, int d_out, 
       if (cfg->h_refresh_iters[q] == t) return true;
     return false;
   };
+  // the run's last iterations, if none of them forms a product (or is a refresh attempt), go in one pass
+  int t_tail = T;
+  while (t_tail > 1 && series_of(t_tail - 1) == 3 && !refresh_at(t_tail - 1)) --t_tail;
+  if (T - t_tail < 2) t_tail = T;
   for (int t = 0; t < T; ++t) {
+    if (t == t_tail) {
+      Timed tt(ctx, ADMMQ_T_ROW_SPLIT);
+      launch_admm_tail(c, e, p, ctx->rho_dev, t, T - t, T);
+      one_plane_iters += T - t;
+      series0_iters += T - t;
+      break;
+    }
     const double rho = c->rho_host[t];
     const double rho_next = (t + 1 < T) ? c->rho_host[t + 1] : rho;
     e.first_iter = (t == 0);

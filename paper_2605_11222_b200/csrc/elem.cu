@@ -1029,6 +1029,110 @@ admm_row_kernel(EpiParams P, int p, int n, bf16* __restrict__ hi, bf16* __restri
   }
 }
 
+// The last iterations of a run, in which no product is formed (||E|| <= 2^-26: W - W_hat' = c R): every element
+// then evolves on its own -- R is rebuilt from its code and dual, the update reads nothing else -- so `count`
+// iterations starting at `first` run in one pass over the state, the element held in registers throughout.  Same
+// arithmetic per element and iteration as admm_row_kernel.  The residual sums of every iteration (Theorem 1) are
+// taken per warp in shared memory and written per CTA at the end, in a fixed order.
+constexpr int TAIL_MAX = 512;                 // iterations per launch (shared memory: 8 warps x 2 sums each)
+__global__ void __launch_bounds__(256)
+admm_tail_kernel(EpiParams P, long long total, int n, const double* __restrict__ rho, const double* __restrict__ shift_c,
+                 int first, int count, int T, float* __restrict__ partials, int slots) {
+  __shared__ float it_rho[TAIL_MAX], it_inv[TAIL_MAX], it_inv_next[TAIL_MAX], it_c[TAIL_MAX];
+  __shared__ float wsum[8][TAIL_MAX][2];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int q = threadIdx.x; q < count; q += blockDim.x) {
+    const int t = first + q;
+    const double r = rho[t], rn = rho[t + 1 < T ? t + 1 : t];
+    it_rho[q] = (float)r;
+    it_inv[q] = (float)(1.0 / r);
+    it_inv_next[q] = (float)(1.0 / rn);
+    it_c[q] = (float)shift_c[t];
+  }
+  for (int q = threadIdx.x; q < 8 * count; q += blockDim.x) {
+    wsum[q / count][q % count][0] = 0.0f;
+    wsum[q / count][q % count][1] = 0.0f;
+  }
+  __syncthreads();
+  const int gs = P.group_size;
+  // whole warps take part in the butterflies: the loop bound is rounded up to a multiple of the grid's stride
+  const long long groups = total / 4, stride = (long long)gridDim.x * blockDim.x;
+  for (long long g0 = (long long)blockIdx.x * blockDim.x; g0 < groups; g0 += stride) {
+    const long long gq = g0 + threadIdx.x;
+    const bool live = gq < groups;
+    const long long idx = live ? gq * 4 : 0;
+    const int col = (int)(idx % n);
+    const long long row = idx / n;
+    const float4 w4 = *reinterpret_cast<const float4*>(P.W0 + idx);
+    float4 v4 = *reinterpret_cast<const float4*>(P.V + idx);
+    const float4 s4 = *reinterpret_cast<const float4*>(P.s + col);
+    const float4 i4 = *reinterpret_cast<const float4*>(P.inv_s + col);
+    uchar4 k4 = *reinterpret_cast<const uchar4*>(P.codes + idx);
+    GridG gg[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const long long gi = row * P.n_groups + (col + e) / gs;
+      gg[e] = grid_g(P.delta[gi], P.zero[gi]);
+    }
+    float w[4] = {w4.x, w4.y, w4.z, w4.w}, v[4] = {v4.x, v4.y, v4.z, v4.w};
+    const float sv[4] = {s4.x, s4.y, s4.z, s4.w}, si[4] = {i4.x, i4.y, i4.z, i4.w};
+    int k[4] = {k4.x, k4.y, k4.z, k4.w};
+    IterF it;
+    it.first_iter = 0;
+    it.kmax = P.kmax;
+    for (int q = 0; q < count; ++q) {
+      it.rho = it_rho[q];
+      it.inv_rho = it_inv[q];
+      it.inv_rho_next = it_inv_next[q];
+      const float cs = it_c[q];
+      float r2 = 0.f, s2 = 0.f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const AdmmElem o = admm_elem(0.0f, w[e], v[e], k[e], sv[e], si[e], gg[e], gg[e], cs, it);
+        v[e] = o.v_new;
+        k[e] = o.code;
+        r2 += o.dr2;
+        s2 += o.ds2;
+      }
+      if (!live) r2 = s2 = 0.f;
+      r2 = warp_sum(r2);
+      s2 = warp_sum(s2);
+      if (lane == 0) {
+        wsum[warp][q][0] += r2;
+        wsum[warp][q][1] += s2;
+      }
+    }
+    if (live) {
+      *reinterpret_cast<float4*>(P.V + idx) = make_float4(v[0], v[1], v[2], v[3]);
+      *reinterpret_cast<uchar4*>(P.codes + idx) = make_uchar4(k[0], k[1], k[2], k[3]);
+    }
+  }
+  __syncthreads();
+  for (int q = threadIdx.x; q < count; q += blockDim.x) {
+    float a = 0.f, b = 0.f;
+    for (int wq = 0; wq < 8; ++wq) {
+      a += wsum[wq][q][0];
+      b += wsum[wq][q][1];
+    }
+    float* ps = partials + ((size_t)(first + q) * slots + blockIdx.x) * 2;
+    ps[0] = a;
+    ps[1] = b;
+  }
+}
+
+// Iterations [first, first + count) of a run, none of which forms a product (and none is the first).
+void launch_admm_tail(Ctx* c, const EpiParams& P, int p, const double* rho_dev, int first, int count, int T) {
+  const long long total = (long long)p * c->n;
+  int blocks = c->num_sms * 4;
+  if (blocks > c->partial_slots) blocks = c->partial_slots;
+  for (int done = 0; done < count; done += TAIL_MAX) {
+    const int m = count - done < TAIL_MAX ? count - done : TAIL_MAX;
+    admm_tail_kernel<<<blocks, 256, 0, c->stream>>>(P, total, c->n, rho_dev, c->shift_c, first + done, m, T,
+                                                   c->partials, c->partial_slots);
+    LAUNCH(c);
+  }
+}
+
 void launch_admm_rows(Ctx* c, const EpiParams& P, int p, bf16* hi, bf16* lo, float* row_inv) {
   const size_t smem = (size_t)c->n * sizeof(float);
   if (ensure_dynamic_smem((const void*)admm_row_kernel, 64 * 1024) != cudaSuccess) return;   // the launch error check reports it

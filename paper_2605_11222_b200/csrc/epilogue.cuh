@@ -95,13 +95,30 @@ __device__ __forceinline__ void diff_exact(float w0, float z0, float& hi, float&
 __device__ __forceinline__ float grid_offset(float s, float dl, float k, float a_hi, float a_lo) {
   const float p = __fmul_rn(dl, k);
   const float pe = __fmaf_rn(dl, k, -p);                  // Delta k = p + pe exactly
-  return s * __fsub_rn(__fadd_rn(__fsub_rn(p, a_hi), pe), a_lo);
+  // (the product by s rounds once, here: left to the compiler it may be contracted into the caller's next
+  // subtraction, and two evaluations of the same grid point would then no longer cancel exactly)
+  return __fmul_rn(s, __fsub_rn(__fadd_rn(__fsub_rn(p, a_hi), pe), a_lo));
 }
 
 // g: the grid the new code is taken on; g_old: the grid code_old refers to (the same one, except in the
 // iteration that accepts a grid refresh).
+// The iteration's scalars in the precision the update uses them in.
+struct IterF {
+  float rho, inv_rho, inv_rho_next;
+  int first_iter, kmax;
+};
+__device__ __forceinline__ IterF iter_f(const EpiParams& P) {
+  IterF q;
+  q.rho = (float)P.rho;
+  q.inv_rho = (float)P.inv_rho;
+  q.inv_rho_next = (float)P.inv_rho_next;
+  q.first_iter = P.first_iter;
+  q.kmax = P.kmax;
+  return q;
+}
+
 __device__ __forceinline__ AdmmElem admm_elem(float zp, float w0, float v, int code_old, float s, float inv_s,
-                                              const GridG& g, const GridG& g_old, float cshift, const EpiParams& P) {
+                                              const GridG& g, const GridG& g_old, float cshift, const IterF& P) {
   AdmmElem o;
   float a_hi, a_lo;
   diff_exact(w0, g.z0, a_hi, a_lo);
@@ -111,7 +128,7 @@ __device__ __forceinline__ AdmmElem admm_elem(float zp, float w0, float v, int c
     if (g_old.z0 != g.z0) diff_exact(w0, g_old.z0, b_hi, b_lo);
     e_old = grid_offset(s, g_old.dl, (float)code_old, b_hi, b_lo);
   }
-  const float inv_rho = (float)P.inv_rho;
+  const float inv_rho = P.inv_rho;
   // z = c R + (product output), R = D^(t) - V/rho - W_hat' exactly as the right-hand side was formed
   const float z = fmaf(cshift, fmaf(-v, inv_rho, e_old), zp);
   const float u = fmaf(v, inv_rho, z) * inv_s;             // (W~ - W_hat') / s: target minus weight  (Eq. 8)
@@ -124,11 +141,15 @@ __device__ __forceinline__ AdmmElem admm_elem(float zp, float w0, float v, int c
   const float wd = z - e_new;                              // W^(t+1) - D^(t+1)
   const float dd = e_new - e_old;                          // D^(t+1) - D^(t)
   o.code = (unsigned char)(int)k;
-  o.v_new = fmaf((float)P.rho, wd, v);                     // V += rho (W - D)               (Eq. 9)
-  o.r_next = fmaf(-o.v_new, (float)P.inv_rho_next, e_new); // next R = D - V/rho' - W_hat'
+  o.v_new = fmaf(P.rho, wd, v);                            // V += rho (W - D)               (Eq. 9)
+  o.r_next = fmaf(-o.v_new, P.inv_rho_next, e_new);        // next R = D - V/rho' - W_hat'
   o.dr2 = wd * wd;
   o.ds2 = dd * dd;
   return o;
+}
+__device__ __forceinline__ AdmmElem admm_elem(float zp, float w0, float v, int code_old, float s, float inv_s,
+                                              const GridG& g, const GridG& g_old, float cshift, const EpiParams& P) {
+  return admm_elem(zp, w0, v, code_old, s, inv_s, g, g_old, cshift, iter_f(P));
 }
 
 // Scalar epilogue for one output element (used by the SIMT kernel and for ragged edges).

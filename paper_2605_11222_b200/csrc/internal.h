@@ -146,6 +146,7 @@ size_t tridiag_blocked_scratch_doubles(int n);
 cudaError_t tridiag_form_qt(Ctx* c);                // reflectors -> P64 = Q^T
 size_t stage_factor_stride(int n);                  // floats per penalty in stage_l / stage_invd
 void launch_stage_factors(Ctx* c, const double* rho_dev, int first, int count);
+void launch_admm_tail(Ctx* c, const EpiParams& P, int p, const double* rho_dev, int first, int count, int T);
 void launch_series_operand(Ctx* c);   // A64 = H~ (before the reduction overwrites it) -> N_hi, fscal[9..11]; mean of its diagonal -> scal[11]
 void launch_tridiag_solve(Ctx* c, const float* Y, int p, int stage, bf16* hi, bf16* lo, float* row_inv);
 
