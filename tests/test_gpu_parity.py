@@ -662,9 +662,10 @@ def test_explicit_operator_route_against_oracle_and_two_product_route(kw):
 
 def test_one_plane_products_of_the_late_iterations():
     """Once the penalty is large the products carry a part of the W-update so small that one fp16 plane per
-    operand resolves it below fp32: the default run switches there, a run forced to two planes does not, and
-    both give the oracle's codes."""
-    spec = wl.small_case(d_in=520, d_out=264, n_tokens=4096, bits=4, group_size=0, T=90, gamma=1.25)
+    operand resolves it below fp32, then so small that a truncated series replaces the route through the
+    factorisation, and at the end none at all: the default run switches there, a run forced to two planes does
+    not, a run without the series keeps the factorisation, and all give the oracle's codes."""
+    spec = wl.small_case(d_in=520, d_out=264, n_tokens=4096, bits=4, group_size=0, T=130, gamma=1.25)
     W = wl.gen_weight(spec, DEV)
     sol = B.Solver(spec.d_in, spec.d_out, T_max=spec.T)
     sol.hessian_reset()
@@ -681,6 +682,7 @@ def test_one_plane_products_of_the_late_iterations():
     # factorisation (one-plane products and the row solve)
     assert rep0.one_plane_iters - 1 <= rep0.series_iters + rep0.series0_iters <= rep0.one_plane_iters
     assert rep2.series_iters == 0 and rep2.series0_iters == 0 and rep1.series0_iters == 0
+    assert rep0.series0_iters >= 5                          # the run ends with iterations that form no product
     assert rep0.series2_iters >= 5 and rep1.series2_iters == 0 and rep2.series2_iters == 0
     assert rep1.one_plane_iters == rep0.one_plane_iters and rep1.series_iters == 0
     assert (c0.cpu().numpy() == res.admm.codes).mean() >= CODE_AGREEMENT
