@@ -507,6 +507,8 @@ def test_pair_swap_parity(kw):
     (dict(d_in=512, d_out=384, n_tokens=6144), list(range(1, 40))),          # g128, asym: first accepted attempt
     (dict(d_in=264, d_out=70, n_tokens=3000, bits=2, group_size=0, symmetric=True), [4]),
     (dict(d_in=256, d_out=64, n_tokens=2048, group_size=64), [0]),            # at t = 0 the refit sees W_hat: no change
+    # a long schedule: an attempt inside the last iterations, which otherwise form no product and run in one pass
+    (dict(d_in=256, d_out=96, n_tokens=2048, group_size=64, T=130, gamma=1.25), [3, 126]),
 ])
 def test_grid_refresh_parity(kw, attempts):
     spec = wl.small_case(**kw)
