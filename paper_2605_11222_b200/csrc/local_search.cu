@@ -1,6 +1,7 @@
 // Greedy single-entry local search (Sec. 3.5; Eq. 11 with the second perturbation zero).
-// One CTA per output channel: its gradient g = H (w_q - w_hat), its codes and diag(H) stay in shared
-// memory (the diagonal as Delta_i^2 H_ii, the quadratic term of a move); every step scans the 2 n
+// One CTA per output channel: its gradient g = H (w_q - w_hat) and its codes stay in shared memory (the
+// quadratic term of a move, Delta_i^2 H_ii, is formed from the cached diagonal on the fly: five bytes per entry
+// instead of nine let more channels share an SM); every step scans the 2 n
 // candidate moves, a block-wide argmin picks the best one, and the gradient takes the rank-1 correction g += d H[:, i] (row i of the symmetric H, contiguous).
 #include "internal.h"
 
@@ -34,8 +35,7 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
                     long long* __restrict__ moves_out, int* __restrict__ capped_out) {
   extern __shared__ float smf[];
   float* g = smf;                  // [n]
-  float* quad = smf + n;           // [n]  Delta_i^2 H_ii, the quadratic term of a move of entry i
-  float* sdl = smf + 2 * n;        // [n / gs]  this channel's Delta per group
+  float* sdl = smf + n;            // [n / gs]  this channel's Delta per group
   float* szr = sdl + n / gs;       // [n / gs]  this channel's z0 per group
   unsigned char* kc = (unsigned char*)(szr + n / gs);   // [n]
   __shared__ Cand wbest[16];
@@ -57,9 +57,7 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
     szr[i] = zero[(long long)j * ng + i];
   }
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
-    const float d = dl[i / gs];
     g[i] = g_glob[(long long)j * n + i];
-    quad[i] = d * d * hdiag[i];
     kc[i] = codes[(long long)j * n + i];
   }
   __syncthreads();
@@ -80,7 +78,7 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
     // four consecutive entries per step (n is a multiple of 8)
     for (int i4 = threadIdx.x * 4; i4 < n; i4 += blockDim.x * 4) {
       float4 g4 = *reinterpret_cast<const float4*>(g + i4);
-      const float4 q4 = *reinterpret_cast<const float4*>(quad + i4);
+      const float4 q4 = __ldg(reinterpret_cast<const float4*>(hdiag + i4));   // H_ii; times Delta_i^2 below
       uchar4 k4 = *reinterpret_cast<const uchar4*>(kc + i4);
       if (i_move >= 0) {
         const float4 h4 = *reinterpret_cast<const float4*>(hrow + i4);   // g += d H[:, i_move] (H symmetric)
@@ -107,8 +105,9 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
         const int i = i4 + e;
         if (e > 0 && (gs & 3) != 0) d = sdl[shift >= 0 ? (i >> shift) : (i / gs)];
         const float lin = 2.0f * d * gv[e];
-        const float cp = kv[e] < kmax ? lin + qv[e] : INFINITY;
-        const float cm = kv[e] > 0 ? qv[e] - lin : INFINITY;
+        const float qd = d * d * qv[e];                     // Delta_i^2 H_ii, the quadratic term of a move of entry i
+        const float cp = kv[e] < kmax ? lin + qd : INFINITY;
+        const float cm = kv[e] > 0 ? qd - lin : INFINITY;
         second = fminf(second, fmaxf(cp, best.cost));
         if (cp < best.cost) {
           best.cost = cp;
@@ -146,8 +145,10 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
       tie_count = 0;
       if (b.idx != 0x7fffffff) {
         const int i = b.idx >> 1;
-        const float thr = -tau * quad[i];
-        const float tol = TIE_MARGIN * fmaxf(fabsf(b.cost), quad[i]);
+        const float di = sdl[shift >= 0 ? (i >> shift) : (i / gs)];
+        const float qi = di * di * hdiag[i];
+        const float thr = -tau * qi;
+        const float tol = TIE_MARGIN * fmaxf(fabsf(b.cost), qi);
         if (sec - b.cost <= tol || fabsf(b.cost - thr) <= tol) {   // too close to call in fp32
           tie_on = 1;
           tie_limit = b.cost + tol;
@@ -166,11 +167,12 @@ local_search_kernel(const float* __restrict__ H, const float* __restrict__ hdiag
         const float d = sdl[shift >= 0 ? (i >> shift) : (i / gs)];
         const float lin = 2.0f * d * g[i];
         const int k = kc[i];
-        if (k < kmax && lin + quad[i] <= lim) {
+        const float qi = d * d * hdiag[i];
+        if (k < kmax && lin + qi <= lim) {
           const int slot = atomicAdd(&tie_count, 1);
           if (slot < TIE_SLOTS) tie_idx[slot] = 2 * i;
         }
-        if (k > 0 && quad[i] - lin <= lim) {
+        if (k > 0 && qi - lin <= lim) {
           const int slot = atomicAdd(&tie_count, 1);
           if (slot < TIE_SLOTS) tie_idx[slot] = 2 * i + 1;
         }
@@ -243,7 +245,7 @@ cudaError_t launch_local_search(Ctx* c, const float* W0, int p, int bits, int gs
                                 float tau, unsigned char* codes, const float* delta, const float* zero,
                                 float* Wq, float* g, long long* d_moves, int* d_capped) {
   const int n = c->n;
-  const size_t smem = (size_t)n * 9 + (size_t)(n / gs) * 8 + 16;
+  const size_t smem = (size_t)n * 5 + (size_t)(n / gs) * 8 + 16;
   const int threads = n >= 8192 ? 512 : 256;               // long rows: more warps per channel
   cudaError_t e = cudaFuncSetAttribute(local_search_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
