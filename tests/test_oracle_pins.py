@@ -74,6 +74,22 @@ def test_move_cost_hand_worked():
 
 
 # ------------------------------------------------------------------ Hessian, damping, scaling
+def test_rho_schedule_is_geometric_with_the_stated_ends():
+    """Sec. 3.6: rho_t = rho_0 gamma^t.  Pinned on the two schedules the workloads use: the paper's default
+    (rho_0 = 0.1, gamma = 1.1, T = 300: the last penalty is 0.1 * 1.1^299) and the 100-step schedule from 1e-2
+    to 1e2 of the small configuration (gamma = 1e4^(1/99)), and on the product workloads.py hands the GPU."""
+    from paper_2605_11222_b200 import workloads as wl
+    r = O.rho_schedule(300, 0.1, 1.1)
+    assert r[0] == 0.1 and len(r) == 300
+    assert np.allclose(r[1:] / r[:-1], 1.1, rtol=1e-14)
+    assert abs(r[-1] / (0.1 * 1.1 ** 299) - 1) < 1e-12 and 2.3e11 < r[-1] < 2.4e11
+    g = 1e4 ** (1.0 / 99)
+    r1 = O.rho_schedule(100, 1e-2, g)
+    assert r1[0] == 1e-2 and abs(r1[-1] - 1e2) < 1e-9 and np.all(np.diff(r1) > 0)
+    for spec in (wl.config1(), wl.config2()):
+        assert np.allclose(np.array(spec.rho()), O.rho_schedule(spec.T, spec.rho0, spec.gamma), rtol=1e-13)
+
+
 def test_hessian_chunked_equals_one_shot_and_entry_definition():
     rng = np.random.default_rng(1)
     X = rng.standard_normal((300, 12))
